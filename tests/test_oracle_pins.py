@@ -1,0 +1,553 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked
+without any GPU.  Each test is chosen so that a plausible slip in the oracle
+(dropped term, wrong sign or index, transposed operand, off-by-one in a budget)
+fails it.  The brute-force routines here are written with plain Python loops and
+`math`, independently of the oracle's numpy code.
+"""
+
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+from scipy.special import softmax as scipy_softmax
+
+from oracle import metok_oracle as O
+from paper_2506_02850_b200 import workloads as W
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.json")
+
+
+# --------------------------------------------------------------------------- #
+# independent brute force (pure Python)
+# --------------------------------------------------------------------------- #
+
+
+def py_cos(a, b):
+    dot = sum(float(x) * float(y) for x, y in zip(a, b))
+    na = max(math.sqrt(sum(float(x) ** 2 for x in a)), 1e-8)
+    nb = max(math.sqrt(sum(float(x) ** 2 for x in b)), 1e-8)
+    return dot / (na * nb)
+
+
+def py_topk_desc(scores, n):
+    """n best (score desc, index asc) by repeated scanning."""
+    left = list(range(len(scores)))
+    picked = []
+    for _ in range(n):
+        best = left[0]
+        for j in left[1:]:
+            if scores[j] > scores[best]:
+                best = j
+        picked.append(best)
+        left.remove(best)
+    return sorted(picked)
+
+
+# --------------------------------------------------------------------------- #
+# P1 / P2: planted events, closed forms (a1, a2)
+# --------------------------------------------------------------------------- #
+
+
+@pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128d1024", "stress"])
+def test_planted_boundaries_recovered(name):
+    cfg = W.CONFIGS[name]
+    vis = W.vision_inputs(cfg)
+    for mode in (O.SIM_FLATTEN, O.SIM_MEANPOOL):
+        if mode == O.SIM_MEANPOOL and (name == "stress" or cfg.near_dup):
+            # averaging the tokens first leaves the 0.98 near-duplicate boundary
+            # at ~0.9985, inside the spread of the within-event values
+            continue
+        seg = O.segment_events(vis["V"], cfg.k, mode)
+        assert np.array_equal(seg["boundaries"], vis["boundaries"]), (name, mode)
+        assert np.array_equal(seg["event_offsets"], vis["event_offsets"])
+        assert seg["frame_event"][0] == 0 and seg["frame_event"][-1] == cfg.k - 1
+        assert np.all(np.diff(seg["frame_event"]) >= 0)
+        if mode == O.SIM_FLATTEN:
+            sims = seg["sims"]
+            inside = np.ones(cfg.T - 1, dtype=bool)
+            inside[vis["boundaries"]] = False
+            # E[cos] of two noisy copies of one base = 1 / (1 + sigma^2)
+            assert abs(sims[inside].mean() - 1.0 / (1.0 + cfg.sigma ** 2)) < 2e-3
+            cross = sims[~inside]
+            if vis["near_dup_boundary"] is not None:
+                b = vis["near_dup_boundary"]
+                assert abs(sims[b] - 0.98) < 5e-3
+                cross = np.delete(sims, np.concatenate([np.nonzero(inside)[0], [b]]))
+            assert np.all(np.abs(cross) < 0.12)
+
+
+def test_similarity_closed_forms():
+    rng = np.random.default_rng(5)
+    a = rng.standard_normal((3, 7))
+    V = np.stack([a, a, 2.5 * a, -a])                      # cos = 1, 1, -1
+    s = O.frame_similarity(V)
+    assert np.allclose(s, [1.0, 1.0, -1.0], atol=1e-12)
+    # orthogonal hand-built frames -> 0 ; 45 degrees -> 1/sqrt(2)
+    e = np.zeros((3, 1, 4))
+    e[0, 0, 0] = 1.0
+    e[1, 0, 1] = 3.0
+    e[2, 0, 1] = 1.0
+    e[2, 0, 2] = 1.0
+    s = O.frame_similarity(e)
+    assert abs(s[0]) < 1e-15 and abs(s[1] - 1 / math.sqrt(2)) < 1e-12
+    # FLATTEN and MEANPOOL differ: tokens that cancel in the mean
+    V2 = np.zeros((2, 2, 2))
+    V2[0] = [[1, 0], [0, 1]]
+    V2[1] = [[0, 1], [1, 0]]                               # Frobenius dot 0, means equal
+    assert abs(O.frame_similarity(V2, O.SIM_FLATTEN)[0]) < 1e-15
+    assert abs(O.frame_similarity(V2, O.SIM_MEANPOOL)[0] - 1.0) < 1e-12
+    # zero frame: clamped norm, finite result
+    V3 = np.zeros((2, 2, 2))
+    V3[1] = 1.0
+    assert O.frame_similarity(V3)[0] == 0.0
+
+
+def test_similarity_against_python_loops():
+    rng = np.random.default_rng(6)
+    V = rng.standard_normal((5, 3, 4))
+    s = O.frame_similarity(V)
+    for i in range(4):
+        assert abs(s[i] - py_cos(V[i].ravel(), V[i + 1].ravel())) < 1e-12
+    sm = O.frame_similarity(V, O.SIM_MEANPOOL)
+    for i in range(4):
+        assert abs(sm[i] - py_cos(V[i].mean(0), V[i + 1].mean(0))) < 1e-12
+
+
+def test_split_events_ties_and_edges():
+    sims = np.array([0.9, 0.1, 0.1, 0.8, 0.1])
+    out = O.split_events(sims, 3)                          # two lowest, lower index first
+    assert out["boundaries"].tolist() == [1, 2]
+    assert out["event_offsets"].tolist() == [0, 2, 3, 6]
+    assert out["frame_event"].tolist() == [0, 0, 1, 2, 2, 2]
+    one = O.split_events(sims, 1)
+    assert one["boundaries"].size == 0 and one["event_offsets"].tolist() == [0, 6]
+    allk = O.split_events(sims, 6)
+    assert allk["event_offsets"].tolist() == [0, 1, 2, 3, 4, 5, 6]
+
+
+@pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128d1024", "stress"])
+def test_planted_relevant_events_become_key(name):
+    cfg = W.CONFIGS[name]
+    vis = W.vision_inputs(cfg)
+    s = O.token_relevance(vis["V"], vis["t"])
+    for agg in (O.AGG_MEAN, O.AGG_MAX):
+        ev = O.key_events(s, cfg.T, cfg.N, vis["event_offsets"], cfg.alpha, agg)
+        assert np.array_equal(np.nonzero(ev["event_is_key"])[0], vis["relevant_events"]), (name, agg)
+    assert ev["event_is_key"].sum() == math.ceil(cfg.alpha * cfg.k)
+
+
+def test_token_relevance_against_python_loops():
+    rng = np.random.default_rng(7)
+    V = rng.standard_normal((2, 3, 5))
+    t = rng.standard_normal(5)
+    s = O.token_relevance(V, t)
+    X = V.reshape(-1, 5)
+    for j in range(6):
+        assert abs(s[j] - py_cos(X[j], t)) < 1e-12
+    # scale invariance and sign
+    assert np.allclose(O.token_relevance(3.0 * V, 0.5 * t), s, atol=1e-12)
+    assert np.allclose(O.token_relevance(V, -t), -s, atol=1e-12)
+
+
+def test_key_events_mean_vs_max_and_ties():
+    # 3 events: frames [0,1], [2], [3,4,5]; N = 1
+    ts = np.array([0.1, 0.9, 0.6, 0.5, 0.5, 0.5])
+    offs = np.array([0, 2, 3, 6])
+    mean = O.key_events(ts, 6, 1, offs, 0.5, O.AGG_MEAN)     # means .5 .6 .5 -> top 2 = {1, 0}
+    assert np.allclose(mean["event_score"], [0.5, 0.6, 0.5])
+    assert mean["event_is_key"].tolist() == [1, 1, 0]        # tie 0 vs 2 -> lower index
+    mx = O.key_events(ts, 6, 1, offs, 0.5, O.AGG_MAX)        # max .9 .6 .5
+    assert np.allclose(mx["event_score"], [0.9, 0.6, 0.5])
+    assert mx["event_is_key"].tolist() == [1, 1, 0]
+    one = O.key_events(ts, 6, 1, offs, 0.3, O.AGG_MAX)       # ceil(.9) = 1
+    assert one["event_is_key"].tolist() == [1, 0, 0]
+
+
+# --------------------------------------------------------------------------- #
+# P6: constants the paper prints
+# --------------------------------------------------------------------------- #
+
+
+def test_printed_key_event_counts_and_schedule():
+    g = json.load(open(GOLDEN))
+    for hp in g["hyperparameters"]:
+        want = g["key_event_counts"][str(hp["k"])]
+        assert min(hp["k"], O.ceilq(hp["alpha"] * hp["k"])) == want
+        ev = O.key_events(np.linspace(0, 1, hp["k"]), hp["k"], 1, np.arange(hp["k"] + 1), hp["alpha"])
+        assert int(ev["event_is_key"].sum()) == want
+    # r = 0.55, alpha = 0.5: Eq. 6 gives 1, r, r^2, 0 and Eq. 7 gives 1, alpha r, 0
+    rk = [O.retention_ratios(0.5, 0.55, s) for s in range(4)]
+    assert rk[0] == (1.0, 1.0)
+    assert abs(rk[1][0] - 0.55) < 1e-7 and abs(rk[1][1] - 0.275) < 1e-7
+    assert abs(rk[2][0] - 0.3025) < 1e-7 and rk[2][1] == 0.0
+    assert rk[3] == (0.0, 0.0)
+    r76 = O.retention_ratios(0.5, 0.76, 2)[0]
+    assert abs(r76 - 0.5776) < 1e-6
+    b = O.retention_budgets(0.5, 0.55, 1, (1000, 2000))
+    assert b.tolist() == [550, 550]
+    b = O.retention_budgets(0.5, 0.55, 2, (1000, 2000))
+    assert b.tolist() == [303, 0]                          # ceil(302.5)
+    assert O.retention_budgets(0.5, 0.55, 3, (1000, 2000)).tolist() == [0, 0]
+    # exact products must not round up: 0.5 * 8 = 4, not 5
+    assert O.ceilq(0.5 * 8) == 4
+    assert O.ceilq(0.3 * 10) == 3 and O.ceilq(0.1 * 3 * 10) == 3   # 3.0000000000000004 is still 3
+    assert O.ceilq(0.065 * 18432) == 1199 and O.ceilq(0.2 * 2304) == 461
+    assert O.event_token_budget(10, 0.25) == 3 and O.event_token_budget(1, 0.01) == 1
+
+
+def test_kv_policy_reproduces_printed_cache_sizes():
+    """Table 3: with visual K/V kept only in layers 0..l1-1 (l1 = 3) and ~80 text
+    tokens kept everywhere, the decode-stage cache is 22.3 / 171.8 of the
+    stage-1 cache.  l1 = 2 or 4 (or 1-based layers) miss it by far."""
+    g = json.load(open(GOLDEN))
+    lay = g["kv_layout_7b"]
+    per_tok = 2 * lay["kv_heads"] * lay["head_dim"] * lay["bytes_per_element"]
+    mb = g["kv_cache_mb_llava_ov_7b"]
+    tok_stage1 = mb["after_vision_encoding"] * 2 ** 20 / (per_tok * lay["layers"])
+    n_text = 80
+    n_vis = int(round(tok_stage1)) - n_text
+    want = mb["after_decoding"] / mb["after_vision_encoding"]
+
+    def ratio(l1):
+        lists = O.kv_select(O.KV_PAPER, lay["layers"], n_vis + n_text, 0, n_vis, l1=l1)
+        full = O.kv_select(O.KV_PAPER, lay["layers"], n_vis + n_text, 0, n_vis, l1=lay["layers"])
+        return O.kv_bytes(lists, lay["kv_heads"], lay["head_dim"], 2) / O.kv_bytes(full, lay["kv_heads"], lay["head_dim"], 2)
+
+    assert abs(ratio(3) - want) < 2e-3
+    assert abs(ratio(2) - want) > 2e-2 and abs(ratio(4) - want) > 2e-2
+    # absolute size in MiB too
+    lists = O.kv_select(O.KV_PAPER, lay["layers"], n_vis + n_text, 0, n_vis, l1=3)
+    assert abs(O.kv_bytes(lists, lay["kv_heads"], lay["head_dim"], 2) / 2 ** 20 - mb["after_decoding"]) < 0.3
+    # Table 2's uncompressed LongVA cache = 128 x 144 visual tokens + ~79 others
+    t2 = g["kv_cache_mb_table2"]
+    tok = t2["longva_base"] * 2 ** 20 / (per_tok * lay["layers"])
+    assert abs(tok - (128 * 144 + 79)) < 2
+
+
+# --------------------------------------------------------------------------- #
+# P3: brute force on tiny inputs (a3, a4, a6)
+# --------------------------------------------------------------------------- #
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_key_token_topk_brute_force(seed):
+    rng = np.random.default_rng(100 + seed)
+    N = int(rng.integers(1, 5))
+    lens = [int(v) for v in rng.integers(1, 5, size=int(rng.integers(1, 5)))]
+    offs = np.concatenate([[0], np.cumsum(lens)])
+    T = int(offs[-1])
+    s = rng.standard_normal(T * N)
+    s[rng.integers(0, T * N, size=T * N // 3)] = 0.25       # force ties
+    is_key = rng.integers(0, 2, size=len(lens)).astype(np.uint8)
+    kk, kn = 0.4, 0.2
+    out = O.key_token_topk(s, N, offs, is_key, kk, kn)
+    want = []
+    for e, ln in enumerate(lens):
+        lo, hi = offs[e] * N, offs[e + 1] * N
+        m = hi - lo
+        ratio = kk if is_key[e] else kn
+        n = min(m, max(1, math.ceil(ratio * m - 1e-9)))
+        assert out["event_budget"][e] == n
+        want += [lo + j for j in py_topk_desc(list(s[lo:hi]), n)]
+    assert out["key_idx"].tolist() == want
+    assert out["is_key_token"].sum() == len(want)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_merge_assign_brute_force(seed):
+    rng = np.random.default_rng(200 + seed)
+    N, d = 3, 5
+    lens = [int(v) for v in rng.integers(1, 4, size=3)]
+    offs = np.concatenate([[0], np.cumsum(lens)])
+    T = int(offs[-1])
+    V = rng.standard_normal((T, N, d))
+    if seed % 2 == 0:
+        V[1] = V[0]                                         # exact duplicate rows: tie -> lower key
+    is_key = np.zeros(T * N, dtype=np.uint8)
+    for e in range(3):
+        lo, hi = offs[e] * N, offs[e + 1] * N
+        pick = rng.choice(np.arange(lo, hi), size=max(1, (hi - lo) // 3), replace=False)
+        is_key[pick] = 1
+    out = O.merge_assign(V, N, offs, is_key, "f32")
+    X = V.reshape(-1, d)
+    keys = [j for j in range(T * N) if is_key[j]]
+    slot = {j: i for i, j in enumerate(keys)}
+    members = {i: [j] for j, i in slot.items()}
+    for e in range(3):
+        lo, hi = offs[e] * N, offs[e + 1] * N
+        ek = [j for j in keys if lo <= j < hi]
+        for a in range(lo, hi):
+            if is_key[a]:
+                assert out["assign"][a] == slot[a]
+                continue
+            best, best_c = None, -2.0
+            for c in ek:                                     # ascending: strict > keeps lower c
+                v = py_cos(X[a], X[c])
+                if v > best_c + 0.0:
+                    if best is None or v > best_c:
+                        best, best_c = c, v
+            assert out["assign"][a] == slot[best], (a, best)
+            members[slot[best]].append(a)
+    assert out["out_src"].tolist() == keys
+    for i, js in members.items():
+        mean = [sum(X[j][c] for j in js) / len(js) for c in range(d)]
+        assert np.allclose(out["out_feats_exact"][i], mean, atol=1e-12)
+        assert out["out_members"][i] == len(js)
+        e = int(np.searchsorted(offs * N, keys[i], side="right") - 1)
+        assert out["out_event"][i] == e
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_weighted_topk_brute_force(seed):
+    rng = np.random.default_rng(300 + seed)
+    n_vis, vis_start, Lt = 23, int(rng.integers(0, 4)), 3
+    S = vis_start + n_vis + Lt
+    s = np.round(rng.standard_normal(n_vis), 1)             # many ties
+    grp = rng.integers(0, 3, size=n_vis).astype(np.int32)
+    budget = [int(rng.integers(0, 12)) for _ in range(3)]
+    out = O.weighted_topk(s, grp, budget, S, vis_start)
+    keep = set(range(vis_start)) | set(range(vis_start + n_vis, S))
+    for g in range(3):
+        idx = [j for j in range(n_vis) if grp[j] == g]
+        n = min(len(idx), budget[g])
+        for r in py_topk_desc([s[j] for j in idx], n):
+            keep.add(vis_start + idx[r])
+    assert out["keep_idx"].tolist() == sorted(keep)
+    assert out["S_out"] == len(keep)
+
+
+# --------------------------------------------------------------------------- #
+# P4: attention scores against textbook routines and closed forms (a5)
+# --------------------------------------------------------------------------- #
+
+
+def test_attention_scores_python_loops():
+    rng = np.random.default_rng(8)
+    Hq, Hkv, Lt, dh, S = 4, 2, 3, 5, 9
+    Q = rng.standard_normal((Hq, Lt, dh))
+    K = rng.standard_normal((Hkv, S, dh))
+    vis_start, n_vis = 1, 4
+    scale = 0.37
+    got = O.attention_scores(Q, K, vis_start, n_vis, scale)
+    sc = float(np.float32(scale))
+    want = [0.0] * n_vis
+    for h in range(Hq):
+        g = h // 2
+        for q in range(Lt):
+            last = S - Lt + q
+            lg = [sc * sum(Q[h, q, c] * K[g, u, c] for c in range(dh)) for u in range(last + 1)]
+            z = sum(math.exp(v) for v in lg)
+            for j in range(n_vis):
+                want[j] += math.exp(lg[vis_start + j]) / z
+    want = [w / (Hq * Lt) for w in want]
+    assert np.allclose(got, want, rtol=1e-12, atol=0)
+
+
+def test_attention_scores_vs_library_softmax_and_mass():
+    rng = np.random.default_rng(9)
+    Hq, Hkv, dh, S = 6, 3, 8, 40
+    Q = rng.standard_normal((Hq, 1, dh))                    # Lt = 1: the query sees all S keys
+    K = rng.standard_normal((Hkv, S, dh))
+    sc = float(np.float32(dh ** -0.5))
+    got = O.attention_scores(Q, K, 0, S - 1, dh ** -0.5)
+    P = np.stack([scipy_softmax(sc * (K[h // 2] @ Q[h, 0])) for h in range(Hq)])
+    assert np.allclose(got, P[:, : S - 1].mean(axis=0), rtol=1e-12)
+    # total probability: visual mass + the text token's own mass = 1
+    assert abs(got.sum() + P[:, S - 1].mean() - 1.0) < 1e-12
+    # transposing the head grouping (h % Hkv instead of h // rep) must change the answer
+    P_wrong = np.stack([scipy_softmax(sc * (K[h % 3] @ Q[h, 0])) for h in range(Hq)])
+    assert not np.allclose(got, P_wrong[:, : S - 1].mean(axis=0), rtol=1e-3)
+
+
+def test_attention_scores_closed_forms():
+    Hq, Hkv, Lt, dh, S = 2, 1, 3, 4, 10
+    K = np.ones((Hkv, S, dh))
+    Q = np.ones((Hq, Lt, dh))
+    # all logits equal: every visible key gets 1/#visible; query q sees S-Lt+q+1 keys
+    got = O.attention_scores(Q, K, 0, S - Lt, 0.5)
+    want = np.mean([1.0 / (S - Lt + q + 1) for q in range(Lt)])
+    assert np.allclose(got, want, rtol=1e-13)
+    # one key with a dominating logit takes all the mass, shifted logits do not overflow
+    K2 = np.zeros((Hkv, S, dh))
+    K2[0, 3] = 500.0
+    got = O.attention_scores(Q, K2, 0, S - Lt, 1.0)
+    assert abs(got[3] - 1.0) < 1e-12 and abs(got.sum() - 1.0) < 1e-12
+    # a later text token is invisible to earlier queries: key S-1 only to the last query
+    K3 = np.zeros((Hkv, S, dh))
+    K3[0, S - 1] = 500.0
+    got = O.attention_scores(Q, K3, 0, S - Lt, 1.0)
+    q_see = [1.0 / (S - Lt + q + 1) for q in range(Lt - 1)] + [0.0]
+    assert np.allclose(got, np.mean(q_see), rtol=1e-12)
+
+
+# --------------------------------------------------------------------------- #
+# P5: invariants on a mid-size random case and on the tiny config
+# --------------------------------------------------------------------------- #
+
+
+def test_compress_vision_invariants():
+    cfg = W.CONFIGS["frames32"]
+    vis = W.vision_inputs(cfg)
+    V = vis["V"][:12, :36]                                   # 12 frames x 36 tokens
+    offs = np.array([0, 3, 4, 9, 12])
+    out = O.compress_vision(V, vis["t"], offs, 0.5, 0.3, 0.1, "bf16")
+    T, N, d = V.shape
+    X = V.reshape(-1, d).astype(np.float64)
+    n_out = out["n_out"]
+    assert n_out == int(out["event_budget"].sum()) == out["key_idx"].size
+    assert out["out_members"].sum() == T * N and out["out_members"].min() >= 1
+    assert np.all(np.diff(out["out_src"]) > 0)
+    tok_event = np.repeat(np.searchsorted(offs, np.arange(T), side="right") - 1, N)
+    assert np.array_equal(out["out_event"][out["assign"]], tok_event)       # stays in its own event
+    assert np.array_equal(out["assign"][out["out_src"]], np.arange(n_out))
+    for e in range(4):                                        # mass conservation per event
+        sl = out["out_event"] == e
+        lhs = (out["out_members"][sl, None] * out["out_feats_exact"][sl]).sum(axis=0)
+        assert np.allclose(lhs, X[tok_event == e].sum(axis=0), atol=1e-9)
+    for c in range(n_out):                                    # convex combination
+        mem = X[out["assign"] == c]
+        assert np.all(out["out_feats_exact"][c] <= mem.max(axis=0) + 1e-12)
+        assert np.all(out["out_feats_exact"][c] >= mem.min(axis=0) - 1e-12)
+    # output rounding: representable in bf16 and within half an ulp
+    r = out["out_feats"]
+    assert np.array_equal(W.round_to_bf16(r.astype(np.float32)).astype(np.float64), r)
+    assert np.all(np.abs(r - out["out_feats_exact"]) <= np.abs(out["out_feats_exact"]) * 2.0 ** -8 + 1e-300)
+
+
+def test_round_bf16_matches_bit_level_rounding():
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal(20000).astype(np.float32) * np.float32(3.0)
+    x[:4] = [1.00390625, 1.01171875, -1.00390625, 0.0]        # exact ties -> even
+    assert np.array_equal(O.round_bf16(x.astype(np.float64)), W.round_to_bf16(x).astype(np.float64))
+
+
+def test_keep_ratio_one_is_identity_and_k1():
+    cfg = W.CONFIGS["tiny"]
+    vis = W.vision_inputs(cfg)
+    seg = O.segment_events(vis["V"], 1)
+    assert seg["event_offsets"].tolist() == [0, cfg.T]
+    out = O.compress_vision(vis["V"], vis["t"], seg["event_offsets"], 0.5, 1.0, 1.0, "f32")
+    assert out["n_out"] == cfg.Nv and np.all(out["out_members"] == 1)
+    assert np.array_equal(out["assign"], np.arange(cfg.Nv))
+    assert np.array_equal(out["out_feats"], vis["V"].reshape(cfg.Nv, cfg.d).astype(np.float64))
+
+
+def test_prefill_prune_invariants_and_budget_zero():
+    cfg = W.CONFIGS["tiny"]
+    vis = W.vision_inputs(cfg)
+    grp = W.token_groups(cfg, cfg.Nv, vis=vis)
+    pf = W.prefill_inputs(cfg, 1, cfg.Nv, grp, vis_start=2)
+    S = pf["S"]
+    hidden = W.payload_rows_np(W.hidden_salt(cfg, 1), np.arange(S), cfg.D, "f32")
+    N0 = [int((grp == 0).sum()), int((grp == 1).sum())]
+    for stage in (1, 2, 3):
+        b = O.retention_budgets(cfg.alpha, cfg.keep_prefill, stage, N0)
+        out = O.prefill_prune(pf["Q"], pf["K"], hidden, 2, cfg.Nv, grp, b, cfg.dh ** -0.5)
+        keep = out["keep_idx"]
+        assert np.all(np.diff(keep) > 0)
+        assert out["S_out"] == 2 + cfg.Lt + int(b.sum())       # survivors = the schedule's budget
+        assert set(range(2)) <= set(keep.tolist()) and set(range(S - cfg.Lt, S)) <= set(keep.tolist())
+        kept_vis = keep[(keep >= 2) & (keep < 2 + cfg.Nv)] - 2
+        for g in (0, 1):
+            assert int((grp[kept_vis] == g).sum()) == b[g]
+        assert np.array_equal(out["hidden_out"], hidden[keep])
+        if stage == 3:
+            assert kept_vis.size == 0
+    # every kept visual token of a class scores at least as high as every dropped one of that class
+    b = O.retention_budgets(cfg.alpha, cfg.keep_prefill, 1, N0)
+    out = O.prefill_prune(pf["Q"], pf["K"], hidden, 2, cfg.Nv, grp, b, cfg.dh ** -0.5)
+    kept = np.zeros(cfg.Nv, dtype=bool)
+    kv = out["keep_idx"][(out["keep_idx"] >= 2) & (out["keep_idx"] < 2 + cfg.Nv)] - 2
+    kept[kv] = True
+    for g in (0, 1):
+        m = grp == g
+        assert out["scores"][m & kept].min() >= out["scores"][m & ~kept].max()
+
+
+def test_planted_relevance_separates_classes():
+    """The planted rank-1 component must make attention scores informative:
+    key-event tokens score higher on average, and the spread is far outside the
+    near-tie band (otherwise index parity would test nothing)."""
+    cfg = W.CONFIGS["frames32"]
+    n_vis = 600
+    grp = W.token_groups(cfg, n_vis, n_key=300)
+    pf = W.prefill_inputs(cfg, 1, n_vis, grp)
+    a = O.attention_scores(pf["Q"], pf["K"], 0, n_vis, cfg.dh ** -0.5)
+    assert a[grp == 0].mean() > 1.5 * a[grp == 1].mean()
+    assert a.std() / a.mean() > 0.5
+    flat = W.prefill_inputs(cfg, 1, n_vis, grp, planted=False)
+    a0 = O.attention_scores(flat["Q"], flat["K"], 0, n_vis, cfg.dh ** -0.5)
+    assert a0.std() / a0.mean() < 0.2
+
+
+# --------------------------------------------------------------------------- #
+# a8 / a9: KV selection and compaction
+# --------------------------------------------------------------------------- #
+
+
+def test_kv_policies_and_compaction():
+    cfg = W.CONFIGS["tiny"]
+    L, Hkv, S, dh = 3, 2, 20, 4
+    n_vis, vis_start = 14, 2
+    rng = np.random.default_rng(12)
+    ks = [rng.integers(0, 1000, size=(Hkv, S, dh)).astype(np.float32) for _ in range(L)]
+    vs = [rng.integers(0, 1000, size=(Hkv, S, dh)).astype(np.float32) for _ in range(L)]
+    paper = O.kv_select(O.KV_PAPER, L, S, vis_start, n_vis, l1=1)
+    assert paper[0].tolist() == list(range(S))
+    assert paper[1].tolist() == [0, 1, 16, 17, 18, 19] == paper[2].tolist()
+    sc = rng.standard_normal((L, n_vis))
+    topk = O.kv_select(O.KV_TOPK, L, S, vis_start, n_vis, keep_ratio=0.3, scores=sc)
+    for layer in range(L):
+        want = sorted([0, 1, 16, 17, 18, 19] + [vis_start + j for j in py_topk_desc(list(sc[layer]), 5)])
+        assert topk[layer].tolist() == want                    # ceil(0.3*14) = 5
+    shared = O.kv_select(O.KV_TOPK, L, S, vis_start, n_vis, keep_ratio=0.3, scores=sc[0])
+    assert all(np.array_equal(s_, topk[0]) for s_ in shared)
+    nk, nv, nl = O.kv_compact(ks, vs, topk)
+    assert nl.tolist() == [11, 11, 11]
+    for layer in range(L):
+        for h in range(Hkv):
+            for i, src in enumerate(topk[layer]):
+                assert np.array_equal(nk[layer][h, i], ks[layer][h, src])
+                assert np.array_equal(nv[layer][h, i], vs[layer][h, src])
+    # no text rows at all (the tiny configuration's cache): only visual survivors remain
+    only = O.kv_select(O.KV_TOPK, 1, n_vis, 0, n_vis, keep_ratio=0.5, scores=sc[0])
+    assert len(only[0]) == 7
+    none = O.kv_select(O.KV_PAPER, 1, n_vis, 0, n_vis, l1=0)
+    assert len(none[0]) == 0
+    assert O.kv_bytes(topk, Hkv, dh, 2) == 33 * 2 * Hkv * dh * 2
+
+
+# --------------------------------------------------------------------------- #
+# the paper's own stage-1 compressor: key frames and adaptive pooling
+# --------------------------------------------------------------------------- #
+
+
+def test_pool2d_and_adaptive_pool():
+    g = np.arange(16, dtype=np.float64).reshape(16, 1)          # 4x4 grid, d = 1
+    p = O.pool2d(g, 4, 2)
+    assert p.ravel().tolist() == [2.5, 4.5, 10.5, 12.5]
+    p3 = O.pool2d(g, 4, 3)                                       # clipped edge windows
+    assert p3.shape == (4, 1)
+    assert p3.ravel().tolist() == [5.0, 7.0, 13.0, 15.0]
+    assert O.pool2d(g, 4, 1).ravel().tolist() == list(range(16))
+    # divisible grid conserves the frame mean
+    rng = np.random.default_rng(13)
+    f = rng.standard_normal((144, 3))
+    for s in (2, 3, 4, 6):
+        assert np.allclose(O.pool2d(f, 12, s).mean(axis=0), f.mean(axis=0), atol=1e-12)
+    # key frames: ceil(beta * len) best per event
+    fs = np.array([.1, .5, .3, .9, .2, .2, .2])
+    kf = O.key_frames(fs, np.array([0, 3, 7]), 0.4)              # ceil(1.2)=2 of 3 ; ceil(1.6)=2 of 4
+    assert kf.tolist() == [0, 1, 1, 1, 1, 0, 0]
+    # strides (2,3) in key events become (4,6) in non-key events with alpha = 0.5
+    cfg = W.CONFIGS["frames32"]
+    vis = W.vision_inputs(cfg)
+    out = O.adaptive_pool(vis["V"][:, :, :32], vis["t"][:32], vis["event_offsets"], 0.5, 0.45,
+                          (2, 3, 4, 6), "bf16")
+    per = {2: 36, 3: 16, 4: 9, 6: 4}
+    assert out["n_out"] == sum(per[int(s)] for s in out["frame_stride"])
+    assert np.all(np.diff(out["out_frame"]) >= 0)
+    ek = np.repeat(out["event_is_key"], np.diff(vis["event_offsets"]))
+    assert set(out["frame_stride"][ek == 1]) <= {2, 3} and set(out["frame_stride"][ek == 0]) <= {4, 6}

@@ -1,0 +1,252 @@
+/*
+ * metok.h -- C ABI of the METok hot path for NVIDIA B200 (sm_100a).
+ *
+ * METok ("Multi-Stage Event-based Token Compression", arXiv 2506.02850) removes
+ * visual tokens of a long video in three places: after the vision encoder
+ * (event segmentation + event-aware reduction, section 3.2.1 and Algorithm 1),
+ * inside LLM prefill (hierarchical pruning by text->visual attention and event
+ * importance, section 3.2.2, Eq. 6 and 7) and in the decode-time KV cache
+ * (section 3.3).  This library is the data-parallel part of that pipeline; the
+ * vision tower, text encoder and LLM layers belong to the caller.
+ *
+ * Conventions shared by every entry point
+ *   - Return value: METOK_OK or a negative METOK_ERR_* code.  Nothing throws,
+ *     aborts or prints.  Arguments are validated on the host before anything is
+ *     launched; a call that fails validation launches nothing.
+ *   - Pointers named in the argument comments as DEVICE point to memory of the
+ *     current CUDA device, owned by the caller, 16-byte aligned, row-major and
+ *     contiguous.  HOST pointers are ordinary host memory read during the call.
+ *   - The library never allocates device memory.
+ *     Scratch comes from a caller workspace `ws` of at least
+ *     metok_*_workspace_bytes(...) bytes (pure host functions).  Its contents
+ *     are undefined afterwards; two calls that overlap on the GPU must not
+ *     share a workspace.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream) and the call returns without synchronising.
+ *     Outputs, including device-resident counts, are valid once the caller has
+ *     synchronised with the stream.
+ *   - Inputs are never written, except the K/V buffers of metok_kv_compact.
+ *   - dtype: METOK_F32 (float) or METOK_BF16 (bfloat16).  bf16 paths accumulate
+ *     in fp32; selections compare fp32 scores; ties always go to the lower index.
+ *   - Ratios are doubles; every count derived from a ratio is
+ *     ceil(ratio * population - 1e-9) evaluated in double.
+ *   - Token index j = f*N + p for frame f and position p.
+ */
+#ifndef METOK_H_
+#define METOK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define METOK_API __attribute__((visibility("default")))
+#else
+#define METOK_API
+#endif
+
+#define METOK_OK               0
+#define METOK_ERR_INVALID_ARG (-1)  /* null pointer, size out of range, bad ratio, misaligned pointer */
+#define METOK_ERR_UNSUPPORTED (-2)  /* well-formed, but outside the compiled shapes / dtypes */
+#define METOK_ERR_WORKSPACE   (-3)  /* ws is NULL or smaller than *_workspace_bytes */
+#define METOK_ERR_CUDA        (-4)  /* a launch or driver call failed; see metok_last_cuda_error */
+#define METOK_ERR_TIMEOUT     (-5)  /* a bounded device-side wait gave up (reported via status words) */
+
+#define METOK_F32  0
+#define METOK_BF16 1
+
+#define METOK_SIM_FLATTEN  0   /* Frobenius inner product of the N x d frame matrices */
+#define METOK_SIM_MEANPOOL 1   /* average the N tokens first, then cosine in R^d      */
+
+#define METOK_AGG_MEAN 0       /* event score = mean of its frame scores (section 3.2.1, body text) */
+#define METOK_AGG_MAX  1       /* event score = max of its frame scores (Algorithm 1)               */
+
+#define METOK_MODE_TOPK_MERGE 0  /* per-event key-token top-k + merge of the rest      */
+#define METOK_MODE_POOL       1  /* Algorithm 1: key frames + adaptive 2-D pooling     */
+
+#define METOK_KV_PAPER 0       /* section 3.3: drop every visual position from layer l1 on */
+#define METOK_KV_TOPK  1       /* keep the ceil(ratio*n_vis) best-scored visual tokens per layer */
+#define METOK_KV_GIVEN 2       /* the caller supplies the keep lists */
+
+#define METOK_MAX_GROUPS 64
+
+/* ------------------------------------------------------------------------- *
+ * (1) Temporal event segmentation -- Eq. 4 and the paragraph after it;
+ *     Algorithm 1, "Event temporal segmentation".
+ *
+ *   sims[i] = cos(v_i, v_{i+1}),  i = 0 .. T-2   (T-1 adjacent pairs)
+ *   boundaries = the k-1 smallest sims (lower i first on ties), ascending;
+ *                boundary b splits between frame b and b+1
+ *   event_offsets = [0, b_1+1, ..., T]  (CSR over frames, k+1 entries)
+ *   frame_event[f] = event of frame f
+ *
+ *   feats        DEVICE [T][N][d] of `dtype`              (input)
+ *   sims         DEVICE float [max(T-1,1)]                (output)
+ *   boundaries   DEVICE int32 [max(k-1,1)]                (output)
+ *   event_offsets DEVICE int32 [k+1]                      (output)
+ *   frame_event  DEVICE int32 [T]                         (output)
+ *
+ *   Norms are clamped below by 1e-8.  There is no minimum event length.
+ *   Errors: INVALID_ARG for null/misaligned pointers, T,N,d < 1, k < 1, k > T,
+ *   unknown sim_mode or dtype; UNSUPPORTED if d*sizeof(elem) is not a multiple
+ *   of 16 or T > 8192; WORKSPACE if ws is too small.
+ * ------------------------------------------------------------------------- */
+METOK_API size_t metok_segment_events_workspace_bytes(int dtype, int T, int N, int d, int sim_mode);
+METOK_API int metok_segment_events(const void* feats, int dtype, int T, int N, int d, int k, int sim_mode,
+                         float* sims, int32_t* boundaries, int32_t* event_offsets,
+                         int32_t* frame_event, void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * (2) Event-aware token reduction after the vision encoder -- Eq. 5 and
+ *     section 3.2.1 ("Key Visual-Text Semantic Identification", "Adaptive
+ *     Pooling Strategy"); Algorithm 1.
+ *
+ *   token_score[j] = cos(x_j, t)                       (Eq. 5, read per token)
+ *   frame_score[f] = mean of its N token scores
+ *   event_score[e] = mean (or max) of its frame scores
+ *   event_is_key   = the ceil(alpha*k) best events
+ *
+ *   mode TOPK_MERGE: in event e with m_e tokens the
+ *     k_e = min(m_e, max(1, ceil(keep*m_e))) best-scored tokens are key tokens
+ *     (keep = keep_key for key events, keep_nonkey otherwise); every other token
+ *     of the event joins the key token of the same event with which it has the
+ *     highest cosine similarity; output token = plain mean, in feature space, of
+ *     a key token and the tokens that joined it.  Outputs are ordered by the
+ *     key token's index.
+ *   mode POOL (Algorithm 1): per event the ceil(beta*len) best-scored frames are
+ *     key frames; every frame's G x G token grid (G*G = N) is average-pooled with
+ *     window = stride = s1 / s2 (key / other frames of key events) or
+ *     s1_nonkey / s2_nonkey (non-key events); edge windows average the cells
+ *     that exist; pooled frames are appended in temporal order.
+ *
+ *   feats         DEVICE [T][N][d]                       (input)
+ *   event_offsets DEVICE int32 [k+1] (from metok_segment_events)  (input)
+ *   text_emb      DEVICE [d] of `dtype`                  (input)
+ *   p             HOST   parameters                      (input)
+ *   out_feats     DEVICE [cap][d] of `dtype`             (output; rows >= *n_out untouched)
+ *   out_src       DEVICE int32 [cap]  TOPK_MERGE: index of the key token;
+ *                                     POOL: index of the window's first token
+ *   out_event     DEVICE int32 [cap]  event of the output token
+ *   out_members   DEVICE int32 [cap]  number of input tokens averaged (>= 1)
+ *   assign        DEVICE int32 [T*N]  output row that each input token went into
+ *   token_score   DEVICE float [T*N]; frame_score DEVICE float [T];
+ *   event_score   DEVICE float [k];   event_is_key DEVICE uint8 [k]
+ *   n_out         DEVICE int32 scalar: number of output tokens
+ *   cap           rows available in the out_* arrays; must be at least
+ *                 metok_compress_vision_bound(T, N, k, p)
+ *
+ *   Errors: INVALID_ARG (null/misaligned pointers, sizes < 1, k > T, alpha/keep/
+ *   beta outside (0,1], strides < 1, N not a square in POOL mode, cap too small);
+ *   UNSUPPORTED (row bytes not a multiple of 16); WORKSPACE.
+ * ------------------------------------------------------------------------- */
+typedef struct metok_vision_params {
+    double alpha;        /* key-event ratio, (0,1]                              */
+    int    event_agg;    /* METOK_AGG_*                                         */
+    int    mode;         /* METOK_MODE_*                                        */
+    double keep_key;     /* TOPK_MERGE: key-token ratio in key events, (0,1]    */
+    double keep_nonkey;  /* TOPK_MERGE: key-token ratio in non-key events       */
+    double beta;         /* POOL: key-frame ratio, (0,1]                        */
+    int    s1, s2;       /* POOL: strides of key / other frames in key events   */
+    int    s1_nonkey, s2_nonkey;  /* POOL: the same for non-key events (the paper: s/alpha) */
+} metok_vision_params;
+
+METOK_API int    metok_compress_vision_bound(int T, int N, int k, const metok_vision_params* p);
+METOK_API size_t metok_compress_vision_workspace_bytes(int dtype, int T, int N, int d, int k, int cap,
+                                             const metok_vision_params* p);
+METOK_API int metok_compress_vision(const void* feats, int dtype, int T, int N, int d,
+                          const int32_t* event_offsets, int k, const void* text_emb,
+                          const metok_vision_params* p,
+                          void* out_feats, int32_t* out_src, int32_t* out_event,
+                          int32_t* out_members, int32_t* assign, float* token_score,
+                          float* frame_score, float* event_score, uint8_t* event_is_key,
+                          int32_t* n_out, int cap, void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * (3) One level of hierarchical token pruning during prefill -- section 3.2.2,
+ *     Eq. 6 and 7; attention form and scale of Eq. 2.
+ *
+ *   The sequence has S positions; the visual tokens occupy
+ *   [vis_start, vis_start + n_vis), the Lt text queries are the LAST Lt positions.
+ *   scores[j] = mean over all Hq heads h and Lt text queries q of
+ *               softmax_u( Q[h][q] . K[g(h)][u] * softmax_scale )[vis_start + j],
+ *   the softmax taken over the keys query q may see, u <= S - Lt + q (causal);
+ *   g(h) = h / (Hq / Hkv).
+ *   Visual token j has a class token_group[j] in [0, G).  In class g the
+ *   min(population, group_budget[g]) best-scored tokens survive; every
+ *   non-visual position survives.  keep_idx lists the surviving positions in
+ *   ascending order, *S_out is their number, and
+ *   hidden_out[i] = hidden[keep_idx[i]].
+ *
+ *   q_text       DEVICE [Hq][Lt][dh]        k_all  DEVICE [Hkv][S][dh]
+ *   hidden       DEVICE [S][D]              (may be NULL with hidden_out NULL: no gather)
+ *   token_group  DEVICE int32 [n_vis]
+ *   group_budget HOST   int32 [G]  (from metok_retention_budgets, or any counts >= 0;
+ *                                   a budget above the population is clamped)
+ *   scores       DEVICE float [n_vis]       keep_idx DEVICE int32 [S]
+ *   S_out        DEVICE int32 scalar        hidden_out DEVICE [S][D] capacity
+ *
+ *   Errors: INVALID_ARG (null/misaligned, sizes < 1, Hq % Hkv != 0, Lt > S,
+ *   visual span outside [0, S-Lt], G outside [1, METOK_MAX_GROUPS], negative
+ *   budget); UNSUPPORTED (dh not in {64,128} for bf16, dh > 128 or dh % 4 for f32,
+ *   D*sizeof(elem) % 16 != 0); WORKSPACE.
+ * ------------------------------------------------------------------------- */
+METOK_API size_t metok_prefill_prune_workspace_bytes(int dtype, int Hq, int Hkv, int Lt, int S, int dh, int n_vis);
+METOK_API int metok_prefill_prune(const void* q_text, const void* k_all, const void* hidden, int dtype,
+                        int Hq, int Hkv, int Lt, int S, int dh, int D, int vis_start, int n_vis,
+                        const int32_t* token_group, int G, const int32_t* group_budget,
+                        float softmax_scale, float* scores, int32_t* keep_idx, int32_t* S_out,
+                        void* hidden_out, void* ws, size_t ws_bytes, void* stream);
+
+/* Eq. 6 and 7: token budgets after pruning level `stage` (1, 2, 3 = layers l1,
+ * l2, l3; 0 = before l1) for N0 = {key-event tokens, non-key-event tokens}
+ * first passed into the LLM:  R_key = 1, r, r^2, 0 ;  R_nonkey = 1, alpha*r, 0, 0.
+ * (The equations leave l = l3 and l = l2 unassigned; both take the next case.)
+ * HOST pointers.  budget[g] = min(N0[g], ceil(R_g * N0[g] - 1e-9)). */
+METOK_API int metok_retention_budgets(double alpha, double r, int stage, const int32_t* N0, int32_t* budget);
+
+/* ------------------------------------------------------------------------- *
+ * (4) KV-cache selection and in-place compaction -- section 3.3.
+ *
+ *   For every layer l a keep list (ascending positions < S_cur) is chosen:
+ *     PAPER: layers l < l1 keep everything; layers l >= l1 drop all visual
+ *            positions [vis_start, vis_start+n_vis) (0-based layers);
+ *     TOPK : keep the ceil(keep_ratio*n_vis) best-scored visual tokens and all
+ *            non-visual positions (scores shared by all layers, or one row per layer);
+ *     GIVEN: keep_idx / keep_len are inputs.
+ *   Then, for K and V of every layer and every head h,
+ *     X[l][h][i][:] = X[l][h][keep_idx[l][i]][:]   for i < keep_len[l], in place;
+ *   rows at and beyond the new length are unspecified afterwards.
+ *
+ *   k_layers, v_layers HOST arrays of L DEVICE pointers, each [Hkv][S_cap][dh]
+ *   scores    DEVICE float [n_vis] or [L][n_vis] (TOPK), else NULL
+ *   keep_idx  DEVICE int32 [L][S_cur]; keep_len DEVICE int32 [L]
+ *             (outputs for PAPER / TOPK, inputs for GIVEN)
+ *   new_len   DEVICE int32 [L] (output; equals keep_len)
+ *
+ *   A GIVEN list that is not strictly ascending or reaches S_cur gives undefined
+ *   cache contents (lists are not validated on the device).
+ *   Errors: INVALID_ARG (null/misaligned, sizes < 1, S_cur > S_cap, span outside
+ *   [0,S_cur], ratio outside [0,1], l1 < 0, unknown policy); UNSUPPORTED
+ *   (dh*sizeof(elem) % 16 != 0); WORKSPACE.
+ * ------------------------------------------------------------------------- */
+METOK_API size_t metok_kv_compact_workspace_bytes(int dtype, int L, int Hkv, int S_cur, int dh, int policy, int n_vis);
+METOK_API int metok_kv_compact(void* const* k_layers, void* const* v_layers, int dtype, int L, int Hkv,
+                     int S_cap, int S_cur, int dh, int policy, int l1, double keep_ratio,
+                     int vis_start, int n_vis, const float* scores, int scores_per_layer,
+                     int32_t* keep_idx, int32_t* keep_len, int32_t* new_len,
+                     void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * helpers (host only, no CUDA work)
+ * ------------------------------------------------------------------------- */
+METOK_API const char* metok_status_string(int status);
+METOK_API int metok_last_cuda_error(void);   /* cudaError_t of the last METOK_ERR_CUDA on this thread, else 0 */
+METOK_API int metok_version(void);           /* major*10000 + minor*100 + patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* METOK_H_ */

@@ -1,0 +1,267 @@
+"""Thin ctypes binding of ``libmetok.so``: argument marshalling only.
+
+Every function here has the name of the C entry point it calls
+(``include/metok.h``), allocates the output tensors and the workspace with
+torch, passes raw device pointers and the current CUDA stream, and returns the
+outputs.  Nothing is computed in Python and there is no fallback: if the
+library is missing, or a call returns an error status, an exception is raised.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "lib", "libmetok.so")
+
+F32, BF16 = 0, 1
+SIM_FLATTEN, SIM_MEANPOOL = 0, 1
+AGG_MEAN, AGG_MAX = 0, 1
+MODE_TOPK_MERGE, MODE_POOL = 0, 1
+KV_PAPER, KV_TOPK, KV_GIVEN = 0, 1, 2
+
+_c = ctypes
+_vp, _i, _sz, _f, _d = _c.c_void_p, _c.c_int, _c.c_size_t, _c.c_float, _c.c_double
+
+
+class VisionParams(_c.Structure):
+    _fields_ = [("alpha", _d), ("event_agg", _i), ("mode", _i), ("keep_key", _d), ("keep_nonkey", _d),
+                ("beta", _d), ("s1", _i), ("s2", _i), ("s1_nonkey", _i), ("s2_nonkey", _i)]
+
+
+class MetokError(RuntimeError):
+    def __init__(self, fn: str, status: int, text: str, cuda_error: int = 0):
+        self.status = status
+        self.cuda_error = cuda_error
+        extra = f" (cudaError {cuda_error})" if cuda_error else ""
+        super().__init__(f"{fn} failed: {status} {text}{extra}")
+
+
+_SIGNATURES = {
+    "metok_segment_events_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
+    "metok_segment_events": (_i, [_vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "metok_compress_vision_bound": (_i, [_i, _i, _i, _c.POINTER(VisionParams)]),
+    "metok_compress_vision_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _c.POINTER(VisionParams)]),
+    "metok_compress_vision": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _vp, _c.POINTER(VisionParams),
+                                   _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
+    "metok_prefill_prune_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
+    "metok_prefill_prune": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i,
+                                 _c.POINTER(_c.c_int32), _f, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "metok_retention_budgets": (_i, [_d, _d, _i, _c.POINTER(_c.c_int32), _c.POINTER(_c.c_int32)]),
+    "metok_kv_compact_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
+    "metok_kv_compact": (_i, [_c.POINTER(_vp), _c.POINTER(_vp), _i, _i, _i, _i, _i, _i, _i, _i, _d, _i, _i,
+                              _vp, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "metok_status_string": (_c.c_char_p, [_i]),
+    "metok_last_cuda_error": (_i, []),
+    "metok_version": (_i, []),
+}
+
+_lib_handle = None
+
+
+def exported_symbols() -> List[str]:
+    return list(_SIGNATURES)
+
+
+def lib():
+    """Loads the CUDA library on first use; there is no other implementation."""
+    global _lib_handle
+    if _lib_handle is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2506_02850_b200.build` "
+                "(the METok hot path has no CPU or PyTorch fallback)")
+        h = _c.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(h, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib_handle = h
+    return _lib_handle
+
+
+def _check(fn: str, status: int) -> None:
+    if status != 0:
+        L = lib()
+        raise MetokError(fn, status, L.metok_status_string(status).decode(), L.metok_last_cuda_error())
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else _vp(t.data_ptr())
+
+
+def _stream() -> _vp:
+    return _vp(torch.cuda.current_stream().cuda_stream)
+
+
+def _cuda_contig(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t
+
+
+_ws_cache: Dict[tuple, torch.Tensor] = {}
+
+
+def workspace(nbytes: int, device) -> torch.Tensor:
+    """A reusable scratch buffer per device (calls on one stream never overlap)."""
+    key = (str(device),)
+    buf = _ws_cache.get(key)
+    if buf is None or buf.numel() < nbytes:
+        buf = torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=device)
+        _ws_cache[key] = buf
+    return buf
+
+
+# --------------------------------------------------------------------------- #
+
+
+def metok_segment_events(feats: torch.Tensor, k: int, sim_mode: int = SIM_FLATTEN) -> Dict[str, torch.Tensor]:
+    feats = _cuda_contig(feats, "feats")
+    T, N, d = feats.shape
+    dev = feats.device
+    L = lib()
+    sims = torch.empty(max(T - 1, 1), dtype=torch.float32, device=dev)
+    boundaries = torch.empty(max(k - 1, 1), dtype=torch.int32, device=dev)
+    offsets = torch.empty(max(k + 1, 2), dtype=torch.int32, device=dev)
+    frame_event = torch.empty(T, dtype=torch.int32, device=dev)
+    need = L.metok_segment_events_workspace_bytes(_dt(feats), T, N, d, sim_mode)
+    ws = workspace(need, dev)
+    st = L.metok_segment_events(_ptr(feats), _dt(feats), T, N, d, k, sim_mode, _ptr(sims), _ptr(boundaries),
+                                _ptr(offsets), _ptr(frame_event), _ptr(ws), ws.numel(), _stream())
+    _check("metok_segment_events", st)
+    return {"sims": sims[: T - 1], "boundaries": boundaries[: max(k - 1, 0)], "event_offsets": offsets[: k + 1],
+            "frame_event": frame_event}
+
+
+def vision_params(alpha: float, keep_key: float = 1.0, keep_nonkey: float = 1.0, event_agg: int = AGG_MEAN,
+                  mode: int = MODE_TOPK_MERGE, beta: float = 0.5, s1: int = 2, s2: int = 3,
+                  s1_nonkey: int = 4, s2_nonkey: int = 6) -> VisionParams:
+    return VisionParams(alpha, event_agg, mode, keep_key, keep_nonkey, beta, s1, s2, s1_nonkey, s2_nonkey)
+
+
+def metok_compress_vision_bound(T: int, N: int, k: int, p: VisionParams) -> int:
+    b = lib().metok_compress_vision_bound(T, N, k, _c.byref(p))
+    if b < 0:
+        _check("metok_compress_vision_bound", b)
+    return b
+
+
+def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text_emb: torch.Tensor,
+                          p: VisionParams, cap: Optional[int] = None) -> Dict[str, torch.Tensor]:
+    feats = _cuda_contig(feats, "feats")
+    event_offsets = _cuda_contig(event_offsets, "event_offsets")
+    text_emb = _cuda_contig(text_emb, "text_emb")
+    T, N, d = feats.shape
+    k = event_offsets.numel() - 1
+    dev = feats.device
+    L = lib()
+    if cap is None:
+        cap = metok_compress_vision_bound(T, N, k, p)
+    i32 = dict(dtype=torch.int32, device=dev)
+    out = {
+        "out_feats": torch.empty((cap, d), dtype=feats.dtype, device=dev),
+        "out_src": torch.empty(cap, **i32), "out_event": torch.empty(cap, **i32),
+        "out_members": torch.empty(cap, **i32), "assign": torch.empty(T * N, **i32),
+        "token_score": torch.empty(T * N, dtype=torch.float32, device=dev),
+        "frame_score": torch.empty(T, dtype=torch.float32, device=dev),
+        "event_score": torch.empty(k, dtype=torch.float32, device=dev),
+        "event_is_key": torch.empty(k, dtype=torch.uint8, device=dev),
+        "n_out": torch.zeros(1, **i32),
+    }
+    need = L.metok_compress_vision_workspace_bytes(_dt(feats), T, N, d, k, cap, _c.byref(p))
+    ws = workspace(need, dev)
+    st = L.metok_compress_vision(_ptr(feats), _dt(feats), T, N, d, _ptr(event_offsets), k, _ptr(text_emb),
+                                 _c.byref(p), _ptr(out["out_feats"]), _ptr(out["out_src"]), _ptr(out["out_event"]),
+                                 _ptr(out["out_members"]), _ptr(out["assign"]), _ptr(out["token_score"]),
+                                 _ptr(out["frame_score"]), _ptr(out["event_score"]), _ptr(out["event_is_key"]),
+                                 _ptr(out["n_out"]), cap, _ptr(ws), ws.numel(), _stream())
+    _check("metok_compress_vision", st)
+    return out
+
+
+def metok_retention_budgets(alpha: float, r: float, stage: int, N0: Sequence[int]) -> List[int]:
+    n0 = (_c.c_int32 * 2)(int(N0[0]), int(N0[1]))
+    out = (_c.c_int32 * 2)()
+    _check("metok_retention_budgets", lib().metok_retention_budgets(alpha, r, stage, n0, out))
+    return [int(out[0]), int(out[1])]
+
+
+def metok_prefill_prune(q_text: torch.Tensor, k_all: torch.Tensor, hidden: Optional[torch.Tensor], vis_start: int,
+                        n_vis: int, token_group: torch.Tensor, group_budget: Sequence[int], softmax_scale: float,
+                        out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    q_text = _cuda_contig(q_text, "q_text")
+    k_all = _cuda_contig(k_all, "k_all")
+    token_group = _cuda_contig(token_group, "token_group")
+    Hq, Lt, dh = q_text.shape
+    Hkv, S, _ = k_all.shape
+    dev = q_text.device
+    D = 0
+    if hidden is not None:
+        hidden = _cuda_contig(hidden, "hidden")
+        D = hidden.shape[1]
+    L = lib()
+    G = len(group_budget)
+    budgets = (_c.c_int32 * G)(*[int(b) for b in group_budget])
+    if out is None:
+        out = {
+            "scores": torch.empty(n_vis, dtype=torch.float32, device=dev),
+            "keep_idx": torch.empty(S, dtype=torch.int32, device=dev),
+            "S_out": torch.zeros(1, dtype=torch.int32, device=dev),
+            "hidden_out": None if hidden is None else torch.empty_like(hidden),
+        }
+    need = L.metok_prefill_prune_workspace_bytes(_dt(q_text), Hq, Hkv, Lt, S, dh, n_vis)
+    ws = workspace(need, dev)
+    st = L.metok_prefill_prune(_ptr(q_text), _ptr(k_all), _ptr(hidden), _dt(q_text), Hq, Hkv, Lt, S, dh, D, vis_start,
+                               n_vis, _ptr(token_group), G, budgets, softmax_scale, _ptr(out["scores"]),
+                               _ptr(out["keep_idx"]), _ptr(out["S_out"]), _ptr(out["hidden_out"]), _ptr(ws),
+                               ws.numel(), _stream())
+    _check("metok_prefill_prune", st)
+    return out
+
+
+def metok_kv_compact(k_layers: Sequence[torch.Tensor], v_layers: Sequence[torch.Tensor], S_cur: int, policy: int,
+                     vis_start: int, n_vis: int, l1: int = 0, keep_ratio: float = 1.0,
+                     scores: Optional[torch.Tensor] = None, keep_idx: Optional[torch.Tensor] = None,
+                     keep_len: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+    nl = len(k_layers)
+    for t in list(k_layers) + list(v_layers):
+        _cuda_contig(t, "k/v layer")
+    Hkv, S_cap, dh = k_layers[0].shape
+    dev = k_layers[0].device
+    L = lib()
+    karr = (_vp * nl)(*[t.data_ptr() for t in k_layers])
+    varr = (_vp * nl)(*[t.data_ptr() for t in v_layers])
+    if keep_idx is None:
+        keep_idx = torch.empty((nl, S_cur), dtype=torch.int32, device=dev)
+        keep_len = torch.zeros(nl, dtype=torch.int32, device=dev)
+    new_len = torch.zeros(nl, dtype=torch.int32, device=dev)
+    per_layer = 0
+    if scores is not None:
+        scores = _cuda_contig(scores, "scores")
+        per_layer = 1 if scores.dim() == 2 else 0
+    need = L.metok_kv_compact_workspace_bytes(_dt(k_layers[0]), nl, Hkv, S_cur, dh, policy, n_vis)
+    ws = workspace(need, dev)
+    st = L.metok_kv_compact(karr, varr, _dt(k_layers[0]), nl, Hkv, S_cap, S_cur, dh, policy, l1, keep_ratio,
+                            vis_start, n_vis, _ptr(scores), per_layer, _ptr(keep_idx), _ptr(keep_len),
+                            _ptr(new_len), _ptr(ws), ws.numel(), _stream())
+    _check("metok_kv_compact", st)
+    return {"keep_idx": keep_idx, "keep_len": keep_len, "new_len": new_len}
+
+
+def metok_version() -> int:
+    return lib().metok_version()

@@ -1,0 +1,18 @@
+// Host-side launch helpers shared between translation units of the METok library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace metok {
+
+// Class-wise top-k + ascending keep list, one CTA per problem p in [0, problems):
+// scores + p*score_stride, keep_idx + p*keep_stride, counts written to count_a[p]
+// and count_b[p] (either may be null).  token_group may be null (single class).
+// budgets_host is a HOST array of G ints.
+int launch_class_topk(const float* scores, size_t score_stride, const int32_t* token_group, int n_vis, int G,
+                      const int32_t* budgets_host, int S, int vis_start, int32_t* keep_idx, size_t keep_stride,
+                      int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st);
+
+}  // namespace metok

@@ -1,0 +1,416 @@
+// metok_prefill_prune: text->visual attention scores at a pruning layer, class-wise
+// top-k under the Eq. 6/7 budgets, and compaction of the surviving hidden states.
+#include "common.cuh"
+#include "select.cuh"
+#include "launchers.h"
+
+namespace metok {
+
+// --------------------------------------------------------------------------- //
+// Attention scores, generic CUDA-core path.
+//
+// Per KV head g the rep = Hq/Hkv query heads of the group form R = rep*Lt rows
+// (row r = local head * Lt + q) that all multiply the same K[g].  The softmax
+// normaliser of a row needs every visible key, the column sums need the
+// normaliser, and the R x S probability matrix is never stored: pass 1 computes
+// per-row running (max, sum) over a split of the columns, pass 2 recomputes the
+// logits, normalises, and sums each column over the rows of the tile.
+// Everything is reduced in a fixed order (no float atomics).
+// --------------------------------------------------------------------------- //
+constexpr int kAtTM = 64, kAtTN = 64;
+constexpr int kAtLD = 65;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kNegInf = -3.0e38f;   // finite stand-in: keeps (m_old - m_new) free of inf - inf
+
+struct AttnDims {
+    int Hq, Hkv, Lt, S, dh, vis_start, n_vis, rep, R, nrt, nsplit, tiles_n;
+    float scale_log2;
+};
+
+template <typename T>
+__device__ __forceinline__ void load_tile_transposed(const T* __restrict__ base, int row0, int row_end, int dh,
+                                                     float* __restrict__ dst /*[dh][kAtLD]*/) {
+    constexpr int VN = Vec16<T>::N;
+    const int cpr = dh / VN;
+    for (int c = threadIdx.x; c < kAtTM * cpr; c += blockDim.x) {
+        const int r = c / cpr, ch = c % cpr;
+        float v[VN];
+        const int row = row0 + r;
+        if (row < row_end) Vec16<T>::load(base + (size_t)row * dh + ch * VN, v);
+        else Vec16<T>::zero(v);
+#pragma unroll
+        for (int q = 0; q < VN; ++q) dst[(ch * VN + q) * kAtLD + r] = v[q];
+    }
+}
+
+__device__ __forceinline__ void tile_logits(const float* __restrict__ Qs, const float* __restrict__ Ks, int dh,
+                                            int ty, int tx, float (&acc)[4][4]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+    for (int kk = 0; kk < dh; ++kk) {
+        float a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = Qs[kk * kAtLD + ty + 16 * i];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) b[j] = Ks[kk * kAtLD + tx + 16 * j];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+attn_stats_kernel(const T* __restrict__ q_text, const T* __restrict__ k_all, AttnDims dm,
+                  float* __restrict__ part_m, float* __restrict__ part_l) {
+    extern __shared__ float smem[];
+    float* Qs = smem;
+    float* Ks = smem + dm.dh * kAtLD;
+    const int split = blockIdx.x, rt = blockIdx.y, g = blockIdx.z;
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const T* Qg = q_text + (size_t)g * dm.R * dm.dh;
+    const T* Kg = k_all + (size_t)g * dm.S * dm.dh;
+    const int text_start = dm.S - dm.Lt;
+    load_tile_transposed<T>(Qg, rt * kAtTM, dm.R, dm.dh, Qs);
+
+    int limit[4];
+    float m_run[4], l_run[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = rt * kAtTM + ty + 16 * i;
+        limit[i] = r < dm.R ? text_start + (r % dm.Lt) : -1;    // last visible key
+        m_run[i] = kNegInf;
+        l_run[i] = 0.f;
+    }
+    const int per = (dm.tiles_n + dm.nsplit - 1) / dm.nsplit;
+    const int t_lo = split * per, t_hi = min(dm.tiles_n, t_lo + per);
+    for (int tn = t_lo; tn < t_hi; ++tn) {
+        __syncthreads();
+        load_tile_transposed<T>(Kg, tn * kAtTN, dm.S, dm.dh, Ks);
+        __syncthreads();
+        float acc[4][4];
+        tile_logits(Qs, Ks, dm.dh, ty, tx, acc);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float tmax = kNegInf;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int u = tn * kAtTN + tx + 16 * j;
+                acc[i][j] = (u <= limit[i]) ? acc[i][j] * dm.scale_log2 : kNegInf;
+                tmax = fmaxf(tmax, acc[i][j]);
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, o));
+            const float m_new = fmaxf(m_run[i], tmax);
+            float s = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s += (acc[i][j] > kNegInf) ? exp2f(acc[i][j] - m_new) : 0.f;
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+            l_run[i] = l_run[i] * exp2f(m_run[i] - m_new) + s;
+            m_run[i] = m_new;
+        }
+    }
+    if (tx == 0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = rt * kAtTM + ty + 16 * i;
+            if (r < dm.R) {
+                const size_t o = ((size_t)g * dm.nsplit + split) * dm.R + r;
+                part_m[o] = m_run[i];
+                part_l[o] = l_run[i];
+            }
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+attn_colsum_kernel(const T* __restrict__ q_text, const T* __restrict__ k_all, AttnDims dm,
+                   const float* __restrict__ part_m, const float* __restrict__ part_l,
+                   float* __restrict__ part_col) {
+    extern __shared__ float smem[];
+    float* Qs = smem;
+    float* Ks = smem + dm.dh * kAtLD;
+    __shared__ float s_M[kAtTM], s_invZ[kAtTM];
+    __shared__ float s_col[8][kAtTN];
+    const int split = blockIdx.x, rt = blockIdx.y, g = blockIdx.z;
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15, warp = tid >> 5;
+    const T* Qg = q_text + (size_t)g * dm.R * dm.dh;
+    const T* Kg = k_all + (size_t)g * dm.S * dm.dh;
+    const int text_start = dm.S - dm.Lt;
+    load_tile_transposed<T>(Qg, rt * kAtTM, dm.R, dm.dh, Qs);
+    if (tid < kAtTM) {
+        const int r = rt * kAtTM + tid;
+        float M = kNegInf, Z = 0.f;
+        if (r < dm.R) {
+            for (int s = 0; s < dm.nsplit; ++s) M = fmaxf(M, part_m[((size_t)g * dm.nsplit + s) * dm.R + r]);
+            for (int s = 0; s < dm.nsplit; ++s) {
+                const size_t o = ((size_t)g * dm.nsplit + s) * dm.R + r;
+                Z += part_l[o] * exp2f(part_m[o] - M);
+            }
+        }
+        s_M[tid] = M;
+        s_invZ[tid] = Z > 0.f ? 1.0f / Z : 0.f;
+    }
+    __syncthreads();
+    int limit[4];
+    float rM[4], rI[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int rl = ty + 16 * i;
+        const int r = rt * kAtTM + rl;
+        limit[i] = r < dm.R ? text_start + (r % dm.Lt) : -1;
+        rM[i] = s_M[rl];
+        rI[i] = s_invZ[rl];
+    }
+    const int per = (dm.tiles_n + dm.nsplit - 1) / dm.nsplit;
+    const int t_lo = split * per, t_hi = min(dm.tiles_n, t_lo + per);
+    const int vis_end = dm.vis_start + dm.n_vis;
+    for (int tn = t_lo; tn < t_hi; ++tn) {
+        const int u0 = tn * kAtTN;
+        if (u0 >= vis_end || u0 + kAtTN <= dm.vis_start) continue;     // no visual column in this tile
+        __syncthreads();
+        load_tile_transposed<T>(Kg, u0, dm.S, dm.dh, Ks);
+        __syncthreads();
+        float acc[4][4];
+        tile_logits(Qs, Ks, dm.dh, ty, tx, acc);
+        float cs[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int u = u0 + tx + 16 * j;
+            float c = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                c += (u <= limit[i]) ? exp2f(acc[i][j] * dm.scale_log2 - rM[i]) * rI[i] : 0.f;
+            c += __shfl_xor_sync(0xFFFFFFFFu, c, 16);            // the warp's two row groups
+            cs[j] = c;
+        }
+        if ((tid & 31) < 16) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s_col[warp][tx + 16 * j] = cs[j];
+        }
+        __syncthreads();
+        if (tid < kAtTN) {
+            const int u = u0 + tid;
+            if (u >= dm.vis_start && u < vis_end) {
+                float c = 0.f;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) c += s_col[w][tid];
+                part_col[((size_t)g * dm.nrt + rt) * dm.n_vis + (u - dm.vis_start)] = c;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+attn_score_reduce_kernel(const float* __restrict__ part_col, int nparts, int n_vis, float inv_rows,
+                         float* __restrict__ scores) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n_vis) return;
+    float a = 0.f;
+    for (int p = 0; p < nparts; ++p) a += part_col[(size_t)p * n_vis + j];
+    scores[j] = a * inv_rows;
+}
+
+// --------------------------------------------------------------------------- //
+// Class-wise top-k + ordered keep list.  One CTA per problem (blockIdx.x): the
+// prefill step launches one, the KV TOPK policy one per layer.
+// --------------------------------------------------------------------------- //
+struct TopkBudgets { int v[METOK_MAX_GROUPS]; };
+
+__global__ void __launch_bounds__(1024)
+class_topk_kernel(const float* __restrict__ scores, size_t score_stride, const int32_t* __restrict__ token_group,
+                  int n_vis, int G, TopkBudgets budgets, int S, int vis_start, int32_t* __restrict__ keep_idx,
+                  size_t keep_stride, int32_t* __restrict__ count_a, int32_t* __restrict__ count_b) {
+    __shared__ SelectSmem sm;
+    __shared__ int s_budget[METOK_MAX_GROUPS];
+    __shared__ int s_clamped[METOK_MAX_GROUPS];
+    extern __shared__ uint32_t hist[];               // [G*256]
+    const float* sc = scores + (size_t)blockIdx.x * score_stride;
+    int32_t* keep = keep_idx + (size_t)blockIdx.x * keep_stride;
+    for (int g = threadIdx.x; g < G; g += blockDim.x) s_budget[g] = budgets.v[g];
+    __syncthreads();
+    auto cls = [=](int i) {
+        if (!token_group) return 0;
+        const int g = token_group[i];
+        return (g >= 0 && g < G) ? g : -1;
+    };
+    auto val = [=](int i) { return sc[i]; };
+    block_select_thresholds(n_vis, G, cls, val, s_budget, hist, sm, s_clamped);
+    const int vis_end = vis_start + n_vis;
+    auto flag = [&](int u) {
+        if (u < vis_start || u >= vis_end) return true;
+        const int i = u - vis_start;
+        const int g = cls(i);
+        return g >= 0 && sm.need[g] > 0 && key64_of(sc[i], i) >= sm.prefix[g];
+    };
+    auto emit = [&](int u, int rank) { keep[rank] = u; };
+    const int total = block_compact(S, flag, emit, sm);
+    if (threadIdx.x == 0) {
+        if (count_a) count_a[blockIdx.x] = total;
+        if (count_b) count_b[blockIdx.x] = total;
+    }
+}
+
+int launch_class_topk(const float* scores, size_t score_stride, const int32_t* token_group, int n_vis, int G,
+                      const int32_t* budgets_host, int S, int vis_start, int32_t* keep_idx, size_t keep_stride,
+                      int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st) {
+    TopkBudgets b;
+    for (int g = 0; g < METOK_MAX_GROUPS; ++g) b.v[g] = g < G ? budgets_host[g] : 0;
+    const size_t smem = (size_t)G * 256 * sizeof(uint32_t);
+    if (smem > 32 * 1024)
+        METOK_CUDA_TRY(cudaFuncSetAttribute(class_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    class_topk_kernel<<<problems, 1024, smem, st>>>(scores, score_stride, token_group, n_vis, G, b, S, vis_start,
+                                                    keep_idx, keep_stride, count_a, count_b);
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
+}
+
+// --------------------------------------------------------------------------- //
+// hidden_out[i] = hidden[keep_idx[i]], i < *S_out.  Rows are whole 16-byte chunks.
+// --------------------------------------------------------------------------- //
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const int32_t* __restrict__ keep_idx,
+                   const int32_t* __restrict__ n_rows, int row_chunks) {
+    const int n = *n_rows;
+    for (int i = blockIdx.x; i < n; i += gridDim.x) {
+        const uint4* s = src + (size_t)keep_idx[i] * row_chunks;
+        uint4* o = dst + (size_t)i * row_chunks;
+        for (int c = threadIdx.x; c < row_chunks; c += 256 * 4) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (c + u * 256 < row_chunks) v[u] = __ldg(s + c + u * 256);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (c + u * 256 < row_chunks) o[c + u * 256] = v[u];
+        }
+    }
+}
+
+static AttnDims make_dims(int Hq, int Hkv, int Lt, int S, int dh, int vis_start, int n_vis, float scale) {
+    AttnDims dm;
+    dm.Hq = Hq; dm.Hkv = Hkv; dm.Lt = Lt; dm.S = S; dm.dh = dh; dm.vis_start = vis_start; dm.n_vis = n_vis;
+    dm.rep = Hq / Hkv;
+    dm.R = dm.rep * Lt;
+    dm.nrt = ceil_div(dm.R, kAtTM);
+    dm.tiles_n = ceil_div(S, kAtTN);
+    int ns = ceil_div(4 * kNumSMs, dm.nrt * Hkv);
+    if (ns > dm.tiles_n) ns = dm.tiles_n;
+    if (ns < 1) ns = 1;
+    if (ns > 64) ns = 64;
+    dm.nsplit = ns;
+    dm.scale_log2 = scale * kLog2e;
+    return dm;
+}
+
+struct PrefillWs {
+    float *part_m, *part_l, *part_col;
+};
+static PrefillWs carve_prefill(Carver& cv, const AttnDims& dm) {
+    PrefillWs w;
+    w.part_m = cv.take<float>((size_t)dm.Hkv * dm.nsplit * dm.R);
+    w.part_l = cv.take<float>((size_t)dm.Hkv * dm.nsplit * dm.R);
+    w.part_col = cv.take<float>((size_t)dm.Hkv * dm.nrt * dm.n_vis);
+    return w;
+}
+
+template <typename T>
+static int launch_attn_scores(const void* q_text, const void* k_all, const AttnDims& dm, const PrefillWs& w,
+                              float* scores, cudaStream_t st) {
+    const size_t smem = (size_t)2 * dm.dh * kAtLD * sizeof(float);
+    METOK_CUDA_TRY(cudaFuncSetAttribute(attn_stats_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    METOK_CUDA_TRY(cudaFuncSetAttribute(attn_colsum_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid(dm.nsplit, dm.nrt, dm.Hkv);
+    attn_stats_kernel<T><<<grid, 256, smem, st>>>(reinterpret_cast<const T*>(q_text), reinterpret_cast<const T*>(k_all),
+                                                  dm, w.part_m, w.part_l);
+    METOK_LAUNCH_CHECK();
+    attn_colsum_kernel<T><<<grid, 256, smem, st>>>(reinterpret_cast<const T*>(q_text),
+                                                   reinterpret_cast<const T*>(k_all), dm, w.part_m, w.part_l,
+                                                   w.part_col);
+    METOK_LAUNCH_CHECK();
+    attn_score_reduce_kernel<<<ceil_div(dm.n_vis, 256), 256, 0, st>>>(w.part_col, dm.Hkv * dm.nrt, dm.n_vis,
+                                                                      1.0f / (float)(dm.Hq * dm.Lt), scores);
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
+}
+
+}  // namespace metok
+
+using namespace metok;
+
+extern "C" size_t metok_prefill_prune_workspace_bytes(int dtype, int Hq, int Hkv, int Lt, int S, int dh, int n_vis) {
+    (void)dtype;
+    if (Hq < 1 || Hkv < 1 || Lt < 1 || S < 1 || dh < 1 || n_vis < 1 || Hq % Hkv) return 0;
+    AttnDims dm = make_dims(Hq, Hkv, Lt, S, dh, 0, n_vis, 1.f);
+    Carver cv(nullptr);
+    carve_prefill(cv, dm);
+    return cv.total();
+}
+
+extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const void* hidden, int dtype, int Hq,
+                                   int Hkv, int Lt, int S, int dh, int D, int vis_start, int n_vis,
+                                   const int32_t* token_group, int G, const int32_t* group_budget,
+                                   float softmax_scale, float* scores, int32_t* keep_idx, int32_t* S_out,
+                                   void* hidden_out, void* ws, size_t ws_bytes, void* stream) {
+    if (!q_text || !k_all || !token_group || !group_budget || !scores || !keep_idx || !S_out)
+        return METOK_ERR_INVALID_ARG;
+    if ((hidden == nullptr) != (hidden_out == nullptr)) return METOK_ERR_INVALID_ARG;
+    if (dtype != METOK_F32 && dtype != METOK_BF16) return METOK_ERR_INVALID_ARG;
+    if (Hq < 1 || Hkv < 1 || Lt < 1 || S < 1 || dh < 1 || n_vis < 1 || (hidden && D < 1)) return METOK_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0 || Lt > S) return METOK_ERR_INVALID_ARG;
+    if (vis_start < 0 || (long long)vis_start + n_vis > (long long)S - Lt) return METOK_ERR_INVALID_ARG;
+    if (G < 1 || G > METOK_MAX_GROUPS) return METOK_ERR_INVALID_ARG;
+    for (int g = 0; g < G; ++g)
+        if (group_budget[g] < 0) return METOK_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f)) return METOK_ERR_INVALID_ARG;
+    if (!aligned16(q_text) || !aligned16(k_all) || (hidden && (!aligned16(hidden) || !aligned16(hidden_out))))
+        return METOK_ERR_INVALID_ARG;
+    const int eb = dtype == METOK_F32 ? 4 : 2;
+    if (dtype == METOK_BF16 && dh != 64 && dh != 128) return METOK_ERR_UNSUPPORTED;
+    if (dtype == METOK_F32 && (dh > 128 || dh % 4 != 0)) return METOK_ERR_UNSUPPORTED;
+    if (hidden && ((long long)D * eb) % 16 != 0) return METOK_ERR_UNSUPPORTED;
+    const size_t need = metok_prefill_prune_workspace_bytes(dtype, Hq, Hkv, Lt, S, dh, n_vis);
+    if (!ws || ws_bytes < need || !aligned16(ws)) return METOK_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+    AttnDims dm = make_dims(Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale);
+    Carver cv(ws);
+    PrefillWs w = carve_prefill(cv, dm);
+    int rc = dtype == METOK_F32 ? launch_attn_scores<float>(q_text, k_all, dm, w, scores, st)
+                                : launch_attn_scores<__nv_bfloat16>(q_text, k_all, dm, w, scores, st);
+    if (rc != METOK_OK) return rc;
+    rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, S_out, nullptr,
+                           1, st);
+    if (rc != METOK_OK) return rc;
+    if (hidden) {
+        const int row_chunks = (int)((long long)D * eb / 16);
+        gather_rows_kernel<<<kNumSMs * 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(hidden),
+                                                        reinterpret_cast<uint4*>(hidden_out), keep_idx, S_out,
+                                                        row_chunks);
+        METOK_LAUNCH_CHECK();
+    }
+    return METOK_OK;
+}
+
+extern "C" int metok_retention_budgets(double alpha, double r, int stage, const int32_t* N0, int32_t* budget) {
+    if (!N0 || !budget) return METOK_ERR_INVALID_ARG;
+    if (!(alpha > 0.0 && alpha <= 1.0) || !(r > 0.0 && r <= 1.0)) return METOK_ERR_INVALID_ARG;
+    if (stage < 0 || stage > 3 || N0[0] < 0 || N0[1] < 0) return METOK_ERR_INVALID_ARG;
+    double rk, rn;
+    switch (stage) {
+        case 0: rk = 1.0; rn = 1.0; break;
+        case 1: rk = r; rn = alpha * r; break;
+        case 2: rk = r * r; rn = 0.0; break;
+        default: rk = 0.0; rn = 0.0; break;
+    }
+    int bk = ceilq(rk * (double)N0[0]), bn = ceilq(rn * (double)N0[1]);
+    budget[0] = bk < N0[0] ? bk : N0[0];
+    budget[1] = bn < N0[1] ? bn : N0[1];
+    return METOK_OK;
+}

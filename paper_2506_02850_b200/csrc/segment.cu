@@ -1,0 +1,273 @@
+// metok_segment_events: adjacent-frame cosine similarity (Eq. 4) and the split at
+// the k-1 lowest similarities.
+//
+// FLATTEN mode is one streaming pass over V.  The flattened frame vector (N*d
+// elements) is cut into slabs of 256 threads x 4 x 16 bytes; a CTA walks a run of
+// consecutive frames of one slab, keeps the previous frame's chunks in registers
+// and accumulates <v_f, v_f> and <v_f, v_{f+1}> in fp32.  Per-(slab, frame)
+// partial sums go to the workspace and are added in a fixed order by the finishing
+// kernel, so the result does not depend on scheduling.
+#include "common.cuh"
+
+namespace metok {
+
+constexpr int kSegThreads = 256;
+constexpr int kSegUnroll = 4;     // 16-byte chunks per thread per frame
+constexpr int kMaxFrames = 8192;
+
+template <typename T>
+__global__ void __launch_bounds__(kSegThreads)
+seg_partial_kernel(const T* __restrict__ feats, int Tn, long long chunks_per_frame, int frames_per_cta,
+                   float* __restrict__ part_dot, float* __restrict__ part_nrm) {
+    constexpr int VN = Vec16<T>::N;
+    __shared__ float red[2][kSegThreads / 32];
+    const int slab = blockIdx.x;
+    const int f0 = blockIdx.y * frames_per_cta;
+    const int f1 = min(Tn, f0 + frames_per_cta);          // own frames [f0, f1)
+    const int f_last = min(Tn - 1, f1);                   // halo frame for the last dot
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    long long chunk[kSegUnroll];
+    bool ok[kSegUnroll];
+#pragma unroll
+    for (int u = 0; u < kSegUnroll; ++u) {
+        chunk[u] = (long long)slab * (kSegThreads * kSegUnroll) + u * kSegThreads + tid;
+        ok[u] = chunk[u] < chunks_per_frame;
+    }
+    float prev[kSegUnroll][VN];
+#pragma unroll
+    for (int u = 0; u < kSegUnroll; ++u) Vec16<T>::zero(prev[u]);
+
+    for (int f = f0; f <= f_last; ++f) {
+        const T* frame = feats + (size_t)f * (size_t)chunks_per_frame * VN;
+        float cur[kSegUnroll][VN];
+#pragma unroll
+        for (int u = 0; u < kSegUnroll; ++u) {
+            if (ok[u]) Vec16<T>::load(frame + chunk[u] * VN, cur[u]);
+            else Vec16<T>::zero(cur[u]);
+        }
+        float nn = 0.f, dp = 0.f;
+#pragma unroll
+        for (int u = 0; u < kSegUnroll; ++u) {
+#pragma unroll
+            for (int e = 0; e < VN; ++e) {
+                nn = fmaf(cur[u][e], cur[u][e], nn);
+                dp = fmaf(cur[u][e], prev[u][e], dp);
+                prev[u][e] = cur[u][e];
+            }
+        }
+        nn = warp_sum(nn);
+        dp = warp_sum(dp);
+        if (lane == 0) { red[0][warp] = nn; red[1][warp] = dp; }
+        __syncthreads();
+        if (tid == 0) {
+            float a = 0.f, b = 0.f;
+#pragma unroll
+            for (int w = 0; w < kSegThreads / 32; ++w) { a += red[0][w]; b += red[1][w]; }
+            if (f < f1) part_nrm[(size_t)slab * Tn + f] = a;
+            if (f > f0) part_dot[(size_t)slab * Tn + (f - 1)] = b;   // dot of frames f-1 and f
+        }
+        __syncthreads();
+    }
+}
+
+// MEANPOOL: mean over the N tokens of each frame, per 16-byte column chunk.
+template <typename T>
+__global__ void __launch_bounds__(128)
+seg_mean_kernel(const T* __restrict__ feats, int N, int d, float* __restrict__ mean) {
+    constexpr int VN = Vec16<T>::N;
+    const int f = blockIdx.y;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c * VN >= d) return;
+    const T* base = feats + ((size_t)f * N) * d + (size_t)c * VN;
+    float acc[VN];
+    Vec16<T>::zero(acc);
+    for (int p = 0; p < N; ++p) {
+        float v[VN];
+        Vec16<T>::load(base + (size_t)p * d, v);
+#pragma unroll
+        for (int e = 0; e < VN; ++e) acc[e] += v[e];
+    }
+    const float inv = 1.0f / (float)N;
+#pragma unroll
+    for (int e = 0; e < VN; ++e) mean[(size_t)f * d + c * VN + e] = acc[e] * inv;
+}
+
+// dot / norm of consecutive mean vectors: one CTA per frame, written as a single "slab".
+__global__ void __launch_bounds__(256)
+seg_meandot_kernel(const float* __restrict__ mean, int Tn, int d, float* __restrict__ part_dot,
+                   float* __restrict__ part_nrm) {
+    __shared__ float red[2][8];
+    const int f = blockIdx.x;
+    const float* a = mean + (size_t)f * d;
+    const float* b = mean + (size_t)(f + 1 < Tn ? f + 1 : f) * d;
+    float nn = 0.f, dp = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        nn = fmaf(a[i], a[i], nn);
+        dp = fmaf(a[i], b[i], dp);
+    }
+    nn = warp_sum(nn);
+    dp = warp_sum(dp);
+    if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = nn; red[1][threadIdx.x >> 5] = dp; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float x = 0.f, y = 0.f;
+        for (int w = 0; w < 8; ++w) { x += red[0][w]; y += red[1][w]; }
+        part_nrm[f] = x;
+        if (f + 1 < Tn) part_dot[f] = y;
+    }
+}
+
+// Adds the slab partials in slab order, forms the cosines, picks the k-1 smallest
+// (rank by counting; ties to the lower index) and writes boundaries, CSR offsets
+// and per-frame event ids.  One CTA of 1024 threads; T <= kMaxFrames.
+__global__ void __launch_bounds__(1024)
+seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ part_nrm, int nslab,
+                  int Tn, int k, float* __restrict__ sims, int32_t* __restrict__ boundaries,
+                  int32_t* __restrict__ event_offsets, int32_t* __restrict__ frame_event) {
+    extern __shared__ float sm_f[];
+    float* s_sim = sm_f;                                   // [Tn]   (Tn-1 used)
+    float* s_nrm = sm_f + Tn;                              // [Tn]
+    int* s_flag = reinterpret_cast<int*>(sm_f + 2 * Tn);   // [Tn]  boundary after frame i
+    __shared__ int s_scan[1024];
+    const int tid = threadIdx.x, nthr = blockDim.x;
+
+    for (int f = tid; f < Tn; f += nthr) {
+        float a = 0.f;
+        for (int s = 0; s < nslab; ++s) a += part_nrm[(size_t)s * Tn + f];
+        s_nrm[f] = fmaxf(sqrtf(a), kEps);
+    }
+    __syncthreads();
+    for (int i = tid; i < Tn - 1; i += nthr) {
+        float a = 0.f;
+        for (int s = 0; s < nslab; ++s) a += part_dot[(size_t)s * Tn + i];
+        const float c = a / (s_nrm[i] * s_nrm[i + 1]);
+        s_sim[i] = c;
+        sims[i] = c;
+    }
+    __syncthreads();
+    const int nb = k - 1;
+    for (int i = tid; i < Tn; i += nthr) {
+        int flag = 0;
+        if (i < Tn - 1 && nb > 0) {
+            const float v = s_sim[i];
+            int rank = 0;
+            for (int j = 0; j < Tn - 1; ++j) {
+                const float w = s_sim[j];
+                rank += (w < v) || (w == v && j < i);
+            }
+            flag = rank < nb;
+        }
+        s_flag[i] = flag;
+    }
+    __syncthreads();
+    // exclusive scan of the flags: contiguous ranges per thread, then a scan of the range totals
+    const int per = (Tn + nthr - 1) / nthr;
+    const int lo = min(Tn, tid * per), hi = min(Tn, lo + per);
+    int local = 0;
+    for (int i = lo; i < hi; ++i) local += s_flag[i];
+    s_scan[tid] = local;
+    __syncthreads();
+    for (int off = 1; off < nthr; off <<= 1) {
+        const int v = (tid >= off) ? s_scan[tid - off] : 0;
+        __syncthreads();
+        s_scan[tid] += v;
+        __syncthreads();
+    }
+    int run = s_scan[tid] - local;                         // boundaries before frame lo
+    for (int i = lo; i < hi; ++i) {
+        frame_event[i] = run;                              // event id = boundaries strictly before i
+        if (s_flag[i] && run < nb) {                       // (NaN similarities could over-flag)
+            boundaries[run] = i;
+            event_offsets[run + 1] = i + 1;
+            ++run;
+        }
+    }
+    if (tid == 0) {
+        event_offsets[0] = 0;
+        event_offsets[k] = Tn;
+    }
+}
+
+template <typename T>
+static int launch_segment(const void* feats, int Tn, int N, int d, int k, int sim_mode, float* sims,
+                          int32_t* boundaries, int32_t* event_offsets, int32_t* frame_event, void* ws,
+                          cudaStream_t st) {
+    constexpr int VN = 16 / sizeof(T);
+    Carver cv(ws);
+    int nslab;
+    float *part_dot, *part_nrm;
+    if (sim_mode == METOK_SIM_FLATTEN) {
+        const long long chunks = (long long)N * d / VN;
+        nslab = (int)((chunks + kSegThreads * kSegUnroll - 1) / (kSegThreads * kSegUnroll));
+        int fpc = 16;
+        while (fpc > 1 && (long long)nslab * ceil_div(Tn, fpc) < 4 * kNumSMs) fpc >>= 1;
+        part_dot = cv.take<float>((size_t)nslab * Tn);
+        part_nrm = cv.take<float>((size_t)nslab * Tn);
+        dim3 grid(nslab, ceil_div(Tn, fpc));
+        seg_partial_kernel<T><<<grid, kSegThreads, 0, st>>>(reinterpret_cast<const T*>(feats), Tn, chunks, fpc,
+                                                            part_dot, part_nrm);
+        METOK_LAUNCH_CHECK();
+    } else {
+        nslab = 1;
+        part_dot = cv.take<float>((size_t)Tn);
+        part_nrm = cv.take<float>((size_t)Tn);
+        float* mean = cv.take<float>((size_t)Tn * d);
+        dim3 grid(ceil_div(d / VN, 128), Tn);
+        seg_mean_kernel<T><<<grid, 128, 0, st>>>(reinterpret_cast<const T*>(feats), N, d, mean);
+        METOK_LAUNCH_CHECK();
+        seg_meandot_kernel<<<Tn, 256, 0, st>>>(mean, Tn, d, part_dot, part_nrm);
+        METOK_LAUNCH_CHECK();
+    }
+    const size_t smem = (size_t)Tn * 3 * sizeof(float);
+    if (smem > 48 * 1024) {
+        METOK_CUDA_TRY(cudaFuncSetAttribute(seg_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)smem));
+    }
+    seg_finish_kernel<<<1, 1024, smem, st>>>(part_dot, part_nrm, nslab, Tn, k, sims, boundaries, event_offsets,
+                                             frame_event);
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
+}
+
+}  // namespace metok
+
+using namespace metok;
+
+extern "C" size_t metok_segment_events_workspace_bytes(int dtype, int T, int N, int d, int sim_mode) {
+    if (T < 1 || N < 1 || d < 1) return 0;
+    const int VN = dtype == METOK_F32 ? 4 : 8;
+    Carver cv(nullptr);
+    if (sim_mode == METOK_SIM_FLATTEN) {
+        const long long chunks = ((long long)N * d + VN - 1) / VN;
+        const size_t nslab = (size_t)((chunks + kSegThreads * kSegUnroll - 1) / (kSegThreads * kSegUnroll));
+        cv.take<float>(nslab * T);
+        cv.take<float>(nslab * T);
+    } else {
+        cv.take<float>((size_t)T);
+        cv.take<float>((size_t)T);
+        cv.take<float>((size_t)T * d);
+    }
+    return cv.total();
+}
+
+extern "C" int metok_segment_events(const void* feats, int dtype, int T, int N, int d, int k, int sim_mode,
+                                    float* sims, int32_t* boundaries, int32_t* event_offsets,
+                                    int32_t* frame_event, void* ws, size_t ws_bytes, void* stream) {
+    if (!feats || !sims || !boundaries || !event_offsets || !frame_event) return METOK_ERR_INVALID_ARG;
+    if (dtype != METOK_F32 && dtype != METOK_BF16) return METOK_ERR_INVALID_ARG;
+    if (sim_mode != METOK_SIM_FLATTEN && sim_mode != METOK_SIM_MEANPOOL) return METOK_ERR_INVALID_ARG;
+    if (T < 1 || N < 1 || d < 1 || k < 1 || k > T) return METOK_ERR_INVALID_ARG;
+    if (!aligned16(feats) || (reinterpret_cast<uintptr_t>(sims) & 3) || (reinterpret_cast<uintptr_t>(boundaries) & 3) ||
+        (reinterpret_cast<uintptr_t>(event_offsets) & 3) || (reinterpret_cast<uintptr_t>(frame_event) & 3))
+        return METOK_ERR_INVALID_ARG;
+    const int eb = dtype == METOK_F32 ? 4 : 2;
+    if (((long long)d * eb) % 16 != 0 || T > kMaxFrames) return METOK_ERR_UNSUPPORTED;
+    const size_t need = metok_segment_events_workspace_bytes(dtype, T, N, d, sim_mode);
+    if (!ws || ws_bytes < need || !aligned16(ws)) return METOK_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (dtype == METOK_F32)
+        return launch_segment<float>(feats, T, N, d, k, sim_mode, sims, boundaries, event_offsets, frame_event, ws, st);
+    return launch_segment<__nv_bfloat16>(feats, T, N, d, k, sim_mode, sims, boundaries, event_offsets, frame_event,
+                                         ws, st);
+}

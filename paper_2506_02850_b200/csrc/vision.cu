@@ -1,0 +1,542 @@
+// metok_compress_vision: text relevance and key events (Eq. 5), per-event key-token
+// top-k, merge-assign of the remaining tokens and averaging.
+#include "common.cuh"
+#include "select.cuh"
+
+namespace metok {
+
+// --------------------------------------------------------------------------- //
+// token_score[j] = <x_j, t> / (max(|x_j|, eps) * max(|t|, eps)); also 1/max(|x_j|, eps).
+// One warp per token row, 16-byte loads, four chunks in flight per lane.
+// --------------------------------------------------------------------------- //
+template <typename T>
+__global__ void __launch_bounds__(256)
+tok_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Nv, int d,
+                 float* __restrict__ token_score, float* __restrict__ inv_norm) {
+    constexpr int VN = Vec16<T>::N;
+    extern __shared__ float s_t[];                 // [d]
+    __shared__ float s_red[8];
+    __shared__ float s_tn;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nchunk = d / VN;
+    // t is stored in planes of 4 floats per chunk so that a lane's 16-byte reads
+    // of consecutive chunks are bank-conflict free
+    for (int i = tid; i < d; i += 256) {
+        const int c = i / VN, q = i % VN;
+        s_t[(q >> 2) * (nchunk * 4) + c * 4 + (q & 3)] = to_float(text[i]);
+    }
+    __syncthreads();
+    float a = 0.f;
+    for (int i = tid; i < d; i += 256) a = fmaf(s_t[i], s_t[i], a);
+    a = warp_sum(a);
+    if (lane == 0) s_red[warp] = a;
+    __syncthreads();
+    if (tid == 0) {
+        float s = 0.f;
+        for (int w = 0; w < 8; ++w) s += s_red[w];
+        s_tn = fmaxf(sqrtf(s), kEps);
+    }
+    __syncthreads();
+    const float tn = s_tn;
+    for (int row = blockIdx.x * 8 + warp; row < Nv; row += gridDim.x * 8) {
+        const T* x = feats + (size_t)row * d;
+        float nn = 0.f, dt = 0.f;
+        for (int c0 = 0; c0 < nchunk; c0 += 128) {
+            float v[4][VN];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = c0 + u * 32 + lane;
+                if (c < nchunk) Vec16<T>::load(x + (size_t)c * VN, v[u]);
+                else Vec16<T>::zero(v[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = c0 + u * 32 + lane;
+                if (c < nchunk) {
+#pragma unroll
+                    for (int h = 0; h < VN / 4; ++h) {
+                        const float4 tt = reinterpret_cast<const float4*>(s_t + h * (nchunk * 4))[c];
+                        nn = fmaf(v[u][4 * h + 0], v[u][4 * h + 0], nn);
+                        dt = fmaf(v[u][4 * h + 0], tt.x, dt);
+                        nn = fmaf(v[u][4 * h + 1], v[u][4 * h + 1], nn);
+                        dt = fmaf(v[u][4 * h + 1], tt.y, dt);
+                        nn = fmaf(v[u][4 * h + 2], v[u][4 * h + 2], nn);
+                        dt = fmaf(v[u][4 * h + 2], tt.z, dt);
+                        nn = fmaf(v[u][4 * h + 3], v[u][4 * h + 3], nn);
+                        dt = fmaf(v[u][4 * h + 3], tt.w, dt);
+                    }
+                }
+            }
+        }
+        nn = warp_sum(nn);
+        dt = warp_sum(dt);
+        if (lane == 0) {
+            const float n = fmaxf(sqrtf(nn), kEps);
+            token_score[row] = dt / (n * tn);
+            inv_norm[row] = 1.0f / n;
+        }
+    }
+}
+
+// frame_score[f] = mean of the frame's N token scores; one warp per frame, fixed order.
+__global__ void __launch_bounds__(256)
+frame_score_kernel(const float* __restrict__ token_score, int Tn, int N, float* __restrict__ frame_score) {
+    const int f = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (f >= Tn) return;
+    const int lane = threadIdx.x & 31;
+    float s = 0.f;
+    for (int p = lane; p < N; p += 32) s += token_score[(size_t)f * N + p];
+    s = warp_sum(s);
+    if (lane == 0) frame_score[f] = s / (float)N;
+}
+
+// Event scores, key events, per-event token budgets and output offsets.  One CTA.
+struct PlanParams {
+    int Tn, N, k, n_key_events, event_agg, mode, tile_rows;
+    double keep_key, keep_nonkey, beta;
+};
+
+__global__ void __launch_bounds__(1024)
+event_plan_kernel(const float* __restrict__ frame_score, const int32_t* __restrict__ event_offsets, PlanParams pp,
+                  float* __restrict__ event_score, uint8_t* __restrict__ event_is_key,
+                  int32_t* __restrict__ ev_lo, int32_t* __restrict__ ev_budget, int32_t* __restrict__ ev_out_off,
+                  int32_t* __restrict__ ev_tile_off, int32_t* __restrict__ n_out) {
+    extern __shared__ float s_score[];      // [k]
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int k = pp.k, Tn = pp.Tn;
+    for (int e = tid; e < k; e += nthr) {
+        int lo = min(max(event_offsets[e], 0), Tn);
+        int hi = min(max(event_offsets[e + 1], lo), Tn);
+        ev_lo[e] = lo;
+        if (e == k - 1) ev_lo[k] = hi;
+        float s;
+        if (hi <= lo) {
+            s = -3.0e38f;
+        } else if (pp.event_agg == METOK_AGG_MEAN) {
+            float a = 0.f;
+            for (int f = lo; f < hi; ++f) a += frame_score[f];
+            s = a / (float)(hi - lo);
+        } else {
+            float a = frame_score[lo];
+            for (int f = lo + 1; f < hi; ++f) a = fmaxf(a, frame_score[f]);
+            s = a;
+        }
+        s_score[e] = s;
+        event_score[e] = s;
+    }
+    __syncthreads();
+    for (int e = tid; e < k; e += nthr) {
+        const float v = s_score[e];
+        int rank = 0;
+        for (int j = 0; j < k; ++j) {
+            const float w = s_score[j];
+            rank += (w > v) || (w == v && j < e);
+        }
+        event_is_key[e] = (uint8_t)(rank < pp.n_key_events);
+    }
+    __syncthreads();
+    if (pp.mode == METOK_MODE_TOPK_MERGE) {
+        for (int e = tid; e < k; e += nthr) {
+            const int lo = min(max(event_offsets[e], 0), Tn);
+            const int hi = min(max(event_offsets[e + 1], lo), Tn);
+            const int m = (hi - lo) * pp.N;
+            const double ratio = event_is_key[e] ? pp.keep_key : pp.keep_nonkey;
+            const double c = ratio * (double)m - 1e-9;
+            long long b = (long long)c;
+            if ((double)b < c) b += 1;
+            if (b < 1) b = 1;
+            if (b > m) b = m;
+            ev_budget[e] = (int)b;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int slots = 0, tiles = 0;
+            for (int e = 0; e < k; ++e) {
+                ev_out_off[e] = slots;
+                ev_tile_off[e] = tiles;
+                const int lo = min(max(event_offsets[e], 0), Tn);
+                const int hi = min(max(event_offsets[e + 1], lo), Tn);
+                slots += ev_budget[e];
+                tiles += ((hi - lo) * pp.N + pp.tile_rows - 1) / pp.tile_rows;
+            }
+            ev_out_off[k] = slots;
+            ev_tile_off[k] = tiles;
+            *n_out = slots;
+        }
+    }
+}
+
+// Per-event key-token top-k: one CTA per event.
+__global__ void __launch_bounds__(1024)
+event_topk_kernel(const float* __restrict__ token_score, const int32_t* __restrict__ ev_lo, int N,
+                  const int32_t* __restrict__ ev_budget, const int32_t* __restrict__ ev_out_off,
+                  uint8_t* __restrict__ is_key, int32_t* __restrict__ out_src, int32_t* __restrict__ out_event,
+                  int32_t* __restrict__ assign) {
+    __shared__ SelectSmem sm;
+    __shared__ uint32_t hist[256];
+    __shared__ int s_budget[1];
+    __shared__ int s_clamped[1];
+    const int e = blockIdx.x;
+    const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
+    const int n = hi - lo;
+    if (n <= 0) return;
+    if (threadIdx.x == 0) s_budget[0] = ev_budget[e];
+    __syncthreads();
+    const float* s = token_score + lo;
+    auto cls = [](int) { return 0; };
+    auto val = [s](int i) { return s[i]; };
+    block_select_thresholds(n, 1, cls, val, s_budget, hist, sm, s_clamped);
+    const unsigned long long thr = sm.prefix[0];
+    const bool any = sm.need[0] > 0;
+    const int slot0 = ev_out_off[e];
+    auto flag = [&](int i) { return any && key64_of(s[i], i) >= thr; };
+    auto emit = [&](int i, int rank) {
+        const int slot = slot0 + rank;
+        out_src[slot] = lo + i;
+        out_event[slot] = e;
+        assign[lo + i] = slot;
+    };
+    block_compact(n, flag, emit, sm);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) is_key[lo + i] = flag(i) ? 1 : 0;
+}
+
+// --------------------------------------------------------------------------- //
+// Merge-assign, generic CUDA-core path (fp32 inputs, and any shape the tensor-core
+// path does not take).  CTA = 64 token rows of one event; loops over the event's
+// key tokens 64 at a time; fp32 accumulate; fused row argmax of dot * inv_norm(key).
+// --------------------------------------------------------------------------- //
+constexpr int kMergeTM = 64, kMergeTN = 64, kMergeTK = 32;
+
+__device__ __forceinline__ int find_event(const int32_t* __restrict__ off, int k, int t) {
+    int lo = 0, hi = k;                     // off[lo] <= t < off[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (off[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+merge_assign_simt_kernel(const T* __restrict__ feats, int d, int N, const int32_t* __restrict__ ev_lo, int k,
+                         const int32_t* __restrict__ ev_out_off, const int32_t* __restrict__ ev_tile_off,
+                         const int32_t* __restrict__ out_src, const float* __restrict__ inv_norm,
+                         const uint8_t* __restrict__ is_key, int32_t* __restrict__ assign) {
+    constexpr int VN = Vec16<T>::N;
+    constexpr int CPR = kMergeTK / VN;      // 16-byte chunks per tile row
+    constexpr int LD = kMergeTM + 1;
+    __shared__ float As[kMergeTK][LD];
+    __shared__ float Bs[kMergeTK][LD];
+    __shared__ int s_src[kMergeTN];
+    __shared__ float s_inv[kMergeTN];
+    const int t = blockIdx.x;
+    if (t >= ev_tile_off[k]) return;
+    const int e = find_event(ev_tile_off, k, t);
+    const int row0 = ev_lo[e] * N + (t - ev_tile_off[e]) * kMergeTM;
+    const int row_end = ev_lo[e + 1] * N;
+    const int s0 = ev_out_off[e], s1 = ev_out_off[e + 1];
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+
+    float best_v[4];
+    int best_s[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { best_v[i] = -3.4e38f; best_s[i] = 0x7FFFFFFF; }
+
+    for (int n0 = s0; n0 < s1; n0 += kMergeTN) {
+        __syncthreads();
+        if (tid < kMergeTN) {
+            const int slot = n0 + tid;
+            const int src = slot < s1 ? out_src[slot] : -1;
+            s_src[tid] = src;
+            s_inv[tid] = src >= 0 ? inv_norm[src] : 0.f;
+        }
+        __syncthreads();
+        float acc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        for (int k0 = 0; k0 < d; k0 += kMergeTK) {
+            for (int c = tid; c < kMergeTM * CPR; c += 256) {
+                const int r = c / CPR, ch = c % CPR;
+                const int kk = k0 + ch * VN;
+                float va[VN], vb[VN];
+                const int row = row0 + r;
+                if (row < row_end && kk < d) Vec16<T>::load(feats + (size_t)row * d + kk, va);
+                else Vec16<T>::zero(va);
+                const int src = s_src[r];
+                if (src >= 0 && kk < d) Vec16<T>::load(feats + (size_t)src * d + kk, vb);
+                else Vec16<T>::zero(vb);
+#pragma unroll
+                for (int q = 0; q < VN; ++q) {
+                    As[ch * VN + q][r] = va[q];
+                    Bs[ch * VN + q][r] = vb[q];
+                }
+            }
+            __syncthreads();
+#pragma unroll 8
+            for (int kk = 0; kk < kMergeTK; ++kk) {
+                float a[4], b[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) a[i] = As[kk][ty + 16 * i];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx + 16 * j];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {                 // ascending slot within this thread
+            const int col = tx + 16 * j;
+            const int slot = n0 + col;
+            if (slot < s1) {
+                const float inv = s_inv[col];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float v = acc[i][j] * inv;
+                    if (v > best_v[i]) { best_v[i] = v; best_s[i] = slot; }
+                }
+            }
+        }
+    }
+    // combine the 16 column owners of each row: larger value, then lower slot
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xFFFFFFFFu, best_v[i], o);
+            const int os = __shfl_xor_sync(0xFFFFFFFFu, best_s[i], o);
+            if (ov > best_v[i] || (ov == best_v[i] && os < best_s[i])) { best_v[i] = ov; best_s[i] = os; }
+        }
+        const int row = row0 + ty + 16 * i;
+        if (tx == 0 && row < row_end && !is_key[row]) assign[row] = best_s[i];
+    }
+}
+
+// --------------------------------------------------------------------------- //
+// Averaging: one CTA per output token.  Walks the event's `assign` range in
+// ascending token order (so the summation order is fixed), sums the member rows in
+// fp32, divides by the member count and rounds once.
+// --------------------------------------------------------------------------- //
+constexpr int kAvgThreads = 128;
+constexpr int kAvgChunks = 4;      // 16-byte chunks per thread per pass over d
+
+template <typename T>
+__global__ void __launch_bounds__(kAvgThreads)
+merge_avg_kernel(const T* __restrict__ feats, int d, int N, const int32_t* __restrict__ ev_lo,
+                 const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
+                 const int32_t* __restrict__ n_out, T* __restrict__ out_feats, int32_t* __restrict__ out_members) {
+    constexpr int VN = Vec16<T>::N;
+    __shared__ int s_list[kAvgThreads];
+    __shared__ int s_wtot[kAvgThreads / 32];
+    const int c = blockIdx.x;
+    if (c >= *n_out) return;
+    const int e = out_event[c];
+    const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nchunk = d / VN;
+    for (int cb = 0; cb < nchunk; cb += kAvgThreads * kAvgChunks) {
+        float acc[kAvgChunks][VN];
+#pragma unroll
+        for (int u = 0; u < kAvgChunks; ++u) Vec16<T>::zero(acc[u]);
+        int count = 0;
+        for (int base = lo; base < hi; base += kAvgThreads) {
+            const int j = base + tid;
+            const bool f = j < hi && assign[j] == c;
+            const unsigned bal = __ballot_sync(0xFFFFFFFFu, f);
+            if (lane == 0) s_wtot[warp] = __popc(bal);
+            __syncthreads();
+            int before = 0, total = 0;
+#pragma unroll
+            for (int w = 0; w < kAvgThreads / 32; ++w) {
+                const int v = s_wtot[w];
+                if (w < warp) before += v;
+                total += v;
+            }
+            if (f) s_list[before + __popc(bal & ((1u << lane) - 1u))] = j;
+            __syncthreads();
+            for (int m = 0; m < total; ++m) {
+                const T* x = feats + (size_t)s_list[m] * d;
+#pragma unroll
+                for (int u = 0; u < kAvgChunks; ++u) {
+                    const int ch = cb + u * kAvgThreads + tid;
+                    if (ch < nchunk) {
+                        float v[VN];
+                        Vec16<T>::load(x + (size_t)ch * VN, v);
+#pragma unroll
+                        for (int q = 0; q < VN; ++q) acc[u][q] += v[q];
+                    }
+                }
+            }
+            count += total;
+            __syncthreads();
+        }
+        const float inv = 1.0f / (float)count;
+#pragma unroll
+        for (int u = 0; u < kAvgChunks; ++u) {
+            const int ch = cb + u * kAvgThreads + tid;
+            if (ch < nchunk) {
+                T* o = out_feats + (size_t)c * d + (size_t)ch * VN;
+                alignas(16) T tmp[VN];
+#pragma unroll
+                for (int q = 0; q < VN; ++q) from_float(tmp[q], acc[u][q] * inv);
+                *reinterpret_cast<uint4*>(o) = *reinterpret_cast<const uint4*>(tmp);
+            }
+        }
+        if (tid == 0 && cb == 0) out_members[c] = count;
+    }
+}
+
+// --------------------------------------------------------------------------- //
+// host side
+// --------------------------------------------------------------------------- //
+struct VisionWs {
+    float* inv_norm;
+    uint8_t* is_key;
+    int32_t *ev_lo, *ev_budget, *ev_out_off, *ev_tile_off;
+};
+
+static VisionWs carve_vision(Carver& cv, int Tn, int N, int k) {
+    VisionWs w;
+    w.inv_norm = cv.take<float>((size_t)Tn * N);
+    w.is_key = cv.take<uint8_t>((size_t)Tn * N);
+    w.ev_lo = cv.take<int32_t>((size_t)k + 1);
+    w.ev_budget = cv.take<int32_t>((size_t)k + 1);
+    w.ev_out_off = cv.take<int32_t>((size_t)k + 1);
+    w.ev_tile_off = cv.take<int32_t>((size_t)k + 1);
+    return w;
+}
+
+static bool ratio_ok(double r) { return r > 0.0 && r <= 1.0; }
+
+template <typename T>
+static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t* event_offsets, int k,
+                         const void* text_, const metok_vision_params* p, void* out_feats_, int32_t* out_src,
+                         int32_t* out_event, int32_t* out_members, int32_t* assign, float* token_score,
+                         float* frame_score, float* event_score, uint8_t* event_is_key, int32_t* n_out, int cap,
+                         void* ws, cudaStream_t st) {
+    const T* feats = reinterpret_cast<const T*>(feats_);
+    const T* text = reinterpret_cast<const T*>(text_);
+    T* out_feats = reinterpret_cast<T*>(out_feats_);
+    const int Nv = Tn * N;
+    Carver cv(ws);
+    VisionWs w = carve_vision(cv, Tn, N, k);
+
+    {
+        const int grid = min(ceil_div(Nv, 8), kNumSMs * 8);
+        const size_t smem = (size_t)d * sizeof(float);
+        if (smem > 48 * 1024)
+            METOK_CUDA_TRY(cudaFuncSetAttribute(tok_score_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)smem));
+        tok_score_kernel<T><<<grid, 256, smem, st>>>(feats, text, Nv, d, token_score, w.inv_norm);
+        METOK_LAUNCH_CHECK();
+    }
+    frame_score_kernel<<<ceil_div(Tn, 8), 256, 0, st>>>(token_score, Tn, N, frame_score);
+    METOK_LAUNCH_CHECK();
+
+    PlanParams pp;
+    pp.Tn = Tn; pp.N = N; pp.k = k;
+    pp.n_key_events = min(k, ceilq(p->alpha * (double)k));
+    pp.event_agg = p->event_agg; pp.mode = p->mode; pp.tile_rows = kMergeTM;
+    pp.keep_key = p->keep_key; pp.keep_nonkey = p->keep_nonkey; pp.beta = p->beta;
+    event_plan_kernel<<<1, 1024, (size_t)k * sizeof(float), st>>>(frame_score, event_offsets, pp, event_score,
+                                                                  event_is_key, w.ev_lo, w.ev_budget, w.ev_out_off,
+                                                                  w.ev_tile_off, n_out);
+    METOK_LAUNCH_CHECK();
+
+    event_topk_kernel<<<k, 1024, 0, st>>>(token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off, w.is_key, out_src,
+                                          out_event, assign);
+    METOK_LAUNCH_CHECK();
+
+    const int max_tiles = Nv / kMergeTM + k;
+    merge_assign_simt_kernel<T><<<max_tiles, 256, 0, st>>>(feats, d, N, w.ev_lo, k, w.ev_out_off, w.ev_tile_off,
+                                                           out_src, w.inv_norm, w.is_key, assign);
+    METOK_LAUNCH_CHECK();
+
+    merge_avg_kernel<T><<<cap, kAvgThreads, 0, st>>>(feats, d, N, w.ev_lo, out_event, assign, n_out, out_feats,
+                                                     out_members);
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
+}
+
+}  // namespace metok
+
+using namespace metok;
+
+static int vision_params_ok(const metok_vision_params* p, int N) {
+    if (!p) return 0;
+    if (!ratio_ok(p->alpha)) return 0;
+    if (p->event_agg != METOK_AGG_MEAN && p->event_agg != METOK_AGG_MAX) return 0;
+    if (p->mode == METOK_MODE_TOPK_MERGE) return ratio_ok(p->keep_key) && ratio_ok(p->keep_nonkey);
+    if (p->mode == METOK_MODE_POOL) {
+        if (!ratio_ok(p->beta)) return 0;
+        if (p->s1 < 1 || p->s2 < 1 || p->s1_nonkey < 1 || p->s2_nonkey < 1) return 0;
+        int g = 1;
+        while (g * g < N) ++g;
+        return g * g == N;
+    }
+    return 0;
+}
+
+extern "C" int metok_compress_vision_bound(int T, int N, int k, const metok_vision_params* p) {
+    if (T < 1 || N < 1 || k < 1 || k > T || !vision_params_ok(p, N)) return METOK_ERR_INVALID_ARG;
+    const long long Nv = (long long)T * N;
+    if (p->mode == METOK_MODE_TOPK_MERGE) {
+        const double r = p->keep_key > p->keep_nonkey ? p->keep_key : p->keep_nonkey;
+        long long b = (long long)ceilq(r * (double)Nv) + k;     // sum of per-event ceilings
+        if (b > Nv) b = Nv;
+        return (int)b;
+    }
+    int smin = p->s1;
+    if (p->s2 < smin) smin = p->s2;
+    if (p->s1_nonkey < smin) smin = p->s1_nonkey;
+    if (p->s2_nonkey < smin) smin = p->s2_nonkey;
+    int g = 1;
+    while (g * g < N) ++g;
+    const int go = (g + smin - 1) / smin;
+    return T * go * go;
+}
+
+extern "C" size_t metok_compress_vision_workspace_bytes(int dtype, int T, int N, int d, int k, int cap,
+                                                        const metok_vision_params* p) {
+    (void)dtype; (void)d; (void)cap; (void)p;
+    if (T < 1 || N < 1 || k < 1) return 0;
+    Carver cv(nullptr);
+    carve_vision(cv, T, N, k);
+    return cv.total();
+}
+
+extern "C" int metok_compress_vision(const void* feats, int dtype, int T, int N, int d,
+                                     const int32_t* event_offsets, int k, const void* text_emb,
+                                     const metok_vision_params* p, void* out_feats, int32_t* out_src,
+                                     int32_t* out_event, int32_t* out_members, int32_t* assign,
+                                     float* token_score, float* frame_score, float* event_score,
+                                     uint8_t* event_is_key, int32_t* n_out, int cap, void* ws, size_t ws_bytes,
+                                     void* stream) {
+    if (!feats || !event_offsets || !text_emb || !p || !out_feats || !out_src || !out_event || !out_members ||
+        !assign || !token_score || !frame_score || !event_score || !event_is_key || !n_out)
+        return METOK_ERR_INVALID_ARG;
+    if (dtype != METOK_F32 && dtype != METOK_BF16) return METOK_ERR_INVALID_ARG;
+    if (T < 1 || N < 1 || d < 1 || k < 1 || k > T) return METOK_ERR_INVALID_ARG;
+    if ((long long)T * N > 0x7FFFFFFFLL / 2) return METOK_ERR_INVALID_ARG;
+    if (!vision_params_ok(p, N)) return METOK_ERR_INVALID_ARG;
+    if (!aligned16(feats) || !aligned16(text_emb) || !aligned16(out_feats)) return METOK_ERR_INVALID_ARG;
+    const int bound = metok_compress_vision_bound(T, N, k, p);
+    if (bound < 0 || cap < bound) return METOK_ERR_INVALID_ARG;
+    const int eb = dtype == METOK_F32 ? 4 : 2;
+    if (((long long)d * eb) % 16 != 0 || T > 8192) return METOK_ERR_UNSUPPORTED;
+    if (p->mode == METOK_MODE_POOL) return METOK_ERR_UNSUPPORTED;
+    const size_t need = metok_compress_vision_workspace_bytes(dtype, T, N, d, k, cap, p);
+    if (!ws || ws_bytes < need || !aligned16(ws)) return METOK_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (dtype == METOK_F32)
+        return launch_vision<float>(feats, T, N, d, event_offsets, k, text_emb, p, out_feats, out_src, out_event,
+                                    out_members, assign, token_score, frame_score, event_score, event_is_key,
+                                    n_out, cap, ws, st);
+    return launch_vision<__nv_bfloat16>(feats, T, N, d, event_offsets, k, text_emb, p, out_feats, out_src,
+                                        out_event, out_members, assign, token_score, frame_score, event_score,
+                                        event_is_key, n_out, cap, ws, st);
+}

@@ -1,0 +1,246 @@
+"""CUDA path vs CPU oracle through the C ABI, on the seeded workloads and on edge
+cases.  Index outputs bit-exact outside the 1e-3 near-tie band; scores and
+features within 2e-2 (bf16) / 1e-5 (fp32); gathers bit-exact."""
+
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import metok_oracle as O
+from paper_2506_02850_b200 import binding as B
+from paper_2506_02850_b200 import workloads as W
+from tests import parity as P
+from tests import runners as R
+
+pytestmark = pytest.mark.gpu
+
+_vis_cache = {}
+
+
+def vis_of(name):
+    if name not in _vis_cache:
+        _vis_cache.clear()                                     # the large ones are several hundred MB
+        _vis_cache[name] = W.vision_inputs(W.CONFIGS[name])
+    return _vis_cache[name]
+
+
+# ------------------------------------------------------------------ a1 ----- #
+
+@pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128", "frames128d1024", "stress"])
+def test_segment_events_workloads(name):
+    cfg = W.CONFIGS[name]
+    vis = vis_of(name)
+    rep = R.segment_case(vis["V"], cfg.dtype, cfg.k, O.SIM_FLATTEN)
+    assert rep["mismatches"] == 0
+    got = B.metok_segment_events(P.to_torch(vis["V"], cfg.dtype), cfg.k)
+    assert np.array_equal(got["boundaries"].cpu().numpy(), vis["boundaries"])   # the planted events
+
+
+@pytest.mark.parametrize("name", ["tiny", "frames32", "frames128d1024"])
+def test_segment_events_meanpool(name):
+    cfg = W.CONFIGS[name]
+    rep = R.segment_case(vis_of(name)["V"], cfg.dtype, cfg.k, O.SIM_MEANPOOL)
+    assert rep["mismatches"] == 0
+
+
+@pytest.mark.parametrize("T,N,d,k,dtype", [
+    (1, 3, 8, 1, "bf16"), (2, 1, 8, 2, "bf16"), (3, 5, 72, 2, "f32"), (9, 7, 40, 9, "bf16"),
+    (17, 33, 200, 5, "bf16"), (40, 130, 264, 1, "f32"), (5, 1030, 1032, 3, "bf16"), (700, 2, 16, 350, "f32")])
+def test_segment_events_ragged(T, N, d, k, dtype):
+    rng = np.random.default_rng(T * 1000 + N)
+    V = W.quantize(rng.standard_normal((T, N, d)).astype(np.float32), dtype)
+    for mode in (O.SIM_FLATTEN, O.SIM_MEANPOOL):
+        R.segment_case(V, dtype, k, mode)
+
+
+def test_segment_events_ties_go_to_lower_index_and_repeatable():
+    base = np.random.default_rng(3).standard_normal((4, 16)).astype(np.float32)
+    V = np.stack([base, base, base, base, -base, -base])      # sims 1,1,1,-1,1 ; ties among the 1s
+    got = B.metok_segment_events(P.to_torch(V, "f32"), 4)
+    assert got["boundaries"].cpu().tolist() == [0, 1, 3]      # the -1, then the two lowest-index ties
+    vis = vis_of("frames32")
+    x = P.to_torch(vis["V"], "bf16")
+    a = B.metok_segment_events(x, 4)["sims"].clone()
+    for _ in range(5):
+        assert torch.equal(a, B.metok_segment_events(x, 4)["sims"])
+
+
+# ------------------------------------------------------------- a2 a3 a4 ---- #
+
+@pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128", "frames128d1024"])
+def test_compress_vision_workloads(name):
+    cfg = W.CONFIGS[name]
+    vis = vis_of(name)
+    rep = R.compress_case(vis["V"], vis["t"], vis["event_offsets"], cfg.dtype, cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+    assert "event_class_flip" not in rep
+    assert rep["key_mismatches"] <= rep["key_near_ties"]
+    assert rep["assign_mismatches"] <= rep["assign_near_ties"]
+    print(name, rep)
+
+
+def test_compress_vision_stress():
+    cfg = W.CONFIGS["stress"]
+    vis = vis_of("stress")
+    rep = R.compress_case(vis["V"], vis["t"], vis["event_offsets"], cfg.dtype, cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+    assert "event_class_flip" not in rep
+    print("stress", rep)
+
+
+@pytest.mark.parametrize("T,N,d,offs,dtype,kk,kn,agg", [
+    (4, 4, 8, [0, 4], "bf16", 0.5, 0.5, 0),
+    (6, 9, 72, [0, 1, 2, 6], "f32", 0.3, 0.1, 1),
+    (12, 36, 136, [0, 3, 4, 9, 12], "bf16", 0.3, 0.1, 0),
+    (10, 25, 264, [0, 5, 10], "bf16", 1.0, 1.0, 0),            # keep everything: identity
+    (7, 16, 40, [0, 1, 2, 3, 4, 5, 6, 7], "f32", 0.01, 0.01, 0),   # one key token per event
+    (5, 130, 64, [0, 2, 5], "bf16", 0.7, 0.05, 1),
+])
+def test_compress_vision_ragged(T, N, d, offs, dtype, kk, kn, agg):
+    rng = np.random.default_rng(T * 100 + N)
+    base = rng.standard_normal((len(offs) - 1, N, d))
+    V = np.concatenate([base[e][None] + 0.3 * rng.standard_normal((offs[e + 1] - offs[e], N, d))
+                        for e in range(len(offs) - 1)]).astype(np.float32)
+    V = W.quantize(V, dtype)
+    t = W.quantize(rng.standard_normal(d).astype(np.float32), dtype)
+    rep = R.compress_case(V, t, np.array(offs, dtype=np.int32), dtype, 0.5, kk, kn, agg)
+    if kk == 1.0:
+        assert rep["n_out"] == T * N
+
+
+def test_compress_vision_identity_is_bit_exact_and_repeatable():
+    cfg = W.CONFIGS["frames32"]
+    vis = vis_of("frames32")
+    V = P.to_torch(vis["V"][:6], "bf16")
+    offs = torch.tensor([0, 2, 6], dtype=torch.int32).cuda()
+    t = P.to_torch(vis["t"], "bf16")
+    out = B.metok_compress_vision(V, offs, t, B.vision_params(0.5, 1.0, 1.0))
+    n = int(out["n_out"].item())
+    assert n == 6 * cfg.N
+    assert torch.equal(out["out_feats"][:n].view(torch.int16), V.reshape(n, -1).view(torch.int16))
+    assert torch.all(out["out_members"][:n] == 1)
+    p = B.vision_params(0.5, 0.3, 0.3)
+    a = B.metok_compress_vision(V, offs, t, p)
+    for _ in range(3):
+        b = B.metok_compress_vision(V, offs, t, p)
+        for key in ("out_feats", "assign", "out_src", "token_score", "out_members"):
+            assert torch.equal(a[key].view(torch.int16) if a[key].dtype == torch.bfloat16 else a[key],
+                               b[key].view(torch.int16) if b[key].dtype == torch.bfloat16 else b[key]), key
+
+
+# ------------------------------------------------------------- a5 a6 a7 ---- #
+
+def _prefill_stage_inputs(cfg, stage, vis):
+    """Shapes of the schedule: stage s sees the survivors of stage s-1."""
+    grp_full = W.token_groups(cfg, cfg.Nv, vis=vis)
+    N0 = [int((grp_full == 0).sum()), int((grp_full == 1).sum())]
+    if stage == 1:
+        groups = grp_full
+    else:
+        prev = O.retention_budgets(cfg.alpha, cfg.keep_prefill, stage - 1, N0)
+        groups = W.token_groups(cfg, int(prev.sum()), n_key=int(prev[0]), stage=stage)
+    budgets = O.retention_budgets(cfg.alpha, cfg.keep_prefill, stage, N0).tolist()
+    return groups, budgets
+
+
+@pytest.mark.parametrize("name,stage", [("tiny", 1), ("frames32", 1), ("frames32", 2), ("frames64", 1),
+                                        ("frames128", 1), ("frames128", 2), ("frames128", 3)])
+def test_prefill_prune_workloads(name, stage):
+    cfg = W.CONFIGS[name]
+    vis = vis_of(name if name != "frames128" else "frames128d1024")
+    groups, budgets = _prefill_stage_inputs(cfg, stage, vis)
+    n_vis = groups.size
+    pf = W.prefill_inputs(cfg, stage, n_vis, groups)
+    hidden = W.payload_torch(W.hidden_salt(cfg, stage), pf["S"], cfg.D, cfg.dtype, "cuda")
+    rep = R.prefill_case(pf["Q"], pf["K"], cfg.dtype, 0, n_vis, groups, budgets, cfg.dh ** -0.5, hidden)
+    assert rep["S_out"] == cfg.Lt + sum(min(b, int((groups == g).sum())) for g, b in enumerate(budgets))
+    print(name, stage, rep)
+
+
+def test_prefill_prune_stress_stage1():
+    cfg = W.CONFIGS["stress"]
+    vis = vis_of("stress")
+    groups, budgets = _prefill_stage_inputs(cfg, 1, vis)
+    pf = W.prefill_inputs(cfg, 1, cfg.Nv, groups)
+    hidden = W.payload_torch(W.hidden_salt(cfg, 1), pf["S"], cfg.D, cfg.dtype, "cuda")
+    rep = R.prefill_case(pf["Q"], pf["K"], cfg.dtype, 0, cfg.Nv, groups, budgets, cfg.dh ** -0.5, hidden)
+    print("stress", rep)
+
+
+@pytest.mark.parametrize("Hq,Hkv,Lt,dh,n_vis,vis_start,G,dtype", [
+    (1, 1, 1, 64, 5, 0, 1, "f32"), (4, 2, 3, 64, 70, 2, 3, "bf16"), (6, 2, 5, 128, 333, 7, 2, "bf16"),
+    (3, 3, 9, 32, 129, 0, 4, "f32"), (8, 1, 17, 128, 1000, 64, 2, "bf16"), (2, 2, 70, 64, 64, 1, 1, "bf16")])
+def test_prefill_prune_ragged(Hq, Hkv, Lt, dh, n_vis, vis_start, G, dtype):
+    rng = np.random.default_rng(Hq * 100 + n_vis)
+    S = vis_start + n_vis + 3 + Lt                              # 3 extra non-visual tokens before the text queries
+    Q = W.quantize(rng.standard_normal((Hq, Lt, dh)).astype(np.float32), dtype)
+    K = W.quantize(rng.standard_normal((Hkv, S, dh)).astype(np.float32), dtype)
+    groups = rng.integers(0, G, size=n_vis).astype(np.int32)
+    budgets = [int(rng.integers(0, n_vis // G + 3)) for _ in range(G)]
+    budgets[0] = 0 if G > 1 else budgets[0]                     # a class that keeps nothing
+    hidden = W.payload_torch(5, S, 24, dtype, "cuda")
+    R.prefill_case(Q, K, dtype, vis_start, n_vis, groups, budgets, 0.3, hidden)
+    big = [n_vis + 5] * G                                       # budgets above the population keep everything
+    rep = R.prefill_case(Q, K, dtype, vis_start, n_vis, groups, big, 0.3, hidden)
+    assert rep["S_out"] == S
+
+
+def test_prefill_prune_tied_scores_keep_lower_index():
+    # identical keys => identical scores: the budget must take the lowest indices of each class
+    Hq, Lt, dh, n_vis = 2, 2, 64, 50
+    Q = np.ones((Hq, Lt, dh), dtype=np.float32)
+    K = np.ones((1, n_vis + Lt, dh), dtype=np.float32)
+    groups = (np.arange(n_vis) % 2).astype(np.int32)
+    got = B.metok_prefill_prune(P.to_torch(Q, "bf16"), P.to_torch(K, "bf16"), None, 0, n_vis,
+                                torch.from_numpy(groups).cuda(), [3, 4], 0.125)
+    n = int(got["S_out"].item())
+    assert got["keep_idx"][:n].cpu().tolist() == [0, 1, 2, 3, 4, 5, 7, 50, 51]
+
+
+# ------------------------------------------------------------- a8 a9 ------- #
+
+@pytest.mark.parametrize("name,policy", [("tiny", O.KV_TOPK), ("tiny", O.KV_PAPER), ("tiny", O.KV_GIVEN),
+                                         ("frames32", O.KV_TOPK), ("frames32", O.KV_PAPER),
+                                         ("frames32", O.KV_GIVEN), ("frames64", O.KV_TOPK),
+                                         ("frames128", O.KV_TOPK), ("frames128", O.KV_PAPER)])
+def test_kv_compact_workloads(name, policy):
+    cfg = W.CONFIGS[name]
+    l1 = 3 if cfg.L > 3 else 0
+    rep = R.kv_case(cfg, policy, l1=l1, given_from=7)
+    print(name, policy, rep)
+
+
+def test_kv_compact_stress_and_per_layer_scores():
+    R.kv_case(W.CONFIGS["stress"], O.KV_TOPK, sample_slabs=6)
+    torch.cuda.empty_cache()
+    R.kv_case(W.CONFIGS["frames32"], O.KV_TOPK, per_layer_scores=True)
+
+
+@pytest.mark.parametrize("ratio", [0.0, 0.03, 0.5, 0.97, 1.0])
+def test_kv_compact_ratios_and_fp32_rows(ratio):
+    import dataclasses
+    cfg = dataclasses.replace(W.CONFIGS["tiny"], T=37, N=29, dh=36, Hkv=3, L=5, kv_text=11, keep_kv=ratio)
+    R.kv_case(cfg, O.KV_TOPK)
+    cfg2 = dataclasses.replace(W.CONFIGS["frames32"], T=9, N=33, dh=24, Hkv=2, L=3, kv_text=5, keep_kv=ratio)
+    R.kv_case(cfg2, O.KV_TOPK)
+
+
+# ------------------------------------------------------------- chained ----- #
+
+def test_chained_pipeline_tiny_and_frames32():
+    """segment -> compress on the GPU's own event offsets; both must equal the oracle's chain."""
+    for name in ("tiny", "frames32"):
+        cfg = W.CONFIGS[name]
+        vis = vis_of(name)
+        Vd = P.to_torch(vis["V"], cfg.dtype)
+        seg = B.metok_segment_events(Vd, cfg.k)
+        p = B.vision_params(cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+        out = B.metok_compress_vision(Vd, seg["event_offsets"], P.to_torch(vis["t"], cfg.dtype), p)
+        want_seg = O.segment_events(vis["V"], cfg.k)
+        want = O.compress_vision(vis["V"], vis["t"], want_seg["event_offsets"], cfg.alpha, cfg.keep_enc,
+                                 cfg.keep_enc, cfg.dtype)
+        n = int(out["n_out"].item())
+        assert n == want["n_out"]
+        assert np.array_equal(out["event_is_key"].cpu().numpy(), want["event_is_key"])
+        same = np.mean(out["out_src"][:n].cpu().numpy() == want["out_src"])
+        assert same > 0.99

@@ -1,0 +1,468 @@
+#!/usr/bin/env python
+"""Benchmark of the METok hot path on B200.
+
+A "step" is one pass of the whole hot path over one synthetic video of the
+128-frame workload (128 x 144 visual tokens, 28-layer 7B-shaped LLM): event
+segmentation, stage-1 compression, the three prefill pruning levels at the
+sizes the Eq. 6/7 schedule implies, and the KV-cache compaction -- all through
+the C ABI.  `value` = visual tokens entering the path per second, inputs resident
+in HBM; `e2e` = the same with every step's inputs copied from pinned host memory
+and its results copied back inside the timed region.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run) every rank compresses its own
+video: independent replicas, no data-path collective, weak scaling.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2506_02850_b200 import workloads as W
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu
+# captures (profiles/), keyed by (kernel, workload); absent -> null in the JSON line.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+# --------------------------------------------------------------------------- #
+# workload
+# --------------------------------------------------------------------------- #
+
+
+def schedule(cfg, B, vis):
+    """Per pruning level: class labels and Eq. 6/7 budgets at the sizes the schedule implies."""
+    grp_full = W.token_groups(cfg, cfg.Nv, vis=vis)
+    N0 = [int((grp_full == 0).sum()), int((grp_full == 1).sum())]
+    stages = []
+    for stage in range(1, cfg.n_stages + 1):
+        if stage == 1:
+            groups = grp_full
+        else:
+            prev = B.metok_retention_budgets(cfg.alpha, cfg.keep_prefill, stage - 1, N0)
+            groups = W.token_groups(cfg, int(sum(prev)), n_key=int(prev[0]), stage=stage)
+        budgets = B.metok_retention_budgets(cfg.alpha, cfg.keep_prefill, stage, N0)
+        stages.append((groups, budgets))
+    return stages
+
+
+class Workload:
+    def __init__(self, cfg, device, host_copies: bool):
+        from paper_2506_02850_b200 import binding as B
+        self.B = B
+        self.cfg = cfg
+        self.dev = device
+        tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+        vis = W.vision_inputs(cfg)
+        self.vis = vis
+        self.h = {}                                   # pinned host inputs (e2e only)
+
+        def put(name, arr_or_tensor):
+            t = arr_or_tensor if isinstance(arr_or_tensor, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(arr_or_tensor))
+            if t.dtype == torch.float32 and tdt == torch.bfloat16 and name not in ("kv_scores",):
+                t = t.to(torch.bfloat16)
+            if host_copies:
+                self.h[name] = t.cpu().pin_memory()
+            return t.to(device)
+
+        self.V = put("V", vis["V"])
+        self.t = put("t", vis["t"])
+        self.params = B.vision_params(cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+        self.stages = []
+        for si, (groups, budgets) in enumerate(schedule(cfg, B, vis), start=1):
+            pf = W.prefill_inputs(cfg, si, groups.size, groups)
+            hidden = W.payload_torch(W.hidden_salt(cfg, si), pf["S"], cfg.D, cfg.dtype, device)
+            self.stages.append({
+                "Q": put(f"Q{si}", pf["Q"]), "K": put(f"K{si}", pf["K"]),
+                "hidden": put(f"hidden{si}", hidden), "groups": put(f"groups{si}", groups.astype(np.int32)),
+                "budgets": budgets, "n_vis": int(groups.size), "S": int(pf["S"]),
+            })
+        self.kv_layers = cfg.L
+        self.S_cur = cfg.Nv + cfg.kv_text
+        self.ks, self.vs = W.kv_cache_torch(cfg, device)
+        if host_copies:
+            self.h["ks"] = [t.cpu().pin_memory() for t in self.ks]
+            self.h["vs"] = [t.cpu().pin_memory() for t in self.vs]
+        self.kv_scores = torch.from_numpy(W.kv_scores(cfg, cfg.Nv)).to(device)
+        self.out = {}
+        self.scale = float(cfg.dh ** -0.5)
+
+    # one pass of the hot path, device-resident inputs
+    def step(self):
+        B, cfg, o = self.B, self.cfg, self.out
+        o["seg"] = B.metok_segment_events(self.V, cfg.k, out=o.get("seg"))
+        o["cv"] = B.metok_compress_vision(self.V, o["seg"]["event_offsets"], self.t, self.params, out=o.get("cv"))
+        for i, s in enumerate(self.stages):
+            o[f"pf{i}"] = B.metok_prefill_prune(s["Q"], s["K"], s["hidden"], 0, s["n_vis"], s["groups"], s["budgets"],
+                                                self.scale, out=o.get(f"pf{i}"))
+        # KV selection uses the first pruning layer's attention scores (n_vis = all visual tokens)
+        scores = o["pf0"]["scores"] if self.stages and self.stages[0]["n_vis"] == cfg.Nv else self.kv_scores
+        kv = o.get("kv")
+        o["kv"] = B.metok_kv_compact(self.ks, self.vs, self.S_cur, B.KV_TOPK, 0, cfg.Nv, keep_ratio=cfg.keep_kv,
+                                     scores=scores, keep_idx=None if kv is None else kv["keep_idx"],
+                                     keep_len=None if kv is None else kv["keep_len"],
+                                     new_len=None if kv is None else kv["new_len"])
+
+    # the same with host buffers: H2D of every input, D2H of every result
+    def e2e_alloc(self):
+        self.d2h = {}
+        self.step()
+        torch.cuda.synchronize()
+        o = self.out
+        n_out = int(o["cv"]["n_out"].item())
+        self.n_out = n_out
+        self.d2h["out_feats"] = torch.empty((n_out, self.cfg.d), dtype=self.V.dtype).pin_memory()
+        self.d2h["out_src"] = torch.empty(n_out, dtype=torch.int32).pin_memory()
+        self.d2h["offsets"] = torch.empty(self.cfg.k + 1, dtype=torch.int32).pin_memory()
+        for i, s in enumerate(self.stages):
+            so = int(o[f"pf{i}"]["S_out"].item())
+            s["S_out"] = so
+            self.d2h[f"keep{i}"] = torch.empty(so, dtype=torch.int32).pin_memory()
+            self.d2h[f"hidden{i}"] = torch.empty((so, self.cfg.D), dtype=self.V.dtype).pin_memory()
+        self.kv_new = int(o["kv"]["new_len"][0].item())
+        self.d2h["kv_k"] = [torch.empty((self.cfg.Hkv, self.kv_new, self.cfg.dh), dtype=self.V.dtype).pin_memory()
+                            for _ in range(self.kv_layers)]
+        self.d2h["kv_v"] = [torch.empty((self.cfg.Hkv, self.kv_new, self.cfg.dh), dtype=self.V.dtype).pin_memory()
+                            for _ in range(self.kv_layers)]
+        h2d = sum(t.numel() * t.element_size() for k_, t in self.h.items() if isinstance(t, torch.Tensor))
+        h2d += sum(t.numel() * t.element_size() for t in self.h["ks"] + self.h["vs"])
+        d2h = sum(t.numel() * t.element_size() for k_, t in self.d2h.items() if isinstance(t, torch.Tensor))
+        d2h += sum(t.numel() * t.element_size() for t in self.d2h["kv_k"] + self.d2h["kv_v"])
+        return h2d, d2h
+
+    def e2e_step(self):
+        h, o = self.h, self.out
+        self.V.copy_(h["V"], non_blocking=True)
+        self.t.copy_(h["t"], non_blocking=True)
+        for i, s in enumerate(self.stages, start=1):
+            s["Q"].copy_(h[f"Q{i}"], non_blocking=True)
+            s["K"].copy_(h[f"K{i}"], non_blocking=True)
+            s["hidden"].copy_(h[f"hidden{i}"], non_blocking=True)
+            s["groups"].copy_(h[f"groups{i}"], non_blocking=True)
+        for d, s in zip(self.ks, h["ks"]):
+            d.copy_(s, non_blocking=True)
+        for d, s in zip(self.vs, h["vs"]):
+            d.copy_(s, non_blocking=True)
+        self.step()
+        self.d2h["out_feats"].copy_(o["cv"]["out_feats"][: self.n_out], non_blocking=True)
+        self.d2h["out_src"].copy_(o["cv"]["out_src"][: self.n_out], non_blocking=True)
+        self.d2h["offsets"].copy_(o["seg"]["event_offsets"], non_blocking=True)
+        for i, s in enumerate(self.stages):
+            self.d2h[f"keep{i}"].copy_(o[f"pf{i}"]["keep_idx"][: s["S_out"]], non_blocking=True)
+            self.d2h[f"hidden{i}"].copy_(o[f"pf{i}"]["hidden_out"][: s["S_out"]], non_blocking=True)
+        for l in range(self.kv_layers):
+            self.d2h["kv_k"][l].copy_(self.ks[l][:, : self.kv_new], non_blocking=True)
+            self.d2h["kv_v"][l].copy_(self.vs[l][:, : self.kv_new], non_blocking=True)
+
+    # algorithmic work of one step per kernel name: (bound, bytes or flops)
+    def algorithmic_work(self):
+        cfg = self.cfg
+        b = cfg.elem_bytes
+        Nv, d = cfg.Nv, cfg.d
+        lens = np.asarray(self.vis["lengths"]) * cfg.N
+        k_e = np.array([min(m, max(1, math.ceil(cfg.keep_enc * m - 1e-9))) for m in lens])
+        n_out = int(k_e.sum())
+        merge_flops = float(np.sum(2.0 * (lens - k_e) * k_e * d))
+        attn_flops = sum(2.0 * cfg.Hq * cfg.Lt * s["S"] * cfg.dh for s in self.stages)
+        hidden_bytes = sum(2.0 * (cfg.Lt + sum(min(bg, int((s["groups"] == g).sum().item()))
+                                               for g, bg in enumerate(s["budgets"]))) * cfg.D * b
+                           for s in self.stages)
+        kv_rows = min(cfg.Nv, math.ceil(cfg.keep_kv * cfg.Nv - 1e-9)) + cfg.kv_text
+        work = {
+            "seg_partial_kernel": ("hbm", float(Nv) * d * b),
+            "tok_score_kernel": ("hbm", float(Nv) * d * b),
+            "merge_assign_simt_kernel": ("tensor", merge_flops),
+            "merge_assign_mma_kernel": ("tensor", merge_flops),
+            "merge_avg_kernel": ("hbm", float(Nv) * d * b + float(n_out) * d * b),
+            "attn_stats_kernel": ("tensor", attn_flops),
+            "attn_colsum_kernel": ("tensor", attn_flops),
+            "attn_stats_mma_kernel": ("tensor", attn_flops),
+            "attn_colsum_mma_kernel": ("tensor", attn_flops),
+            "gather_rows_kernel": ("hbm", hidden_bytes),
+            "kv_gather_kernel": ("hbm", 2.0 * kv_rows * cfg.dh * b * 2 * cfg.Hkv * cfg.L),
+            "class_topk_kernel": ("hbm", 8.0 * (sum(s["n_vis"] for s in self.stages) + cfg.L * cfg.Nv)),
+            "event_topk_kernel": ("hbm", 8.0 * Nv),
+        }
+        return work
+
+
+# --------------------------------------------------------------------------- #
+# clocks
+# --------------------------------------------------------------------------- #
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+            self.f.close()
+            rows = [r.strip().split(",") for r in open(self.path) if r.strip()]
+            os.unlink(self.path)
+            sm = [float(r[0]) for r in rows if len(r) >= 6]
+            if sm:
+                out["sm_mhz"] = float(np.median(sm))
+                out["sm_max_mhz"] = float(rows[0][1])
+                names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+                for j, n in enumerate(names):
+                    if any(r[2 + j].strip().lower().startswith("active") for r in rows if len(r) >= 6):
+                        out["reasons"].append(n)
+                out["samples"] = len(sm)
+        except Exception:
+            pass
+        return out
+
+
+# --------------------------------------------------------------------------- #
+# CPU baseline: the oracle, as it stands, on a bounded sample of the workload
+# --------------------------------------------------------------------------- #
+
+
+def oracle_sample_step(cfg, sample):
+    """One pass of the oracle over the sample (a prefix of the video, fewer KV layers)."""
+    from oracle import metok_oracle as O
+    V, t, offs, groups, budgets, Q, K, hidden, kv = sample
+    O.segment_events(V, len(offs) - 1)
+    O.compress_vision(V, t, offs, cfg.alpha, cfg.keep_enc, cfg.keep_enc, cfg.dtype)
+    pr = O.prefill_prune(Q, K, hidden, 0, groups.size, groups, budgets, cfg.dh ** -0.5)
+    lists = O.kv_select(O.KV_TOPK, len(kv[0]), kv[0][0].shape[1], 0, groups.size, keep_ratio=cfg.keep_kv,
+                        scores=pr["scores"])
+    O.kv_compact(kv[0], kv[1], lists)
+
+
+def oracle_sample(cfg, frames=24, kv_layers=2):
+    from oracle import metok_oracle as O
+    vis = W.vision_inputs(cfg)
+    T = min(frames, cfg.T)
+    V = vis["V"][:T]
+    offs = np.unique(np.clip(vis["event_offsets"], 0, T)).astype(np.int32)
+    n_vis = T * cfg.N
+    groups = W.token_groups(cfg, cfg.Nv, vis=vis)[:n_vis]
+    N0 = [int((groups == 0).sum()), int((groups == 1).sum())]
+    budgets = O.retention_budgets(cfg.alpha, cfg.keep_prefill, 1, N0).tolist()
+    pf = W.prefill_inputs(cfg, 1, n_vis, groups)
+    hidden = W.payload_rows_np(W.hidden_salt(cfg, 1), np.arange(pf["S"]), cfg.D, cfg.dtype)
+    S = n_vis + cfg.kv_text
+    kv = ([np.stack([W.payload_rows_np(W.kv_salt(cfg, l, w, h), np.arange(S), cfg.dh, cfg.dtype)
+                     for h in range(cfg.Hkv)]) for l in range(kv_layers)] for w in (0, 1))
+    kv = tuple(kv)
+    what = (f"first {T} of {cfg.T} frames ({n_vis} visual tokens): segmentation, stage-1 compression, "
+            f"pruning level 1, KV TOPK compaction of {kv_layers} of {cfg.L} layers")
+    return (V, vis["t"], offs, groups, budgets, pf["Q"], pf["K"], hidden, kv), n_vis, what
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(cfg, steps, warmup):
+    sample, n_tok, what = oracle_sample(cfg)
+    for _ in range(warmup):
+        oracle_sample_step(cfg, sample)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_sample_step(cfg, sample)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    return n_tok / dt, dt, what
+
+
+# --------------------------------------------------------------------------- #
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="frames128")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = W.CONFIGS[args.config]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    workload_name = (f"{cfg.name}: {cfg.T} frames x {cfg.N} tokens, d={cfg.d} {cfg.dtype}, k={cfg.k} events, "
+                     f"{cfg.Lt} text tokens, {cfg.Hq}/{cfg.Hkv} heads dh={cfg.dh}, hidden {cfg.D}, "
+                     f"{cfg.n_stages} pruning levels, {cfg.L}-layer K/V cache, keep {cfg.keep_enc}/{cfg.keep_prefill}/{cfg.keep_kv}")
+
+    if args.impl == "reference":
+        # the oracle on the host cores; rank 0 alone
+        if rank != 0:
+            return
+        W_ = max(args.warmup, 0)
+        val, dt, what = time_oracle(cfg, args.steps, min(W_, 1))
+        line = {"impl": "reference", "metric": "visual_tokens_per_s", "value": val, "unit": "tokens/s",
+                "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                "data": "synthetic", "config": {"workload": workload_name},
+                "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cpu_threads(), "kind": "oracle",
+                                 "sample": what},
+                "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the METok hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2506_02850_b200 import binding as B
+    B.lib()
+    wl = Workload(cfg, dev, host_copies=not args.no_e2e)
+    warm = max(args.warmup, 3)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        for _ in range(warm):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            tms = torch.tensor([ms], device=dev)
+            dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+            ms = float(tms.item())
+        return ms
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    total_ms = timed(wl.step, args.steps)
+    clocks = sampler.stop()
+    ms_per_step = total_ms / args.steps
+    value = world * cfg.Nv / (ms_per_step * 1e-3)
+
+    # per-kernel times: the same K steps again with the library's event brackets on
+    barrier()
+    B.metok_profile_begin()
+    for _ in range(args.steps):
+        wl.step()
+    prof = B.metok_profile_end()
+    launches_per_step = sum(v["launches"] for v in prof.values()) // args.steps
+    work = wl.algorithmic_work()
+    peaks = load_peaks()
+    kern_ms = {k_: v["ms"] / args.steps for k_, v in prof.items()}
+    top = max(kern_ms, key=kern_ms.get)
+    bound, units = work.get(top, ("hbm", float("nan")))
+    if bound == "tensor":
+        achieved = units / (kern_ms[top] * 1e-3) / 1e12
+        peak, unit = float(peaks["bf16_tflops_sustained"]), "TFLOP/s"
+    else:
+        achieved = units / (kern_ms[top] * 1e-3) / 1e9
+        peak, unit = float(peaks["hbm_gbs"]), "GB/s"
+    roofline = {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "peak_source": peaks["_source"],
+                "traffic": NCU_TRAFFIC_BYTES.get((top, cfg.name)),
+                "ms_per_step_in_kernel": kern_ms[top],
+                "per_kernel": {}}
+    for k_, ms in sorted(kern_ms.items(), key=lambda kv: -kv[1]):
+        bd, u = work.get(k_, (None, None))
+        ent = {"ms": round(ms, 5), "launches": prof[k_]["launches"] // args.steps}
+        if bd == "tensor":
+            ent["TFLOP/s"] = round(u / (ms * 1e-3) / 1e12, 2)
+            ent["frac"] = round(ent["TFLOP/s"] / float(peaks["bf16_tflops_sustained"]), 4)
+        elif bd == "hbm":
+            ent["GB/s"] = round(u / (ms * 1e-3) / 1e9, 1)
+            ent["frac"] = round(ent["GB/s"] / float(peaks["hbm_gbs"]), 4)
+        roofline["per_kernel"][k_] = ent
+
+    e2e = None
+    if not args.no_e2e:
+        h2d, d2h = wl.e2e_alloc()
+        e2e_steps = max(3, min(args.steps, 10))
+        ms = timed(wl.e2e_step, e2e_steps) / e2e_steps
+        e2e = {"value": world * cfg.Nv / (ms * 1e-3), "unit": "tokens/s", "ms_per_step": ms,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, dt, what = time_oracle(cfg, 1, 0)
+        cpu = {"value": v, "unit": "tokens/s", "cores": cpu_threads(), "kind": "oracle", "sample": what,
+               "seconds": dt}
+
+    if rank == 0:
+        line = {"metric": "visual_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+                "steps": args.steps, "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+                "config": {"workload": workload_name, "l2": "inputs larger than L2 (V 132 MB, hidden 133 MB, K/V 1.06 GB touched between reuses)",
+                           "parallelism": f"replicas x{world}"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+                "roofline": roofline, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

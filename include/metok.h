@@ -242,6 +242,17 @@ METOK_API int metok_kv_compact(void* const* k_layers, void* const* v_layers, int
 /* ------------------------------------------------------------------------- *
  * helpers (host only, no CUDA work)
  * ------------------------------------------------------------------------- */
+/* Per-kernel timing for benchmarks.  Between metok_profile_begin() and
+ * metok_profile_end() every kernel the library launches is bracketed by CUDA
+ * events on the launching stream.  metok_profile_end synchronises with those
+ * events and writes one text line per kernel name, "name launches total_ms\n",
+ * in first-launch order, into `out` (HOST, `cap` bytes, NUL-terminated; truncated
+ * if too small).  Returns the number of kernel launches recorded, or a negative
+ * status.  Not thread-safe against concurrent calls into the library; adds two
+ * event records per launch, so never leave it on outside a measurement. */
+METOK_API int metok_profile_begin(void);
+METOK_API int metok_profile_end(char* out, size_t cap);
+
 METOK_API const char* metok_status_string(int status);
 METOK_API int metok_last_cuda_error(void);   /* cudaError_t of the last METOK_ERR_CUDA on this thread, else 0 */
 METOK_API int metok_version(void);           /* major*10000 + minor*100 + patch */

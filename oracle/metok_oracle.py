@@ -76,6 +76,14 @@ def round_out(x: np.ndarray, dtype: str) -> np.ndarray:
     return np.asarray(x, dtype=np.float64).astype(np.float32).astype(np.float64)
 
 
+def near_threshold(s: np.ndarray, tau: float) -> np.ndarray:
+    """Near-tie band of a top-k decision: scores within 1e-3 (relative to the
+    threshold score tau, the last one kept) of the threshold.  For thresholds
+    close to zero the band is floored at 1e-3 of 1e-3 of the largest |score|."""
+    floor = NEAR_TIE * max(float(np.max(np.abs(s))), 1e-300)
+    return np.abs(s - tau) < NEAR_TIE * max(abs(float(tau)), floor)
+
+
 def _order_desc(score: np.ndarray) -> np.ndarray:
     """Indices sorted by (score descending, index ascending)."""
     return np.lexsort((np.arange(score.size), -score))
@@ -191,8 +199,7 @@ def key_token_topk(token_score: np.ndarray, N: int, event_offsets: np.ndarray, e
         budgets[e] = k_e
         order = _order_desc(s)
         is_key_token[lo + order[:k_e]] = 1
-        tau = s[order[k_e - 1]]
-        near[lo:hi] = np.abs(s - tau) < NEAR_TIE * max(float(np.max(np.abs(s))), 1e-300)
+        near[lo:hi] = near_threshold(s, s[order[k_e - 1]])
     key_idx = np.nonzero(is_key_token)[0].astype(np.int32)
     return {"is_key_token": is_key_token, "key_idx": key_idx, "event_budget": budgets, "near_tie": near}
 
@@ -399,8 +406,7 @@ def weighted_topk(scores: np.ndarray, token_group: np.ndarray, group_budget: Seq
         order = _order_desc(s)
         keep_vis[idx[order[:n]]] = True
         if n < idx.size:
-            tau = s[order[n - 1]]
-            near[idx] = np.abs(s - tau) < NEAR_TIE * max(float(np.max(np.abs(s))), 1e-300)
+            near[idx] = near_threshold(s, s[order[n - 1]])
     keep = np.ones(S, dtype=bool)
     keep[vis_start:vis_start + n_vis] = keep_vis
     keep_idx = np.nonzero(keep)[0].astype(np.int32)

@@ -55,6 +55,8 @@ _SIGNATURES = {
     "metok_kv_compact_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "metok_kv_compact": (_i, [_c.POINTER(_vp), _c.POINTER(_vp), _i, _i, _i, _i, _i, _i, _i, _i, _d, _i, _i,
                               _vp, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "metok_profile_begin": (_i, []),
+    "metok_profile_end": (_i, [_c.c_char_p, _sz]),
     "metok_status_string": (_c.c_char_p, [_i]),
     "metok_last_cuda_error": (_i, []),
     "metok_version": (_i, []),
@@ -130,22 +132,27 @@ def workspace(nbytes: int, device) -> torch.Tensor:
 # --------------------------------------------------------------------------- #
 
 
-def metok_segment_events(feats: torch.Tensor, k: int, sim_mode: int = SIM_FLATTEN) -> Dict[str, torch.Tensor]:
+def metok_segment_events(feats: torch.Tensor, k: int, sim_mode: int = SIM_FLATTEN,
+                         out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """`out` (a dict returned by an earlier call with the same shapes) reuses its buffers."""
     feats = _cuda_contig(feats, "feats")
     T, N, d = feats.shape
     dev = feats.device
     L = lib()
-    sims = torch.empty(max(T - 1, 1), dtype=torch.float32, device=dev)
-    boundaries = torch.empty(max(k - 1, 1), dtype=torch.int32, device=dev)
-    offsets = torch.empty(max(k + 1, 2), dtype=torch.int32, device=dev)
-    frame_event = torch.empty(T, dtype=torch.int32, device=dev)
+    if out is not None:
+        sims, boundaries, offsets, frame_event = out["_sims"], out["_boundaries"], out["_offsets"], out["frame_event"]
+    else:
+        sims = torch.empty(max(T - 1, 1), dtype=torch.float32, device=dev)
+        boundaries = torch.empty(max(k - 1, 1), dtype=torch.int32, device=dev)
+        offsets = torch.empty(max(k + 1, 2), dtype=torch.int32, device=dev)
+        frame_event = torch.empty(T, dtype=torch.int32, device=dev)
     need = L.metok_segment_events_workspace_bytes(_dt(feats), T, N, d, sim_mode)
     ws = workspace(need, dev)
     st = L.metok_segment_events(_ptr(feats), _dt(feats), T, N, d, k, sim_mode, _ptr(sims), _ptr(boundaries),
                                 _ptr(offsets), _ptr(frame_event), _ptr(ws), ws.numel(), _stream())
     _check("metok_segment_events", st)
     return {"sims": sims[: T - 1], "boundaries": boundaries[: max(k - 1, 0)], "event_offsets": offsets[: k + 1],
-            "frame_event": frame_event}
+            "frame_event": frame_event, "_sims": sims, "_boundaries": boundaries, "_offsets": offsets}
 
 
 def vision_params(alpha: float, keep_key: float = 1.0, keep_nonkey: float = 1.0, event_agg: int = AGG_MEAN,
@@ -162,7 +169,8 @@ def metok_compress_vision_bound(T: int, N: int, k: int, p: VisionParams) -> int:
 
 
 def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text_emb: torch.Tensor,
-                          p: VisionParams, cap: Optional[int] = None) -> Dict[str, torch.Tensor]:
+                          p: VisionParams, cap: Optional[int] = None,
+                          out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
     feats = _cuda_contig(feats, "feats")
     event_offsets = _cuda_contig(event_offsets, "event_offsets")
     text_emb = _cuda_contig(text_emb, "text_emb")
@@ -173,16 +181,19 @@ def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text
     if cap is None:
         cap = metok_compress_vision_bound(T, N, k, p)
     i32 = dict(dtype=torch.int32, device=dev)
-    out = {
-        "out_feats": torch.empty((cap, d), dtype=feats.dtype, device=dev),
-        "out_src": torch.empty(cap, **i32), "out_event": torch.empty(cap, **i32),
-        "out_members": torch.empty(cap, **i32), "assign": torch.empty(T * N, **i32),
-        "token_score": torch.empty(T * N, dtype=torch.float32, device=dev),
-        "frame_score": torch.empty(T, dtype=torch.float32, device=dev),
-        "event_score": torch.empty(k, dtype=torch.float32, device=dev),
-        "event_is_key": torch.empty(k, dtype=torch.uint8, device=dev),
-        "n_out": torch.zeros(1, **i32),
-    }
+    if out is not None:
+        cap = out["out_src"].numel()
+    else:
+        out = {
+            "out_feats": torch.empty((cap, d), dtype=feats.dtype, device=dev),
+            "out_src": torch.empty(cap, **i32), "out_event": torch.empty(cap, **i32),
+            "out_members": torch.empty(cap, **i32), "assign": torch.empty(T * N, **i32),
+            "token_score": torch.empty(T * N, dtype=torch.float32, device=dev),
+            "frame_score": torch.empty(T, dtype=torch.float32, device=dev),
+            "event_score": torch.empty(k, dtype=torch.float32, device=dev),
+            "event_is_key": torch.empty(k, dtype=torch.uint8, device=dev),
+            "n_out": torch.zeros(1, **i32),
+        }
     need = L.metok_compress_vision_workspace_bytes(_dt(feats), T, N, d, k, cap, _c.byref(p))
     ws = workspace(need, dev)
     st = L.metok_compress_vision(_ptr(feats), _dt(feats), T, N, d, _ptr(event_offsets), k, _ptr(text_emb),
@@ -237,7 +248,8 @@ def metok_prefill_prune(q_text: torch.Tensor, k_all: torch.Tensor, hidden: Optio
 def metok_kv_compact(k_layers: Sequence[torch.Tensor], v_layers: Sequence[torch.Tensor], S_cur: int, policy: int,
                      vis_start: int, n_vis: int, l1: int = 0, keep_ratio: float = 1.0,
                      scores: Optional[torch.Tensor] = None, keep_idx: Optional[torch.Tensor] = None,
-                     keep_len: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+                     keep_len: Optional[torch.Tensor] = None,
+                     new_len: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
     nl = len(k_layers)
     for t in list(k_layers) + list(v_layers):
         _cuda_contig(t, "k/v layer")
@@ -249,7 +261,8 @@ def metok_kv_compact(k_layers: Sequence[torch.Tensor], v_layers: Sequence[torch.
     if keep_idx is None:
         keep_idx = torch.empty((nl, S_cur), dtype=torch.int32, device=dev)
         keep_len = torch.zeros(nl, dtype=torch.int32, device=dev)
-    new_len = torch.zeros(nl, dtype=torch.int32, device=dev)
+    if new_len is None:
+        new_len = torch.zeros(nl, dtype=torch.int32, device=dev)
     per_layer = 0
     if scores is not None:
         scores = _cuda_contig(scores, "scores")
@@ -265,3 +278,20 @@ def metok_kv_compact(k_layers: Sequence[torch.Tensor], v_layers: Sequence[torch.
 
 def metok_version() -> int:
     return lib().metok_version()
+
+
+def metok_profile_begin() -> None:
+    _check("metok_profile_begin", lib().metok_profile_begin())
+
+
+def metok_profile_end() -> Dict[str, Dict[str, float]]:
+    """{kernel name: {"launches": n, "ms": total}} for the launches since metok_profile_begin."""
+    buf = _c.create_string_buffer(1 << 16)
+    n = lib().metok_profile_end(buf, len(buf))
+    if n < 0:
+        _check("metok_profile_end", n)
+    out: Dict[str, Dict[str, float]] = {}
+    for line in buf.value.decode().splitlines():
+        name, cnt, ms = line.split()
+        out[name] = {"launches": int(cnt), "ms": float(ms)}
+    return out

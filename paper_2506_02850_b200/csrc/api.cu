@@ -1,10 +1,78 @@
 // Host-only helpers of the C ABI: status strings, last CUDA error, version.
+#include <mutex>
+#include <string>
+#include <vector>
+#include <cstdio>
+#include <cstring>
+
 #include "common.cuh"
 
 namespace metok {
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+
+bool g_profiling = false;
+namespace {
+struct Rec { const char* name; cudaEvent_t a, b; };
+std::vector<Rec> g_recs;
+std::mutex g_mu;
+}  // namespace
+
+KernelTimer::KernelTimer(const char* n, cudaStream_t s) : name(n), st(s), a(nullptr), b(nullptr), active(g_profiling) {
+    if (!active) return;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { active = false; return; }
+    cudaEventRecord(a, st);
+}
+KernelTimer::~KernelTimer() {
+    if (!active) return;
+    cudaEventRecord(b, st);
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_recs.push_back({name, a, b});
+}
 }  // namespace metok
+
+extern "C" int metok_profile_begin(void) {
+    std::lock_guard<std::mutex> lk(metok::g_mu);
+    for (auto& r : metok::g_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    metok::g_recs.clear();
+    metok::g_profiling = true;
+    return METOK_OK;
+}
+
+extern "C" int metok_profile_end(char* out, size_t cap) {
+    metok::g_profiling = false;
+    std::lock_guard<std::mutex> lk(metok::g_mu);
+    struct Agg { const char* name; int n; double ms; };
+    std::vector<Agg> agg;
+    int launches = 0;
+    for (auto& r : metok::g_recs) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&ms, r.a, r.b) != cudaSuccess) {
+            metok::set_last_cuda_error((int)cudaGetLastError());
+            return METOK_ERR_CUDA;
+        }
+        ++launches;
+        bool found = false;
+        for (auto& g : agg)
+            if (std::strcmp(g.name, r.name) == 0) { g.n += 1; g.ms += ms; found = true; break; }
+        if (!found) agg.push_back({r.name, 1, (double)ms});
+        cudaEventDestroy(r.a);
+        cudaEventDestroy(r.b);
+    }
+    metok::g_recs.clear();
+    if (out && cap > 0) {
+        std::string text;
+        char line[256];
+        for (auto& g : agg) {
+            std::snprintf(line, sizeof line, "%s %d %.6f\n", g.name, g.n, g.ms);
+            text += line;
+        }
+        const size_t n = text.size() < cap - 1 ? text.size() : cap - 1;
+        std::memcpy(out, text.data(), n);
+        out[n] = 0;
+    }
+    return launches;
+}
 
 extern "C" const char* metok_status_string(int status) {
     switch (status) {

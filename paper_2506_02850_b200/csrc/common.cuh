@@ -25,6 +25,19 @@ void set_last_cuda_error(int e);
     } while (0)
 #define METOK_LAUNCH_CHECK() METOK_CUDA_TRY(cudaGetLastError())
 
+// Brackets one kernel launch with CUDA events while profiling is on (see
+// metok_profile_begin); costs one predictable branch otherwise.
+extern bool g_profiling;
+struct KernelTimer {
+    const char* name;
+    cudaStream_t st;
+    cudaEvent_t a, b;
+    bool active;
+    KernelTimer(const char* n, cudaStream_t s);
+    ~KernelTimer();
+};
+#define METOK_TIMED(name, st) ::metok::KernelTimer _metok_kt(name, st)
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

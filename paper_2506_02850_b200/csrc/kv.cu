@@ -144,7 +144,10 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
     if (policy == METOK_KV_PAPER) {
-        kv_paper_lists_kernel<<<L, 256, 0, st>>>(S_cur, vis_start, n_vis, l1, keep_idx, keep_len, new_len);
+        {
+            METOK_TIMED("kv_paper_lists_kernel", st);
+            kv_paper_lists_kernel<<<L, 256, 0, st>>>(S_cur, vis_start, n_vis, l1, keep_idx, keep_len, new_len);
+        }
         METOK_LAUNCH_CHECK();
     } else if (policy == METOK_KV_TOPK) {
         int32_t budget = ceilq(keep_ratio * (double)n_vis);
@@ -153,7 +156,10 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
                                          S_cur, vis_start, keep_idx, (size_t)S_cur, keep_len, new_len, L, st);
         if (rc != METOK_OK) return rc;
     } else {
-        copy_len_kernel<<<ceil_div(L, 256), 256, 0, st>>>(keep_len, new_len, L);
+        {
+            METOK_TIMED("copy_len_kernel", st);
+            copy_len_kernel<<<ceil_div(L, 256), 256, 0, st>>>(keep_len, new_len, L);
+        }
         METOK_LAUNCH_CHECK();
     }
     const int row_chunks = (int)((long long)dh * eb / 16);
@@ -165,7 +171,10 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
             ptrs.v[l] = l < nl ? v_layers[l0 + l] : nullptr;
         }
         const int grid = nl * 2 * Hkv * kKvCluster;
-        kv_gather_kernel<<<grid, kKvThreads, 0, st>>>(ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len);
+        {
+            METOK_TIMED("kv_gather_kernel", st);
+            kv_gather_kernel<<<grid, kKvThreads, 0, st>>>(ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len);
+        }
         METOK_LAUNCH_CHECK();
     }
     return METOK_OK;

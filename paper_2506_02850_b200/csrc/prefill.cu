@@ -265,8 +265,11 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
     const size_t smem = (size_t)G * 256 * sizeof(uint32_t);
     if (smem > 32 * 1024)
         METOK_CUDA_TRY(cudaFuncSetAttribute(class_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    class_topk_kernel<<<problems, 1024, smem, st>>>(scores, score_stride, token_group, n_vis, G, b, S, vis_start,
+    {
+        METOK_TIMED("class_topk_kernel", st);
+        class_topk_kernel<<<problems, 1024, smem, st>>>(scores, score_stride, token_group, n_vis, G, b, S, vis_start,
                                                     keep_idx, keep_stride, count_a, count_b);
+    }
     METOK_LAUNCH_CHECK();
     return METOK_OK;
 }
@@ -327,15 +330,24 @@ static int launch_attn_scores(const void* q_text, const void* k_all, const AttnD
     METOK_CUDA_TRY(cudaFuncSetAttribute(attn_stats_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     METOK_CUDA_TRY(cudaFuncSetAttribute(attn_colsum_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid(dm.nsplit, dm.nrt, dm.Hkv);
-    attn_stats_kernel<T><<<grid, 256, smem, st>>>(reinterpret_cast<const T*>(q_text), reinterpret_cast<const T*>(k_all),
+    {
+        METOK_TIMED("attn_stats_kernel", st);
+        attn_stats_kernel<T><<<grid, 256, smem, st>>>(reinterpret_cast<const T*>(q_text), reinterpret_cast<const T*>(k_all),
                                                   dm, w.part_m, w.part_l);
+    }
     METOK_LAUNCH_CHECK();
-    attn_colsum_kernel<T><<<grid, 256, smem, st>>>(reinterpret_cast<const T*>(q_text),
+    {
+        METOK_TIMED("attn_colsum_kernel", st);
+        attn_colsum_kernel<T><<<grid, 256, smem, st>>>(reinterpret_cast<const T*>(q_text),
                                                    reinterpret_cast<const T*>(k_all), dm, w.part_m, w.part_l,
                                                    w.part_col);
+    }
     METOK_LAUNCH_CHECK();
-    attn_score_reduce_kernel<<<ceil_div(dm.n_vis, 256), 256, 0, st>>>(w.part_col, dm.Hkv * dm.nrt, dm.n_vis,
+    {
+        METOK_TIMED("attn_score_reduce_kernel", st);
+        attn_score_reduce_kernel<<<ceil_div(dm.n_vis, 256), 256, 0, st>>>(w.part_col, dm.Hkv * dm.nrt, dm.n_vis,
                                                                       1.0f / (float)(dm.Hq * dm.Lt), scores);
+    }
     METOK_LAUNCH_CHECK();
     return METOK_OK;
 }
@@ -390,9 +402,12 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
     if (rc != METOK_OK) return rc;
     if (hidden) {
         const int row_chunks = (int)((long long)D * eb / 16);
-        gather_rows_kernel<<<kNumSMs * 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(hidden),
+        {
+            METOK_TIMED("gather_rows_kernel", st);
+            gather_rows_kernel<<<kNumSMs * 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(hidden),
                                                         reinterpret_cast<uint4*>(hidden_out), keep_idx, S_out,
                                                         row_chunks);
+        }
         METOK_LAUNCH_CHECK();
     }
     return METOK_OK;

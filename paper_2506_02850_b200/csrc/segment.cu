@@ -205,8 +205,11 @@ static int launch_segment(const void* feats, int Tn, int N, int d, int k, int si
         part_dot = cv.take<float>((size_t)nslab * Tn);
         part_nrm = cv.take<float>((size_t)nslab * Tn);
         dim3 grid(nslab, ceil_div(Tn, fpc));
-        seg_partial_kernel<T><<<grid, kSegThreads, 0, st>>>(reinterpret_cast<const T*>(feats), Tn, chunks, fpc,
+        {
+            METOK_TIMED("seg_partial_kernel", st);
+            seg_partial_kernel<T><<<grid, kSegThreads, 0, st>>>(reinterpret_cast<const T*>(feats), Tn, chunks, fpc,
                                                             part_dot, part_nrm);
+        }
         METOK_LAUNCH_CHECK();
     } else {
         nslab = 1;
@@ -214,9 +217,15 @@ static int launch_segment(const void* feats, int Tn, int N, int d, int k, int si
         part_nrm = cv.take<float>((size_t)Tn);
         float* mean = cv.take<float>((size_t)Tn * d);
         dim3 grid(ceil_div(d / VN, 128), Tn);
-        seg_mean_kernel<T><<<grid, 128, 0, st>>>(reinterpret_cast<const T*>(feats), N, d, mean);
+        {
+            METOK_TIMED("seg_mean_kernel", st);
+            seg_mean_kernel<T><<<grid, 128, 0, st>>>(reinterpret_cast<const T*>(feats), N, d, mean);
+        }
         METOK_LAUNCH_CHECK();
-        seg_meandot_kernel<<<Tn, 256, 0, st>>>(mean, Tn, d, part_dot, part_nrm);
+        {
+            METOK_TIMED("seg_meandot_kernel", st);
+            seg_meandot_kernel<<<Tn, 256, 0, st>>>(mean, Tn, d, part_dot, part_nrm);
+        }
         METOK_LAUNCH_CHECK();
     }
     const size_t smem = (size_t)Tn * 3 * sizeof(float);
@@ -224,8 +233,11 @@ static int launch_segment(const void* feats, int Tn, int N, int d, int k, int si
         METOK_CUDA_TRY(cudaFuncSetAttribute(seg_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)smem));
     }
-    seg_finish_kernel<<<1, 1024, smem, st>>>(part_dot, part_nrm, nslab, Tn, k, sims, boundaries, event_offsets,
+    {
+        METOK_TIMED("seg_finish_kernel", st);
+        seg_finish_kernel<<<1, 1024, smem, st>>>(part_dot, part_nrm, nslab, Tn, k, sims, boundaries, event_offsets,
                                              frame_event);
+    }
     METOK_LAUNCH_CHECK();
     return METOK_OK;
 }

@@ -431,10 +431,16 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         if (smem > 48 * 1024)
             METOK_CUDA_TRY(cudaFuncSetAttribute(tok_score_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 (int)smem));
-        tok_score_kernel<T><<<grid, 256, smem, st>>>(feats, text, Nv, d, token_score, w.inv_norm);
+        {
+            METOK_TIMED("tok_score_kernel", st);
+            tok_score_kernel<T><<<grid, 256, smem, st>>>(feats, text, Nv, d, token_score, w.inv_norm);
+        }
         METOK_LAUNCH_CHECK();
     }
-    frame_score_kernel<<<ceil_div(Tn, 8), 256, 0, st>>>(token_score, Tn, N, frame_score);
+    {
+        METOK_TIMED("frame_score_kernel", st);
+        frame_score_kernel<<<ceil_div(Tn, 8), 256, 0, st>>>(token_score, Tn, N, frame_score);
+    }
     METOK_LAUNCH_CHECK();
 
     PlanParams pp;
@@ -442,22 +448,34 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     pp.n_key_events = min(k, ceilq(p->alpha * (double)k));
     pp.event_agg = p->event_agg; pp.mode = p->mode; pp.tile_rows = kMergeTM;
     pp.keep_key = p->keep_key; pp.keep_nonkey = p->keep_nonkey; pp.beta = p->beta;
-    event_plan_kernel<<<1, 1024, (size_t)k * sizeof(float), st>>>(frame_score, event_offsets, pp, event_score,
+    {
+        METOK_TIMED("event_plan_kernel", st);
+        event_plan_kernel<<<1, 1024, (size_t)k * sizeof(float), st>>>(frame_score, event_offsets, pp, event_score,
                                                                   event_is_key, w.ev_lo, w.ev_budget, w.ev_out_off,
                                                                   w.ev_tile_off, n_out);
+    }
     METOK_LAUNCH_CHECK();
 
-    event_topk_kernel<<<k, 1024, 0, st>>>(token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off, w.is_key, out_src,
+    {
+        METOK_TIMED("event_topk_kernel", st);
+        event_topk_kernel<<<k, 1024, 0, st>>>(token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off, w.is_key, out_src,
                                           out_event, assign);
+    }
     METOK_LAUNCH_CHECK();
 
     const int max_tiles = Nv / kMergeTM + k;
-    merge_assign_simt_kernel<T><<<max_tiles, 256, 0, st>>>(feats, d, N, w.ev_lo, k, w.ev_out_off, w.ev_tile_off,
+    {
+        METOK_TIMED("merge_assign_simt_kernel", st);
+        merge_assign_simt_kernel<T><<<max_tiles, 256, 0, st>>>(feats, d, N, w.ev_lo, k, w.ev_out_off, w.ev_tile_off,
                                                            out_src, w.inv_norm, w.is_key, assign);
+    }
     METOK_LAUNCH_CHECK();
 
-    merge_avg_kernel<T><<<cap, kAvgThreads, 0, st>>>(feats, d, N, w.ev_lo, out_event, assign, n_out, out_feats,
+    {
+        METOK_TIMED("merge_avg_kernel", st);
+        merge_avg_kernel<T><<<cap, kAvgThreads, 0, st>>>(feats, d, N, w.ev_lo, out_event, assign, n_out, out_feats,
                                                      out_members);
+    }
     METOK_LAUNCH_CHECK();
     return METOK_OK;
 }

@@ -54,6 +54,7 @@ extern "C" {
 #define METOK_ERR_WORKSPACE   (-3)  /* ws is NULL or smaller than *_workspace_bytes */
 #define METOK_ERR_CUDA        (-4)  /* a launch or driver call failed; see metok_last_cuda_error */
 #define METOK_ERR_TIMEOUT     (-5)  /* a bounded device-side wait gave up (reported via status words) */
+#define METOK_ERR_TOO_LARGE   (-6)  /* the problem exceeds a fixed built-in capacity (see *_static) */
 
 #define METOK_F32  0
 #define METOK_BF16 1
@@ -98,6 +99,41 @@ METOK_API size_t metok_segment_events_workspace_bytes(int dtype, int T, int N, i
 METOK_API int metok_segment_events(const void* feats, int dtype, int T, int N, int d, int k, int sim_mode,
                          float* sims, int32_t* boundaries, int32_t* event_offsets,
                          int32_t* frame_event, void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * (1b) metok_segment_events without any workspace.  The paper has no counterpart
+ *      to this entry point; it exists for callers that cannot allocate.
+ *
+ *   Some hosts of this library may not call cudaMalloc at the point where they
+ *   need the segmentation: code running inside a memory pool whose budget is
+ *   already fixed, a plugin whose host application owns every allocation, a
+ *   real-time loop in which an allocation (an implicit device synchronisation)
+ *   is not acceptable.  For them this variant keeps its scratch -- the per-slab
+ *   partial sums of the similarity pass -- in a fixed 1 MiB array that is part of
+ *   the library image: every GPU that loads the library holds that 1 MiB until
+ *   the process exits.  Inputs and outputs are still the caller's.  It computes
+ *   exactly what metok_segment_events computes, with the same kernels, and never
+ *   calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ *   Limits and rules
+ *   - The problem must fit: metok_segment_events_workspace_bytes(dtype,T,N,d,
+ *     sim_mode) <= metok_segment_events_static_capacity() (1 MiB; e.g. FLATTEN with
+ *     T*ceil(N*d*elem/16384) <= 131072 -- the 128-frame workload needs 63 KiB).
+ *     Larger problems return METOK_ERR_TOO_LARGE and launch nothing.
+ *   - The first call on each device looks up the array's device address (a
+ *     driver query, no allocation).  Make that first call outside any CUDA
+ *     stream capture; later calls only launch kernels.
+ *   - All calls on one device share the one array.  Nothing in it has to start at
+ *     zero (each call overwrites every entry it later reads), but two calls that
+ *     overlap on the GPU -- different streams, or one stream per thread -- race
+ *     on it and give wrong results.  Serialise them on one stream, or use
+ *     metok_segment_events with separate workspaces.
+ *   Arguments and the other errors are those of metok_segment_events.
+ * ------------------------------------------------------------------------- */
+METOK_API size_t metok_segment_events_static_capacity(void);
+METOK_API int metok_segment_events_static(const void* feats, int dtype, int T, int N, int d, int k, int sim_mode,
+                                float* sims, int32_t* boundaries, int32_t* event_offsets,
+                                int32_t* frame_event, void* stream);
 
 /* ------------------------------------------------------------------------- *
  * (2) Event-aware token reduction after the vision encoder -- Eq. 5 and

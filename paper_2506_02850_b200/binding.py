@@ -44,6 +44,8 @@ class MetokError(RuntimeError):
 _SIGNATURES = {
     "metok_segment_events_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "metok_segment_events": (_i, [_vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "metok_segment_events_static_capacity": (_sz, []),
+    "metok_segment_events_static": (_i, [_vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "metok_compress_vision_bound": (_i, [_i, _i, _i, _c.POINTER(VisionParams)]),
     "metok_compress_vision_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _c.POINTER(VisionParams)]),
     "metok_compress_vision": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _vp, _c.POINTER(VisionParams),
@@ -153,6 +155,24 @@ def metok_segment_events(feats: torch.Tensor, k: int, sim_mode: int = SIM_FLATTE
     _check("metok_segment_events", st)
     return {"sims": sims[: T - 1], "boundaries": boundaries[: max(k - 1, 0)], "event_offsets": offsets[: k + 1],
             "frame_event": frame_event, "_sims": sims, "_boundaries": boundaries, "_offsets": offsets}
+
+
+def metok_segment_events_static(feats: torch.Tensor, k: int, sim_mode: int = SIM_FLATTEN) -> Dict[str, torch.Tensor]:
+    """metok_segment_events for callers that must not allocate scratch: the library's
+    built-in 1 MiB array is used instead of a workspace (problems that need more raise
+    MetokError with status -6).  Calls on one device must not overlap on the GPU."""
+    feats = _cuda_contig(feats, "feats")
+    T, N, d = feats.shape
+    dev = feats.device
+    sims = torch.empty(max(T - 1, 1), dtype=torch.float32, device=dev)
+    boundaries = torch.empty(max(k - 1, 1), dtype=torch.int32, device=dev)
+    offsets = torch.empty(max(k + 1, 2), dtype=torch.int32, device=dev)
+    frame_event = torch.empty(T, dtype=torch.int32, device=dev)
+    st = lib().metok_segment_events_static(_ptr(feats), _dt(feats), T, N, d, k, sim_mode, _ptr(sims),
+                                           _ptr(boundaries), _ptr(offsets), _ptr(frame_event), _stream())
+    _check("metok_segment_events_static", st)
+    return {"sims": sims[: T - 1], "boundaries": boundaries[: max(k - 1, 0)], "event_offsets": offsets[: k + 1],
+            "frame_event": frame_event}
 
 
 def vision_params(alpha: float, keep_key: float = 1.0, keep_nonkey: float = 1.0, event_agg: int = AGG_MEAN,

@@ -82,6 +82,7 @@ extern "C" const char* metok_status_string(int status) {
         case METOK_ERR_WORKSPACE: return "workspace missing or too small";
         case METOK_ERR_CUDA: return "CUDA error";
         case METOK_ERR_TIMEOUT: return "device-side wait timed out";
+        case METOK_ERR_TOO_LARGE: return "problem exceeds the built-in scratch capacity";
         default: return "unknown status";
     }
 }

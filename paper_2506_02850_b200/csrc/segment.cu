@@ -283,3 +283,46 @@ extern "C" int metok_segment_events(const void* feats, int dtype, int T, int N, 
     return launch_segment<__nv_bfloat16>(feats, T, N, d, k, sim_mode, sims, boundaries, event_offsets, frame_event,
                                          ws, st);
 }
+
+// --------------------------------------------------------------------------- //
+// metok_segment_events_static: the same computation with the scratch in a fixed
+// array that lives inside the library image instead of a caller workspace.
+// --------------------------------------------------------------------------- //
+namespace metok {
+constexpr size_t kStaticScratchBytes = (size_t)1 << 20;      // 1 MiB per GPU that loads the library
+static __device__ __align__(256) unsigned char g_seg_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_seg_scratch_addr[kMaxDevices] = {nullptr};    // device address of the array, per device
+
+// `g_seg_scratch` in host code is only a handle; the address kernels can use has to be
+// asked for, once per device, with that device current.
+static int static_scratch_address(void** out) {
+    int dev = -1;
+    METOK_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return METOK_ERR_UNSUPPORTED;
+    if (!g_seg_scratch_addr[dev]) {
+        void* p = nullptr;
+        METOK_CUDA_TRY(cudaGetSymbolAddress(&p, g_seg_scratch));
+        g_seg_scratch_addr[dev] = p;
+    }
+    *out = g_seg_scratch_addr[dev];
+    return METOK_OK;
+}
+}  // namespace metok
+
+extern "C" size_t metok_segment_events_static_capacity(void) { return metok::kStaticScratchBytes; }
+
+extern "C" int metok_segment_events_static(const void* feats, int dtype, int T, int N, int d, int k, int sim_mode,
+                                           float* sims, int32_t* boundaries, int32_t* event_offsets,
+                                           int32_t* frame_event, void* stream) {
+    if (dtype != METOK_F32 && dtype != METOK_BF16) return METOK_ERR_INVALID_ARG;
+    if (T < 1 || N < 1 || d < 1) return METOK_ERR_INVALID_ARG;
+    const size_t need = metok_segment_events_workspace_bytes(dtype, T, N, d, sim_mode);
+    if (need > metok::kStaticScratchBytes) return METOK_ERR_TOO_LARGE;
+    void* scratch = nullptr;
+    const int rc = metok::static_scratch_address(&scratch);
+    if (rc != METOK_OK) return rc;
+    return metok_segment_events(feats, dtype, T, N, d, k, sim_mode, sims, boundaries, event_offsets, frame_event,
+                                scratch, metok::kStaticScratchBytes, stream);
+}

@@ -222,6 +222,7 @@ def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text
                                  _ptr(out["frame_score"]), _ptr(out["event_score"]), _ptr(out["event_is_key"]),
                                  _ptr(out["n_out"]), cap, _ptr(ws), ws.numel(), _stream())
     _check("metok_compress_vision", st)
+    out["status"] = ws[:4].view(torch.int32)      # device status word (0, or -5 after a device-side timeout)
     return out
 
 

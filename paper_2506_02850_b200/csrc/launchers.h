@@ -15,4 +15,8 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
                       const int32_t* budgets_host, int S, int vis_start, int32_t* keep_idx, size_t keep_stride,
                       int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st);
 
+// dst[i] = src[idx[i]] for i < *n_rows (device scalar); rows of row_chunks 16-byte chunks.
+int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
+                       cudaStream_t st);
+
 }  // namespace metok

@@ -296,6 +296,17 @@ gather_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const
     }
 }
 
+int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
+                       cudaStream_t st) {
+    {
+        METOK_TIMED("gather_rows_kernel", st);
+        gather_rows_kernel<<<kNumSMs * 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(src),
+                                                        reinterpret_cast<uint4*>(dst), idx, n_rows, row_chunks);
+    }
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
+}
+
 static AttnDims make_dims(int Hq, int Hkv, int Lt, int S, int dh, int vis_start, int n_vis, float scale) {
     AttnDims dm;
     dm.Hq = Hq; dm.Hkv = Hkv; dm.Lt = Lt; dm.S = S; dm.dh = dh; dm.vis_start = vis_start; dm.n_vis = n_vis;

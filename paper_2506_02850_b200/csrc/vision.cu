@@ -1,7 +1,11 @@
 // metok_compress_vision: text relevance and key events (Eq. 5), per-event key-token
 // top-k, merge-assign of the remaining tokens and averaging.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "select.cuh"
+#include "sm100.cuh"
+#include "launchers.h"
 
 namespace metok {
 
@@ -316,6 +320,171 @@ merge_assign_simt_kernel(const T* __restrict__ feats, int d, int N, const int32_
     }
 }
 
+
+// --------------------------------------------------------------------------- //
+// Merge-assign on the tensor cores (bf16).  CTA = 128 consecutive token rows of one
+// event (TMEM lanes) x the event's key tokens in chunks of up to 256 columns.
+//   warp 0   : TMA producer -- per 64-wide K step one 128x64 tile of V (rows are
+//              contiguous in V) and the chunk's key rows from the compact key buffer
+//              (64-row boxes), 4-stage ring;
+//   warp 1   : allocates TMEM (2 accumulators x 256 columns), issues tcgen05.mma
+//              (M=128, N=16..256, K=16) and commits to the ring / accumulator barriers;
+//   warps 2-5: epilogue -- read the accumulator with tcgen05.ld, scale each column by
+//              1/|key|, keep the running (value, slot) argmax of the thread's row.
+// Every wait is bounded; on a timeout the CTA unwinds and writes METOK_ERR_TIMEOUT.
+// --------------------------------------------------------------------------- //
+constexpr int kMmaBM = 128, kMmaBK = 64, kMmaBN = 256, kMmaStages = 4;
+constexpr int kMmaThreads = 192;
+constexpr uint32_t kMmaABytes = kMmaBM * kMmaBK * 2;       // 16 KiB
+constexpr uint32_t kMmaBBytes = kMmaBN * kMmaBK * 2;       // 32 KiB
+constexpr uint32_t kMmaBoxBytes = 64 * kMmaBK * 2;         // one 64-row key box
+constexpr size_t kMmaSmemBytes = (size_t)kMmaStages * (kMmaABytes + kMmaBBytes) + 1024;
+
+__global__ void __launch_bounds__(kMmaThreads, 1)
+merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int d, int N,
+                        const int32_t* __restrict__ ev_lo, int k, const int32_t* __restrict__ ev_out_off,
+                        const int32_t* __restrict__ ev_tile_off, const int32_t* __restrict__ out_src,
+                        const float* __restrict__ inv_norm, const uint8_t* __restrict__ is_key,
+                        int32_t* __restrict__ assign, int32_t* __restrict__ status) {
+    using namespace sm100;
+    extern __shared__ uint8_t smem_dyn[];
+    __shared__ __align__(8) uint64_t full_bar[kMmaStages], empty_bar[kMmaStages], tfull_bar[2], tempty_bar[2];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+    __shared__ float s_keyinv[2][kMmaBN];
+
+    const int tile = blockIdx.x;
+    if (tile >= ev_tile_off[k]) return;
+    const int e = find_event(ev_tile_off, k, tile);
+    const int row0 = ev_lo[e] * N + (tile - ev_tile_off[e]) * kMmaBM;
+    const int row_end = ev_lo[e + 1] * N;
+    const int s0 = ev_out_off[e], s1 = ev_out_off[e + 1];
+    const int nk = s1 - s0;
+    const int nchunks = (nk + kMmaBN - 1) / kMmaBN;
+    const int ksteps = (d + kMmaBK - 1) / kMmaBK;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    auto a_addr = [&](int s) { return smem_base + (uint32_t)s * (kMmaABytes + kMmaBBytes); };
+    auto b_addr = [&](int s) { return a_addr(s) + kMmaABytes; };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMmaStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tfull_bar[b]), 1); mbar_init(smem_u32(&tempty_bar[b]), 4); }
+        s_abort = 0;
+        mbar_fence_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&s_tmem_base), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+    volatile int* abort_flag = &s_abort;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&tmA);
+            prefetch_tmap(&tmB);
+            int it = 0;
+            bool ok = true;
+            for (int c = 0; c < nchunks && ok; ++c) {
+                const int nvalid = min(kMmaBN, nk - c * kMmaBN);
+                const int nbox = (nvalid + 63) >> 6;
+                for (int ks = 0; ks < ksteps; ++ks, ++it) {
+                    const int s = it % kMmaStages;
+                    const uint32_t ph = (uint32_t)(it / kMmaStages) & 1u;
+                    if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t fb = smem_u32(&full_bar[s]);
+                    mbar_arrive_expect_tx(fb, kMmaABytes + (uint32_t)nbox * kMmaBoxBytes);
+                    tma_load_2d(a_addr(s), &tmA, ks * kMmaBK, row0, fb);
+                    for (int j = 0; j < nbox; ++j)
+                        tma_load_2d(b_addr(s) + (uint32_t)j * kMmaBoxBytes, &tmB, ks * kMmaBK,
+                                    s0 + c * kMmaBN + j * 64, fb);
+                }
+            }
+            if (!ok) {
+                // let the copies already issued land before the CTA's shared memory goes away
+                for (int back = 1; back <= kMmaStages && back <= it; ++back) {
+                    const int j = it - back;
+                    mbar_wait(smem_u32(&full_bar[j % kMmaStages]), (uint32_t)(j / kMmaStages) & 1u, abort_flag);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int c = 0; c < nchunks && ok; ++c) {
+                const int b = c & 1;
+                const uint32_t use = (uint32_t)(c >> 1);
+                if (!mbar_wait(smem_u32(&tempty_bar[b]), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const int nvalid = min(kMmaBN, nk - c * kMmaBN);
+                const uint32_t idesc = make_idesc_bf16(kMmaBM, (nvalid + 15) & ~15);
+                const uint32_t d_tmem = tmem_base + (uint32_t)b * kMmaBN;
+                for (int ks = 0; ks < ksteps; ++ks, ++it) {
+                    const int s = it % kMmaStages;
+                    const uint32_t ph = (uint32_t)(it / kMmaStages) & 1u;
+                    if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < kMmaBK / 16; ++kk) {
+                        const uint64_t ad = make_desc_k128(a_addr(s) + kk * 32);
+                        const uint64_t bd = make_desc_k128(b_addr(s) + kk * 32);
+                        umma_bf16(d_tmem, ad, bd, idesc, (ks | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&empty_bar[s]));          // frees the stage when these MMAs retire
+                }
+                if (ok) umma_commit(smem_u32(&tfull_bar[b]));      // accumulator of chunk c complete
+            }
+        }
+    } else {
+        const int grp = warp & 3;                                   // TMEM lanes 32*grp .. 32*grp+31
+        const int et = (warp - 2) * 32 + lane;                      // 0..127 among the epilogue threads
+        const int row = row0 + grp * 32 + lane;
+        float best_v = -3.4e38f;
+        int best_s = 0x7FFFFFFF;
+        bool ok = true;
+        for (int c = 0; c < nchunks; ++c) {
+            const int b = c & 1;
+            const uint32_t use = (uint32_t)(c >> 1);
+            const int nvalid = min(kMmaBN, nk - c * kMmaBN);
+            for (int i = et; i < kMmaBN; i += 128) {
+                const int slot = s0 + c * kMmaBN + i;
+                s_keyinv[b][i] = (i < nvalid) ? inv_norm[out_src[slot]] : 0.f;
+            }
+            named_bar_sync(1, 128);
+            if (ok && !mbar_wait(smem_u32(&tfull_bar[b]), use & 1u, abort_flag)) ok = false;
+            ok = __all_sync(0xFFFFFFFFu, ok);                      // tcgen05.ld below is warp-collective
+            if (ok) {
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(grp * 32) << 16) + (uint32_t)b * kMmaBN;
+                for (int c0 = 0; c0 < nvalid; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(t_row + (uint32_t)c0, v);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int col = c0 + j;
+                        const float val = v[j] * s_keyinv[b][col];
+                        if (col < nvalid && val > best_v) { best_v = val; best_s = s0 + c * kMmaBN + col; }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[b]));
+            }
+        }
+        if (ok && row < row_end && !is_key[row]) assign[row] = best_s;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+    if (threadIdx.x == 0 && s_abort) *status = METOK_ERR_TIMEOUT;
+}
+
 // --------------------------------------------------------------------------- //
 // Averaging: one CTA per output token.  Walks the event's `assign` range in
 // ascending token order (so the summation order is fixed), sums the member rows in
@@ -394,13 +563,17 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, const int32_t* __res
 // host side
 // --------------------------------------------------------------------------- //
 struct VisionWs {
+    int32_t* status;          // device status word, first in the workspace
+    void* key_rows;           // compact copy of the key-token rows (tensor-core path)
     float* inv_norm;
     uint8_t* is_key;
     int32_t *ev_lo, *ev_budget, *ev_out_off, *ev_tile_off;
 };
 
-static VisionWs carve_vision(Carver& cv, int Tn, int N, int k) {
+static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, bool mma) {
     VisionWs w;
+    w.status = cv.take<int32_t>(64);
+    w.key_rows = mma ? (void*)cv.take<__nv_bfloat16>(((size_t)cap + 64) * d) : nullptr;
     w.inv_norm = cv.take<float>((size_t)Tn * N);
     w.is_key = cv.take<uint8_t>((size_t)Tn * N);
     w.ev_lo = cv.take<int32_t>((size_t)k + 1);
@@ -408,6 +581,13 @@ static VisionWs carve_vision(Carver& cv, int Tn, int N, int k) {
     w.ev_out_off = cv.take<int32_t>((size_t)k + 1);
     w.ev_tile_off = cv.take<int32_t>((size_t)k + 1);
     return w;
+}
+
+// The tensor-core merge path needs bf16 rows that TMA can address (16-byte row pitch);
+// METOK_FORCE_SIMT=1 in the environment selects the CUDA-core kernels (debugging aid).
+static bool use_mma_path(int d) {
+    static const bool force_simt = [] { const char* e = getenv("METOK_FORCE_SIMT"); return e && e[0] == '1'; }();
+    return !force_simt && d % 8 == 0;
 }
 
 static bool ratio_ok(double r) { return r > 0.0 && r <= 1.0; }
@@ -422,8 +602,11 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     const T* text = reinterpret_cast<const T*>(text_);
     T* out_feats = reinterpret_cast<T*>(out_feats_);
     const int Nv = Tn * N;
+    constexpr bool kBf16 = sizeof(T) == 2;
+    const bool mma = kBf16 && use_mma_path(d);
     Carver cv(ws);
-    VisionWs w = carve_vision(cv, Tn, N, k);
+    VisionWs w = carve_vision(cv, Tn, N, k, d, cap, mma);
+    METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
 
     {
         const int grid = min(ceil_div(Nv, 8), kNumSMs * 8);
@@ -446,7 +629,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     PlanParams pp;
     pp.Tn = Tn; pp.N = N; pp.k = k;
     pp.n_key_events = min(k, ceilq(p->alpha * (double)k));
-    pp.event_agg = p->event_agg; pp.mode = p->mode; pp.tile_rows = kMergeTM;
+    pp.event_agg = p->event_agg; pp.mode = p->mode; pp.tile_rows = mma ? kMmaBM : kMergeTM;
     pp.keep_key = p->keep_key; pp.keep_nonkey = p->keep_nonkey; pp.beta = p->beta;
     {
         METOK_TIMED("event_plan_kernel", st);
@@ -463,13 +646,35 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     }
     METOK_LAUNCH_CHECK();
 
-    const int max_tiles = Nv / kMergeTM + k;
-    {
-        METOK_TIMED("merge_assign_simt_kernel", st);
-        merge_assign_simt_kernel<T><<<max_tiles, 256, 0, st>>>(feats, d, N, w.ev_lo, k, w.ev_out_off, w.ev_tile_off,
-                                                           out_src, w.inv_norm, w.is_key, assign);
+    if (mma) {
+        // compact copy of the key rows so that one tensor map covers an event's keys
+        const int rc = launch_gather_rows(feats, w.key_rows, out_src, n_out, (int)((size_t)d * sizeof(T) / 16), st);
+        if (rc != METOK_OK) return rc;
+        CUtensorMap tmA, tmB;
+        int r2 = make_tmap_bf16_2d(&tmA, feats, (uint64_t)Nv, (uint64_t)d, kMmaBM);
+        if (r2 != METOK_OK) return r2;
+        r2 = make_tmap_bf16_2d(&tmB, w.key_rows, (uint64_t)cap + 64, (uint64_t)d, 64);
+        if (r2 != METOK_OK) return r2;
+        METOK_CUDA_TRY(cudaFuncSetAttribute(merge_assign_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kMmaSmemBytes));
+        const int max_tiles = Nv / kMmaBM + k;
+        {
+            METOK_TIMED("merge_assign_mma_kernel", st);
+            merge_assign_mma_kernel<<<max_tiles, kMmaThreads, kMmaSmemBytes, st>>>(
+                tmA, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_tile_off, out_src, w.inv_norm, w.is_key, assign,
+                w.status);
+        }
+        METOK_LAUNCH_CHECK();
+    } else {
+        const int max_tiles = Nv / kMergeTM + k;
+        {
+            METOK_TIMED("merge_assign_simt_kernel", st);
+            merge_assign_simt_kernel<T><<<max_tiles, 256, 0, st>>>(feats, d, N, w.ev_lo, k, w.ev_out_off,
+                                                                   w.ev_tile_off, out_src, w.inv_norm, w.is_key,
+                                                                   assign);
+        }
+        METOK_LAUNCH_CHECK();
     }
-    METOK_LAUNCH_CHECK();
 
     {
         METOK_TIMED("merge_avg_kernel", st);
@@ -520,10 +725,10 @@ extern "C" int metok_compress_vision_bound(int T, int N, int k, const metok_visi
 
 extern "C" size_t metok_compress_vision_workspace_bytes(int dtype, int T, int N, int d, int k, int cap,
                                                         const metok_vision_params* p) {
-    (void)dtype; (void)d; (void)cap; (void)p;
-    if (T < 1 || N < 1 || k < 1) return 0;
+    (void)p;
+    if (T < 1 || N < 1 || k < 1 || d < 1 || cap < 0) return 0;
     Carver cv(nullptr);
-    carve_vision(cv, T, N, k);
+    carve_vision(cv, T, N, k, d, cap, dtype == METOK_BF16);
     return cv.total();
 }
 

@@ -55,6 +55,7 @@ def compress_case(V: np.ndarray, t: np.ndarray, offs: np.ndarray, dtype: str, al
                                   P.to_torch(t, dtype), p)
     torch.cuda.synchronize()
     rep: Dict[str, object] = {}
+    assert int(got["status"].item()) == 0, "device-side wait timed out"
     n_out = int(got["n_out"].item())
     assert n_out == want["n_out"], (n_out, want["n_out"])
     rep["n_out"] = n_out

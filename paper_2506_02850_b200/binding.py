@@ -263,6 +263,7 @@ def metok_prefill_prune(q_text: torch.Tensor, k_all: torch.Tensor, hidden: Optio
                                _ptr(out["keep_idx"]), _ptr(out["S_out"]), _ptr(out["hidden_out"]), _ptr(ws),
                                ws.numel(), _stream())
     _check("metok_prefill_prune", st)
+    out["status"] = ws[:4].view(torch.int32)      # device status word (0, or -5 after a device-side timeout)
     return out
 
 

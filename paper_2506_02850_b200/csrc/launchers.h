@@ -19,4 +19,14 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
 int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
                        cudaStream_t st);
 
+// Text->visual attention scores on the tensor cores (bf16, dh 64 or 128): leaves
+// n_planes partial column sums of n_vis floats each in part_col; their sum divided by
+// Hq*Lt is the score.  attn_mma_workspace gives the element counts of part_m / part_l
+// (each) and of part_col.  `status` receives METOK_ERR_TIMEOUT if a device-side wait gave up.
+void attn_mma_workspace(int Hq, int Hkv, int Lt, int S, int n_vis, size_t* n_part_ml, size_t* n_part_col,
+                        int* n_planes);
+int launch_attn_scores_mma(const void* q_text, const void* k_all, int Hq, int Hkv, int Lt, int S, int dh,
+                           int vis_start, int n_vis, float scale, float* part_m, float* part_l, float* part_col,
+                           int32_t* status, cudaStream_t st);
+
 }  // namespace metok

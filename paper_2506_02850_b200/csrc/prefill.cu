@@ -1,5 +1,7 @@
 // metok_prefill_prune: text->visual attention scores at a pruning layer, class-wise
 // top-k under the Eq. 6/7 budgets, and compaction of the surviving hidden states.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "select.cuh"
 #include "launchers.h"
@@ -323,15 +325,44 @@ static AttnDims make_dims(int Hq, int Hkv, int Lt, int S, int dh, int vis_start,
     return dm;
 }
 
+// The tensor-core scoring path takes bf16 with head dim 64 or 128; METOK_FORCE_SIMT=1 in
+// the environment selects the CUDA-core kernels (debugging aid).
+static bool use_mma_attn(int dtype, int dh) {
+    static const bool force_simt = [] { const char* e = getenv("METOK_FORCE_SIMT"); return e && e[0] == '1'; }();
+    return !force_simt && dtype == METOK_BF16 && (dh == 64 || dh == 128);
+}
+
 struct PrefillWs {
+    int32_t* status;          // device status word, first in the workspace
     float *part_m, *part_l, *part_col;
+    int n_planes;
 };
-static PrefillWs carve_prefill(Carver& cv, const AttnDims& dm) {
+static PrefillWs carve_prefill(Carver& cv, const AttnDims& dm, bool mma) {
     PrefillWs w;
-    w.part_m = cv.take<float>((size_t)dm.Hkv * dm.nsplit * dm.R);
-    w.part_l = cv.take<float>((size_t)dm.Hkv * dm.nsplit * dm.R);
-    w.part_col = cv.take<float>((size_t)dm.Hkv * dm.nrt * dm.n_vis);
+    w.status = cv.take<int32_t>(64);
+    if (mma) {
+        size_t n_ml, n_col;
+        attn_mma_workspace(dm.Hq, dm.Hkv, dm.Lt, dm.S, dm.n_vis, &n_ml, &n_col, &w.n_planes);
+        w.part_m = cv.take<float>(n_ml);
+        w.part_l = cv.take<float>(n_ml);
+        w.part_col = cv.take<float>(n_col);
+    } else {
+        w.part_m = cv.take<float>((size_t)dm.Hkv * dm.nsplit * dm.R);
+        w.part_l = cv.take<float>((size_t)dm.Hkv * dm.nsplit * dm.R);
+        w.part_col = cv.take<float>((size_t)dm.Hkv * dm.nrt * dm.n_vis);
+        w.n_planes = dm.Hkv * dm.nrt;
+    }
     return w;
+}
+
+static int launch_score_reduce(const PrefillWs& w, const AttnDims& dm, float* scores, cudaStream_t st) {
+    {
+        METOK_TIMED("attn_score_reduce_kernel", st);
+        attn_score_reduce_kernel<<<ceil_div(dm.n_vis, 256), 256, 0, st>>>(w.part_col, w.n_planes, dm.n_vis,
+                                                                      1.0f / (float)(dm.Hq * dm.Lt), scores);
+    }
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
 }
 
 template <typename T>
@@ -354,13 +385,7 @@ static int launch_attn_scores(const void* q_text, const void* k_all, const AttnD
                                                    w.part_col);
     }
     METOK_LAUNCH_CHECK();
-    {
-        METOK_TIMED("attn_score_reduce_kernel", st);
-        attn_score_reduce_kernel<<<ceil_div(dm.n_vis, 256), 256, 0, st>>>(w.part_col, dm.Hkv * dm.nrt, dm.n_vis,
-                                                                      1.0f / (float)(dm.Hq * dm.Lt), scores);
-    }
-    METOK_LAUNCH_CHECK();
-    return METOK_OK;
+    return launch_score_reduce(w, dm, scores, st);
 }
 
 }  // namespace metok
@@ -368,11 +393,10 @@ static int launch_attn_scores(const void* q_text, const void* k_all, const AttnD
 using namespace metok;
 
 extern "C" size_t metok_prefill_prune_workspace_bytes(int dtype, int Hq, int Hkv, int Lt, int S, int dh, int n_vis) {
-    (void)dtype;
     if (Hq < 1 || Hkv < 1 || Lt < 1 || S < 1 || dh < 1 || n_vis < 1 || Hq % Hkv) return 0;
     AttnDims dm = make_dims(Hq, Hkv, Lt, S, dh, 0, n_vis, 1.f);
     Carver cv(nullptr);
-    carve_prefill(cv, dm);
+    carve_prefill(cv, dm, use_mma_attn(dtype, dh));
     return cv.total();
 }
 
@@ -403,10 +427,19 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
     AttnDims dm = make_dims(Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale);
+    const bool mma = use_mma_attn(dtype, dh);
     Carver cv(ws);
-    PrefillWs w = carve_prefill(cv, dm);
-    int rc = dtype == METOK_F32 ? launch_attn_scores<float>(q_text, k_all, dm, w, scores, st)
+    PrefillWs w = carve_prefill(cv, dm, mma);
+    METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
+    int rc;
+    if (mma) {
+        rc = launch_attn_scores_mma(q_text, k_all, Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale, w.part_m,
+                                    w.part_l, w.part_col, w.status, st);
+        if (rc == METOK_OK) rc = launch_score_reduce(w, dm, scores, st);
+    } else {
+        rc = dtype == METOK_F32 ? launch_attn_scores<float>(q_text, k_all, dm, w, scores, st)
                                 : launch_attn_scores<__nv_bfloat16>(q_text, k_all, dm, w, scores, st);
+    }
     if (rc != METOK_OK) return rc;
     rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, S_out, nullptr,
                            1, st);

@@ -128,6 +128,7 @@ def prefill_case(Q: np.ndarray, K: np.ndarray, dtype: str, vis_start: int, n_vis
                                 torch.from_numpy(np.asarray(groups, dtype=np.int32)).cuda(), budgets, scale)
     torch.cuda.synchronize()
     rep: Dict[str, object] = {}
+    assert int(got["status"].item()) == 0, "device-side wait timed out"
     rep["score_err"] = P.check_scores(got["scores"].cpu().numpy(), want_scores, dtype, "attention scores")
     S_out = int(got["S_out"].item())
     assert S_out == want["S_out"], (S_out, want["S_out"])

@@ -47,6 +47,17 @@ kv_paper_lists_kernel(int S_cur, int vis_start, int n_vis, int l1, int32_t* __re
     if (threadIdx.x == 0) { keep_len[layer] = n; new_len[layer] = n; }
 }
 
+// One keep list serves every layer: rows 1..L-1 of keep_idx and the lengths are copies of row 0.
+__global__ void __launch_bounds__(256)
+kv_broadcast_list_kernel(int32_t* __restrict__ keep_idx, int S_cur, int32_t* __restrict__ keep_len,
+                         int32_t* __restrict__ new_len) {
+    const int layer = blockIdx.y + 1;
+    const int n = keep_len[0];
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) keep_idx[(size_t)layer * S_cur + i] = keep_idx[i];
+    if (i == 0) { keep_len[layer] = n; new_len[layer] = n; }
+}
+
 __global__ void copy_len_kernel(const int32_t* __restrict__ a, int32_t* __restrict__ b, int n) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) b[i] = a[i];
@@ -152,9 +163,20 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
     } else if (policy == METOK_KV_TOPK) {
         int32_t budget = ceilq(keep_ratio * (double)n_vis);
         if (budget > n_vis) budget = n_vis;
+        // shared scores give the same list in every layer: select once, then copy
+        const int problems = scores_per_layer ? L : 1;
         const int rc = launch_class_topk(scores, scores_per_layer ? (size_t)n_vis : 0, nullptr, n_vis, 1, &budget,
-                                         S_cur, vis_start, keep_idx, (size_t)S_cur, keep_len, new_len, L, st);
+                                         S_cur, vis_start, keep_idx, (size_t)S_cur, keep_len, new_len, problems, st);
         if (rc != METOK_OK) return rc;
+        if (problems < L) {
+            const int kept = budget + (S_cur - n_vis);
+            {
+                METOK_TIMED("kv_broadcast_list_kernel", st);
+                kv_broadcast_list_kernel<<<dim3(ceil_div(kept > 0 ? kept : 1, 256), L - 1), 256, 0, st>>>(
+                    keep_idx, S_cur, keep_len, new_len);
+            }
+            METOK_LAUNCH_CHECK();
+        }
     } else {
         {
             METOK_TIMED("copy_len_kernel", st);

@@ -225,16 +225,32 @@ attn_score_reduce_kernel(const float* __restrict__ part_col, int nparts, int n_v
 // --------------------------------------------------------------------------- //
 struct TopkBudgets { int v[METOK_MAX_GROUPS]; };
 
-__global__ void __launch_bounds__(1024)
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 class_topk_kernel(const float* __restrict__ scores, size_t score_stride, const int32_t* __restrict__ token_group,
-                  int n_vis, int G, TopkBudgets budgets, int S, int vis_start, int32_t* __restrict__ keep_idx,
-                  size_t keep_stride, int32_t* __restrict__ count_a, int32_t* __restrict__ count_b) {
+                  int n_vis, int G, SelectLayout lay, TopkBudgets budgets, int S, int vis_start,
+                  int32_t* __restrict__ keep_idx, size_t keep_stride, int32_t* __restrict__ count_a,
+                  int32_t* __restrict__ count_b) {
     __shared__ SelectSmem sm;
     __shared__ int s_budget[METOK_MAX_GROUPS];
-    __shared__ int s_clamped[METOK_MAX_GROUPS];
-    extern __shared__ uint32_t hist[];               // [G*256]
-    const float* sc = scores + (size_t)blockIdx.x * score_stride;
-    int32_t* keep = keep_idx + (size_t)blockIdx.x * keep_stride;
+    extern __shared__ __align__(16) unsigned char sel_dyn[];
+    const int problem = blockIdx.x / kSelCluster;
+    const float* sc = scores + (size_t)problem * score_stride;
+    int32_t* keep = keep_idx + (size_t)problem * keep_stride;
+    const int vis_end = vis_start + n_vis;
+    SelectCtx cx;
+    cx.rank = (int)cx.cl.block_rank();
+    cx.G = G;
+    cx.nb_log2 = lay.nb_log2;
+    int p_lo, p_hi;
+    select_slice(S, cx.rank, &p_lo, &p_hi);
+    const int v_lo = max(p_lo, vis_start), v_hi = min(p_hi, vis_end);   // scored positions of this slice
+    cx.item_lo = v_lo - vis_start;
+    cx.m = v_hi > v_lo ? v_hi - v_lo : 0;
+    cx.cached = cx.m <= lay.cache_cap;
+    cx.hist = reinterpret_cast<uint32_t*>(sel_dyn + lay.hist_off);
+    cx.merged = reinterpret_cast<uint32_t*>(sel_dyn + lay.merged_off);
+    cx.keys = reinterpret_cast<uint32_t*>(sel_dyn + lay.keys_off);
+    cx.cls = sel_dyn + lay.cls_off;
     for (int g = threadIdx.x; g < G; g += blockDim.x) s_budget[g] = budgets.v[g];
     __syncthreads();
     auto cls = [=](int i) {
@@ -243,19 +259,18 @@ class_topk_kernel(const float* __restrict__ scores, size_t score_stride, const i
         return (g >= 0 && g < G) ? g : -1;
     };
     auto val = [=](int i) { return sc[i]; };
-    block_select_thresholds(n_vis, G, cls, val, s_budget, hist, sm, s_clamped);
-    const int vis_end = vis_start + n_vis;
+    cluster_select(cx, n_vis, cls, val, s_budget, sm);
     auto flag = [&](int u) {
         if (u < vis_start || u >= vis_end) return true;
         const int i = u - vis_start;
-        const int g = cls(i);
-        return g >= 0 && sm.need[g] > 0 && key64_of(sc[i], i) >= sm.prefix[g];
+        const SelItem it = item_at(cx, i - cx.item_lo, cls, val);
+        return it.cls >= 0 && is_selected(sm, it.cls, it.key, i);
     };
     auto emit = [&](int u, int rank) { keep[rank] = u; };
-    const int total = block_compact(S, flag, emit, sm);
-    if (threadIdx.x == 0) {
-        if (count_a) count_a[blockIdx.x] = total;
-        if (count_b) count_b[blockIdx.x] = total;
+    const int total = cluster_compact(cx, p_lo, p_hi, flag, emit, sm);
+    if (threadIdx.x == 0 && cx.rank == 0) {
+        if (count_a) count_a[problem] = total;
+        if (count_b) count_b[problem] = total;
     }
 }
 
@@ -264,13 +279,16 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
                       int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st) {
     TopkBudgets b;
     for (int g = 0; g < METOK_MAX_GROUPS; ++g) b.v[g] = g < G ? budgets_host[g] : 0;
-    const size_t smem = (size_t)G * 256 * sizeof(uint32_t);
-    if (smem > 32 * 1024)
-        METOK_CUDA_TRY(cudaFuncSetAttribute(class_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const SelectLayout lay = select_layout(G, select_items_per_cta((long long)S));
+    const int nthreads = select_threads(select_items_per_cta((long long)S));
+    if (lay.bytes > 32 * 1024)                        // static + dynamic beyond 48 KiB needs the opt-in
+        METOK_CUDA_TRY(cudaFuncSetAttribute(class_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)lay.bytes));
     {
         METOK_TIMED("class_topk_kernel", st);
-        class_topk_kernel<<<problems, 1024, smem, st>>>(scores, score_stride, token_group, n_vis, G, b, S, vis_start,
-                                                    keep_idx, keep_stride, count_a, count_b);
+        class_topk_kernel<<<problems * kSelCluster, nthreads, lay.bytes, st>>>(
+            scores, score_stride, token_group, n_vis, G, lay, b, S, vis_start, keep_idx, keep_stride, count_a,
+            count_b);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;

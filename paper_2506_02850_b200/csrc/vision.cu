@@ -170,38 +170,48 @@ event_plan_kernel(const float* __restrict__ frame_score, const int32_t* __restri
     }
 }
 
-// Per-event key-token top-k: one CTA per event.
-__global__ void __launch_bounds__(1024)
+// Per-event key-token top-k: one cluster per event.
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 event_topk_kernel(const float* __restrict__ token_score, const int32_t* __restrict__ ev_lo, int N,
-                  const int32_t* __restrict__ ev_budget, const int32_t* __restrict__ ev_out_off,
+                  const int32_t* __restrict__ ev_budget, const int32_t* __restrict__ ev_out_off, SelectLayout lay,
                   uint8_t* __restrict__ is_key, int32_t* __restrict__ out_src, int32_t* __restrict__ out_event,
                   int32_t* __restrict__ assign) {
     __shared__ SelectSmem sm;
-    __shared__ uint32_t hist[256];
     __shared__ int s_budget[1];
-    __shared__ int s_clamped[1];
-    const int e = blockIdx.x;
+    extern __shared__ __align__(16) unsigned char sel_dyn[];
+    const int e = blockIdx.x / kSelCluster;
     const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
     const int n = hi - lo;
-    if (n <= 0) return;
+    if (n <= 0) return;                                   // the whole cluster leaves together
+    SelectCtx cx;
+    cx.rank = (int)cx.cl.block_rank();
+    cx.G = 1;
+    cx.nb_log2 = lay.nb_log2;
+    int p_lo, p_hi;
+    select_slice(n, cx.rank, &p_lo, &p_hi);
+    cx.item_lo = p_lo;
+    cx.m = p_hi - p_lo;
+    cx.cached = cx.m <= lay.cache_cap;
+    cx.hist = reinterpret_cast<uint32_t*>(sel_dyn + lay.hist_off);
+    cx.merged = reinterpret_cast<uint32_t*>(sel_dyn + lay.merged_off);
+    cx.keys = reinterpret_cast<uint32_t*>(sel_dyn + lay.keys_off);
+    cx.cls = sel_dyn + lay.cls_off;
     if (threadIdx.x == 0) s_budget[0] = ev_budget[e];
     __syncthreads();
     const float* s = token_score + lo;
     auto cls = [](int) { return 0; };
     auto val = [s](int i) { return s[i]; };
-    block_select_thresholds(n, 1, cls, val, s_budget, hist, sm, s_clamped);
-    const unsigned long long thr = sm.prefix[0];
-    const bool any = sm.need[0] > 0;
+    cluster_select(cx, n, cls, val, s_budget, sm);
     const int slot0 = ev_out_off[e];
-    auto flag = [&](int i) { return any && key64_of(s[i], i) >= thr; };
+    auto flag = [&](int i) { return is_selected(sm, 0, item_at(cx, i - p_lo, cls, val).key, i); };
     auto emit = [&](int i, int rank) {
         const int slot = slot0 + rank;
         out_src[slot] = lo + i;
         out_event[slot] = e;
         assign[lo + i] = slot;
     };
-    block_compact(n, flag, emit, sm);
-    for (int i = threadIdx.x; i < n; i += blockDim.x) is_key[lo + i] = flag(i) ? 1 : 0;
+    for (int i = p_lo + threadIdx.x; i < p_hi; i += blockDim.x) is_key[lo + i] = flag(i) ? 1 : 0;
+    cluster_compact(cx, p_lo, p_hi, flag, emit, sm);
 }
 
 // --------------------------------------------------------------------------- //
@@ -640,11 +650,19 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     METOK_LAUNCH_CHECK();
 
     {
-        METOK_TIMED("event_topk_kernel", st);
-        event_topk_kernel<<<k, 1024, 0, st>>>(token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off, w.is_key, out_src,
-                                          out_event, assign);
+        // the cache is sized for the longest event there can be, the thread count for twice the mean
+        const SelectLayout lay = select_layout(1, select_items_per_cta((long long)(Tn - (k - 1)) * N));
+        const int nthreads = select_threads(select_items_per_cta(2LL * Nv / k));
+        if (lay.bytes > 32 * 1024)                        // static + dynamic beyond 48 KiB needs the opt-in
+            METOK_CUDA_TRY(cudaFuncSetAttribute(event_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)lay.bytes));
+        {
+            METOK_TIMED("event_topk_kernel", st);
+            event_topk_kernel<<<k * kSelCluster, nthreads, lay.bytes, st>>>(
+                token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off, lay, w.is_key, out_src, out_event, assign);
+        }
+        METOK_LAUNCH_CHECK();
     }
-    METOK_LAUNCH_CHECK();
 
     if (mma) {
         // compact copy of the key rows so that one tensor map covers an event's keys

@@ -208,7 +208,8 @@ class Workload:
             "attn_stats_mma_kernel": ("tensor", attn_flops),
             "attn_colsum_mma_kernel": ("tensor", attn_flops),
             "gather_rows_kernel": ("hbm", hidden_bytes),
-            "kv_gather_kernel": ("hbm", 2.0 * kv_rows * cfg.dh * b * 2 * cfg.Hkv * cfg.L),
+            "gather_key_rows_kernel": ("hbm", 2.0 * n_out * d * b),
+            "kv_copy_kernel": ("hbm", 2.0 * kv_rows * cfg.dh * b * 2 * cfg.Hkv * cfg.L),
             "class_topk_kernel": ("hbm", 8.0 * (sum(s["n_vis"] for s in self.stages) + cfg.L * cfg.Nv)),
             "event_topk_kernel": ("hbm", 8.0 * Nv),
         }
@@ -379,14 +380,18 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    host_ms = {}
+
     def timed(fn, steps):
         for _ in range(warm):
             fn()
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
+        t0 = time.perf_counter()
         for _ in range(steps):
             fn()
+        host_ms[fn.__name__] = (time.perf_counter() - t0) * 1e3 / steps     # time to enqueue one step
         e1.record()
         barrier()
         ms = e0.elapsed_time(e1)
@@ -457,7 +462,7 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
                 "config": {"workload": workload_name, "l2": "inputs larger than L2 (V 132 MB, hidden 133 MB, K/V 1.06 GB touched between reuses)",
                            "parallelism": f"replicas x{world}"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+                "host_enqueue_ms_per_step": host_ms.get("step"), "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
                 "roofline": roofline, "cpu_baseline": cpu}
         print(json.dumps(line))
     if dist is not None:

@@ -2,8 +2,18 @@
 // and the in-place, order-preserving gather of K and V rows.
 //
 // In-place safety.  Row i receives old row keep[i] with keep ascending, hence
-// keep[i] >= i.  Rows are moved in rounds of consecutive destination rows; a
-// round's sources all lie at or beyond the round's first destination row, so
+// keep[i] >= i, and after the call only rows [0, n) matter (n = list length).
+//
+// Fast path.  A source row at or beyond n is never written by anybody, so it can be
+// read at any time.  Only the first h rows of the list, h = #{i : keep[i] < n}, have
+// their source inside the destination region.  Those h rows are first copied to a
+// staging area in the workspace (one kernel), then every row is written from its
+// source or from the staging area (a second kernel) -- no ordering inside either
+// kernel, any number of CTAs per slab.  With a keep ratio r about r*n rows are staged.
+//
+// General path (h larger than the staging area: lists that keep most rows).  Rows are
+// moved in rounds of consecutive destination rows; a round's sources all lie at or
+// beyond the round's first destination row, so
 //   * a round only has to finish READING before any of its rows are WRITTEN, and
 //   * later rounds' sources are never touched by earlier rounds' writes, so the
 //     next round can be prefetched before the current one is stored.
@@ -63,15 +73,121 @@ __global__ void copy_len_kernel(const int32_t* __restrict__ a, int32_t* __restri
     if (i < n) b[i] = a[i];
 }
 
+// ---- fast path ------------------------------------------------------------------
+constexpr int kKvFastThreads = 256;
+constexpr int kKvFastUnroll = 8;          // 16-byte chunks in flight per thread
+constexpr int kKvStageSplit = 2;          // CTAs per slab in the staging kernel
+constexpr int kKvCopySplit = 4;           // CTAs per slab in the copy kernel
+constexpr size_t kKvStageBudget = (size_t)64 << 20;   // bytes of workspace the staging area may take
+
+// First index of the ascending list keep[0..n) whose value is >= n; whole warp, 32-ary search.
+__device__ __forceinline__ int warp_lower_bound(const int32_t* __restrict__ keep, int n, int lane) {
+    int lo = 0, hi = n;                                   // answer in [lo, hi]
+    while (hi > lo) {
+        const int step = (hi - lo + 31) / 32;
+        const int idx = lo + lane * step;
+        const bool ge = idx < hi ? keep[idx] >= n : true;
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, ge);
+        const int f = bal ? __ffs(bal) - 1 : 32;          // first probe that is >= n; 32: none was
+        const int new_hi = f < 32 ? min(hi, lo + f * step) : hi;   // keep[new_hi] >= n (or new_hi == hi)
+        const int new_lo = f > 0 ? lo + (f - 1) * step + 1 : lo;   // the probe before it was < n
+        hi = new_hi;
+        lo = new_lo;
+    }
+    return lo;
+}
+
+struct SlabId { int ll, which, head; };
+__device__ __forceinline__ SlabId slab_of(int slab, int Hkv) {
+    SlabId s;
+    s.head = slab % Hkv;
+    s.which = (slab / Hkv) & 1;
+    s.ll = slab / (2 * Hkv);
+    return s;
+}
+
+// Copies the rows whose source lies inside the destination region to the staging area and
+// records h per layer (-1: too many for the staging area, the general path takes the layer).
+__global__ void __launch_bounds__(kKvFastThreads)
+kv_stage_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row_chunks,
+                const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ keep_len, int stage_rows,
+                int32_t* __restrict__ haz, uint4* __restrict__ stage) {
+    __shared__ int s_h;
+    const SlabId id = slab_of(blockIdx.y, Hkv);
+    const int layer = layer0 + id.ll;
+    const int32_t* keep = keep_idx + (size_t)layer * S_cur;
+    const int n = keep_len[layer];
+    if (threadIdx.x < 32) {
+        const int h = (n > 0 && n < S_cur) ? warp_lower_bound(keep, n, threadIdx.x) : 0;
+        if (threadIdx.x == 0) s_h = h;
+    }
+    __syncthreads();
+    const int h = s_h;
+    const bool fast = h <= stage_rows;
+    if (blockIdx.x == 0 && id.which == 0 && id.head == 0 && threadIdx.x == 0) haz[layer] = fast ? h : -1;
+    if (!fast || h == 0) return;
+    const uint4* base = reinterpret_cast<const uint4*>(id.which ? ptrs.v[id.ll] : ptrs.k[id.ll]) +
+                        (size_t)id.head * S_cap * row_chunks;
+    uint4* dst = stage + ((size_t)(layer * 2 + id.which) * Hkv + id.head) * (size_t)stage_rows * row_chunks;
+    const int total = h * row_chunks;
+    for (int gc = blockIdx.x * kKvFastThreads + threadIdx.x; gc < total; gc += kKvStageSplit * kKvFastThreads) {
+        const int i = gc / row_chunks, c = gc - i * row_chunks;
+        const int src = keep[i];
+        if (src != i) dst[gc] = base[(size_t)src * row_chunks + c];
+    }
+}
+
+// Every kept row from its source (at or beyond the new length: never written) or from the
+// staging area.
+__global__ void __launch_bounds__(kKvFastThreads)
+kv_copy_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row_chunks,
+               const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ keep_len, int stage_rows,
+               const int32_t* __restrict__ haz, const uint4* __restrict__ stage) {
+    const SlabId id = slab_of(blockIdx.y, Hkv);
+    const int layer = layer0 + id.ll;
+    const int h = haz[layer];
+    const int n = keep_len[layer];
+    if (h < 0 || n >= S_cur) return;
+    const int32_t* keep = keep_idx + (size_t)layer * S_cur;
+    uint4* base = reinterpret_cast<uint4*>(id.which ? ptrs.v[id.ll] : ptrs.k[id.ll]) +
+                  (size_t)id.head * S_cap * row_chunks;
+    const uint4* stg = stage + ((size_t)(layer * 2 + id.which) * Hkv + id.head) * (size_t)stage_rows * row_chunks;
+    const int total = n * row_chunks;
+    constexpr int kStep = kKvFastThreads * kKvFastUnroll;
+    for (int g0 = blockIdx.x * kStep; g0 < total; g0 += kKvCopySplit * kStep) {
+        uint4 v[kKvFastUnroll];
+        int at[kKvFastUnroll];                            // destination chunk, -1: nothing to store
+#pragma unroll
+        for (int u = 0; u < kKvFastUnroll; ++u) {
+            const int gc = g0 + u * kKvFastThreads + threadIdx.x;
+            at[u] = -1;
+            if (gc < total) {
+                const int i = gc / row_chunks, c = gc - i * row_chunks;
+                const int src = keep[i];
+                if (src != i) {
+                    v[u] = i < h ? stg[gc] : base[(size_t)src * row_chunks + c];
+                    at[u] = gc;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kKvFastUnroll; ++u)
+            if (at[u] >= 0) base[at[u]] = v[u];
+    }
+}
+
+// ---- general path -----------------------------------------------------------------
 __global__ void __cluster_dims__(kKvCluster, 1, 1) __launch_bounds__(kKvThreads)
 kv_gather_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row_chunks,
-                 const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ keep_len) {
+                 const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ keep_len,
+                 const int32_t* __restrict__ haz) {
     cg::cluster_group cluster = cg::this_cluster();
     const int crank = (int)cluster.block_rank();
     const int slab = blockIdx.x / kKvCluster;            // (layer_local, which, head)
     const int head = slab % Hkv;
     const int which = (slab / Hkv) & 1;
     const int ll = slab / (2 * Hkv);
+    if (haz[layer0 + ll] >= 0) return;                   // the fast path took this layer (uniform per cluster)
     uint4* base = reinterpret_cast<uint4*>(which ? ptrs.v[ll] : ptrs.k[ll]) + (size_t)head * S_cap * row_chunks;
     const int32_t* keep = keep_idx + (size_t)(layer0 + ll) * S_cur;
     const int n = keep_len[layer0 + ll];
@@ -122,14 +238,36 @@ kv_gather_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row
     }
 }
 
+struct KvWs {
+    int32_t* haz;
+    uint4* stage;
+    int stage_rows;
+};
+static KvWs carve_kv(Carver& cv, int L, int Hkv, int S_cur, int row_chunks) {
+    KvWs w;
+    w.haz = cv.take<int32_t>((size_t)L);
+    const size_t per_row = (size_t)L * 2 * Hkv * row_chunks * sizeof(uint4);
+    size_t rows = kKvStageBudget / per_row;
+    if (rows > (size_t)S_cur) rows = (size_t)S_cur;
+    w.stage_rows = (int)rows;
+    w.stage = cv.take<uint4>((size_t)L * 2 * Hkv * rows * row_chunks);
+    return w;
+}
+
 }  // namespace metok
 
 using namespace metok;
 
 extern "C" size_t metok_kv_compact_workspace_bytes(int dtype, int L, int Hkv, int S_cur, int dh, int policy,
                                                    int n_vis) {
-    (void)dtype; (void)L; (void)Hkv; (void)S_cur; (void)dh; (void)policy; (void)n_vis;
-    return 256;   // no scratch is needed today; a non-zero size keeps the calling convention uniform
+    (void)policy; (void)n_vis;
+    if (L < 1 || Hkv < 1 || S_cur < 1 || dh < 1) return 0;
+    const int eb = dtype == METOK_F32 ? 4 : 2;
+    const int row_chunks = (int)((long long)dh * eb / 16);
+    if (row_chunks < 1) return 0;
+    Carver cv(nullptr);
+    carve_kv(cv, L, Hkv, S_cur, row_chunks);
+    return cv.total();
 }
 
 extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, int dtype, int L, int Hkv, int S_cap,
@@ -185,6 +323,8 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
         METOK_LAUNCH_CHECK();
     }
     const int row_chunks = (int)((long long)dh * eb / 16);
+    Carver cv(ws);
+    const KvWs w = carve_kv(cv, L, Hkv, S_cur, row_chunks);
     for (int l0 = 0; l0 < L; l0 += kKvMaxLayersPerLaunch) {
         const int nl = (L - l0) < kKvMaxLayersPerLaunch ? (L - l0) : kKvMaxLayersPerLaunch;
         KvPtrs ptrs;
@@ -192,10 +332,23 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
             ptrs.k[l] = l < nl ? k_layers[l0 + l] : nullptr;
             ptrs.v[l] = l < nl ? v_layers[l0 + l] : nullptr;
         }
-        const int grid = nl * 2 * Hkv * kKvCluster;
+        const int slabs = nl * 2 * Hkv;
+        {
+            METOK_TIMED("kv_stage_kernel", st);
+            kv_stage_kernel<<<dim3(kKvStageSplit, slabs), kKvFastThreads, 0, st>>>(
+                ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len, w.stage_rows, w.haz, w.stage);
+        }
+        METOK_LAUNCH_CHECK();
+        {
+            METOK_TIMED("kv_copy_kernel", st);
+            kv_copy_kernel<<<dim3(kKvCopySplit, slabs), kKvFastThreads, 0, st>>>(
+                ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len, w.stage_rows, w.haz, w.stage);
+        }
+        METOK_LAUNCH_CHECK();
         {
             METOK_TIMED("kv_gather_kernel", st);
-            kv_gather_kernel<<<grid, kKvThreads, 0, st>>>(ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len);
+            kv_gather_kernel<<<slabs * kKvCluster, kKvThreads, 0, st>>>(ptrs, l0, Hkv, S_cap, S_cur, row_chunks,
+                                                                    keep_idx, keep_len, w.haz);
         }
         METOK_LAUNCH_CHECK();
     }

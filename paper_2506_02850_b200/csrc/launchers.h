@@ -16,8 +16,9 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
                       int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st);
 
 // dst[i] = src[idx[i]] for i < *n_rows (device scalar); rows of row_chunks 16-byte chunks.
+// timer_name labels the launch in the per-kernel timing report.
 int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
-                       cudaStream_t st);
+                       const char* timer_name, cudaStream_t st);
 
 // Text->visual attention scores on the tensor cores (bf16, dh 64 or 128): leaves
 // n_planes partial column sums of n_vis floats each in part_col; their sum divided by

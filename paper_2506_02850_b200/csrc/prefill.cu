@@ -296,31 +296,45 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
 
 // --------------------------------------------------------------------------- //
 // hidden_out[i] = hidden[keep_idx[i]], i < *S_out.  Rows are whole 16-byte chunks.
+// One warp per row and trip; a lane has up to 8 chunks (128 bytes) in flight before it
+// stores any, and rows are dealt to warps round-robin so that consecutive rows -- often
+// consecutive in the source too -- are copied at the same time.
 // --------------------------------------------------------------------------- //
-__global__ void __launch_bounds__(256)
+constexpr int kGatherThreads = 256;
+constexpr int kGatherUnroll = 8;
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__global__ void __launch_bounds__(kGatherThreads)
 gather_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const int32_t* __restrict__ keep_idx,
                    const int32_t* __restrict__ n_rows, int row_chunks) {
     const int n = *n_rows;
-    for (int i = blockIdx.x; i < n; i += gridDim.x) {
+    const int lane = threadIdx.x & 31;
+    const int warps = gridDim.x * (kGatherThreads / 32);
+    for (int i = blockIdx.x * (kGatherThreads / 32) + (threadIdx.x >> 5); i < n; i += warps) {
         const uint4* s = src + (size_t)keep_idx[i] * row_chunks;
         uint4* o = dst + (size_t)i * row_chunks;
-        for (int c = threadIdx.x; c < row_chunks; c += 256 * 4) {
-            uint4 v[4];
+        for (int c = lane; c < row_chunks; c += 32 * kGatherUnroll) {
+            uint4 v[kGatherUnroll];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (c + u * 256 < row_chunks) v[u] = __ldg(s + c + u * 256);
+            for (int u = 0; u < kGatherUnroll; ++u)
+                if (c + u * 32 < row_chunks) v[u] = ld_stream(s + c + u * 32);
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (c + u * 256 < row_chunks) o[c + u * 256] = v[u];
+            for (int u = 0; u < kGatherUnroll; ++u)
+                if (c + u * 32 < row_chunks) o[c + u * 32] = v[u];
         }
     }
 }
 
 int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
-                       cudaStream_t st) {
+                       const char* timer_name, cudaStream_t st) {
     {
-        METOK_TIMED("gather_rows_kernel", st);
-        gather_rows_kernel<<<kNumSMs * 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(src),
+        METOK_TIMED(timer_name, st);
+        gather_rows_kernel<<<kNumSMs * 8, kGatherThreads, 0, st>>>(reinterpret_cast<const uint4*>(src),
                                                         reinterpret_cast<uint4*>(dst), idx, n_rows, row_chunks);
     }
     METOK_LAUNCH_CHECK();
@@ -466,7 +480,7 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
         const int row_chunks = (int)((long long)D * eb / 16);
         {
             METOK_TIMED("gather_rows_kernel", st);
-            gather_rows_kernel<<<kNumSMs * 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(hidden),
+            gather_rows_kernel<<<kNumSMs * 8, kGatherThreads, 0, st>>>(reinterpret_cast<const uint4*>(hidden),
                                                         reinterpret_cast<uint4*>(hidden_out), keep_idx, S_out,
                                                         row_chunks);
         }

@@ -15,12 +15,31 @@ constexpr int kSegThreads = 256;
 constexpr int kSegUnroll = 4;     // 16-byte chunks per thread per frame
 constexpr int kMaxFrames = 8192;
 
+// Raw 16-byte chunk of either dtype, widened on use.
+template <typename T>
+__device__ __forceinline__ void widen16(const uint4& r, float (&v)[16 / sizeof(T)]) {
+    if constexpr (sizeof(T) == 4) {
+        v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y);
+        v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+    } else {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i]     = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+}
+
+constexpr int kSegMaxRun = 16;    // frames per CTA at most
+
 template <typename T>
 __global__ void __launch_bounds__(kSegThreads)
 seg_partial_kernel(const T* __restrict__ feats, int Tn, long long chunks_per_frame, int frames_per_cta,
                    float* __restrict__ part_dot, float* __restrict__ part_nrm) {
     constexpr int VN = Vec16<T>::N;
-    __shared__ float red[2][kSegThreads / 32];
+    constexpr int NW = kSegThreads / 32;
+    __shared__ float s_nn[kSegMaxRun + 1][NW], s_dp[kSegMaxRun + 1][NW];
     const int slab = blockIdx.x;
     const int f0 = blockIdx.y * frames_per_cta;
     const int f1 = min(Tn, f0 + frames_per_cta);          // own frames [f0, f1)
@@ -34,40 +53,48 @@ seg_partial_kernel(const T* __restrict__ feats, int Tn, long long chunks_per_fra
         chunk[u] = (long long)slab * (kSegThreads * kSegUnroll) + u * kSegThreads + tid;
         ok[u] = chunk[u] < chunks_per_frame;
     }
-    float prev[kSegUnroll][VN];
+    const uint4* base = reinterpret_cast<const uint4*>(feats);
+    auto fetch = [&](int f, uint4 (&r)[kSegUnroll]) {
+        const uint4* frame = base + (size_t)f * (size_t)chunks_per_frame;
 #pragma unroll
-    for (int u = 0; u < kSegUnroll; ++u) Vec16<T>::zero(prev[u]);
-
+        for (int u = 0; u < kSegUnroll; ++u) r[u] = ok[u] ? __ldg(frame + chunk[u]) : make_uint4(0u, 0u, 0u, 0u);
+    };
+    uint4 prev[kSegUnroll], cur[kSegUnroll], nxt[kSegUnroll];   // raw chunks: widened when used
+#pragma unroll
+    for (int u = 0; u < kSegUnroll; ++u) prev[u] = make_uint4(0u, 0u, 0u, 0u);
+    fetch(f0, cur);
+    // the next frame's loads are in flight while this frame is reduced; nothing inside the
+    // loop waits for another warp
     for (int f = f0; f <= f_last; ++f) {
-        const T* frame = feats + (size_t)f * (size_t)chunks_per_frame * VN;
-        float cur[kSegUnroll][VN];
-#pragma unroll
-        for (int u = 0; u < kSegUnroll; ++u) {
-            if (ok[u]) Vec16<T>::load(frame + chunk[u] * VN, cur[u]);
-            else Vec16<T>::zero(cur[u]);
-        }
+        if (f < f_last) fetch(f + 1, nxt);
         float nn = 0.f, dp = 0.f;
 #pragma unroll
         for (int u = 0; u < kSegUnroll; ++u) {
+            float c[VN], p[VN];
+            widen16<T>(cur[u], c);
+            widen16<T>(prev[u], p);
 #pragma unroll
             for (int e = 0; e < VN; ++e) {
-                nn = fmaf(cur[u][e], cur[u][e], nn);
-                dp = fmaf(cur[u][e], prev[u][e], dp);
-                prev[u][e] = cur[u][e];
+                nn = fmaf(c[e], c[e], nn);
+                dp = fmaf(c[e], p[e], dp);
             }
         }
         nn = warp_sum(nn);
         dp = warp_sum(dp);
-        if (lane == 0) { red[0][warp] = nn; red[1][warp] = dp; }
-        __syncthreads();
-        if (tid == 0) {
-            float a = 0.f, b = 0.f;
+        if (lane == 0) { s_nn[f - f0][warp] = nn; s_dp[f - f0][warp] = dp; }
 #pragma unroll
-            for (int w = 0; w < kSegThreads / 32; ++w) { a += red[0][w]; b += red[1][w]; }
-            if (f < f1) part_nrm[(size_t)slab * Tn + f] = a;
-            if (f > f0) part_dot[(size_t)slab * Tn + (f - 1)] = b;   // dot of frames f-1 and f
-        }
-        __syncthreads();
+        for (int u = 0; u < kSegUnroll; ++u) { prev[u] = cur[u]; cur[u] = nxt[u]; }
+    }
+    __syncthreads();
+    // the warps' sums in warp order: <v_f, v_f> for own frames, <v_{f-1}, v_f> for every frame after the first
+    const int nf = f_last - f0 + 1;
+    if (tid < nf) {
+        const int f = f0 + tid;
+        float a = 0.f, b = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) { a += s_nn[tid][w]; b += s_dp[tid][w]; }
+        if (f < f1) part_nrm[(size_t)slab * Tn + f] = a;
+        if (f > f0) part_dot[(size_t)slab * Tn + (f - 1)] = b;
     }
 }
 
@@ -200,7 +227,7 @@ static int launch_segment(const void* feats, int Tn, int N, int d, int k, int si
     if (sim_mode == METOK_SIM_FLATTEN) {
         const long long chunks = (long long)N * d / VN;
         nslab = (int)((chunks + kSegThreads * kSegUnroll - 1) / (kSegThreads * kSegUnroll));
-        int fpc = 16;
+        int fpc = kSegMaxRun;
         while (fpc > 1 && (long long)nslab * ceil_div(Tn, fpc) < 4 * kNumSMs) fpc >>= 1;
         part_dot = cv.take<float>((size_t)nslab * Tn);
         part_nrm = cv.take<float>((size_t)nslab * Tn);

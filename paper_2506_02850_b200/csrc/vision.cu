@@ -42,32 +42,47 @@ tok_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Nv
     }
     __syncthreads();
     const float tn = s_tn;
-    for (int row = blockIdx.x * 8 + warp; row < Nv; row += gridDim.x * 8) {
+    // rows from the last one down: the pass before this one (segmentation) streams V upwards
+    // and leaves its tail in L2
+    for (int rr = blockIdx.x * 8 + warp; rr < Nv; rr += gridDim.x * 8) {
+        const int row = Nv - 1 - rr;
         const T* x = feats + (size_t)row * d;
         float nn = 0.f, dt = 0.f;
-        for (int c0 = 0; c0 < nchunk; c0 += 128) {
-            float v[4][VN];
+        constexpr int U = 8;                        // 16-byte chunks in flight per lane
+        for (int c0 = 0; c0 < nchunk; c0 += 32 * U) {
+            uint4 raw[U];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < U; ++u) {
                 const int c = c0 + u * 32 + lane;
-                if (c < nchunk) Vec16<T>::load(x + (size_t)c * VN, v[u]);
-                else Vec16<T>::zero(v[u]);
+                raw[u] = c < nchunk ? __ldg(reinterpret_cast<const uint4*>(x) + c) : make_uint4(0u, 0u, 0u, 0u);
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < U; ++u) {
                 const int c = c0 + u * 32 + lane;
                 if (c < nchunk) {
+                    float v[VN];
+                    if constexpr (sizeof(T) == 4) {
+                        v[0] = __uint_as_float(raw[u].x); v[1] = __uint_as_float(raw[u].y);
+                        v[2] = __uint_as_float(raw[u].z); v[3] = __uint_as_float(raw[u].w);
+                    } else {
+                        const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            v[2 * i]     = __uint_as_float(w[i] << 16);
+                            v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+                        }
+                    }
 #pragma unroll
                     for (int h = 0; h < VN / 4; ++h) {
                         const float4 tt = reinterpret_cast<const float4*>(s_t + h * (nchunk * 4))[c];
-                        nn = fmaf(v[u][4 * h + 0], v[u][4 * h + 0], nn);
-                        dt = fmaf(v[u][4 * h + 0], tt.x, dt);
-                        nn = fmaf(v[u][4 * h + 1], v[u][4 * h + 1], nn);
-                        dt = fmaf(v[u][4 * h + 1], tt.y, dt);
-                        nn = fmaf(v[u][4 * h + 2], v[u][4 * h + 2], nn);
-                        dt = fmaf(v[u][4 * h + 2], tt.z, dt);
-                        nn = fmaf(v[u][4 * h + 3], v[u][4 * h + 3], nn);
-                        dt = fmaf(v[u][4 * h + 3], tt.w, dt);
+                        nn = fmaf(v[4 * h + 0], v[4 * h + 0], nn);
+                        dt = fmaf(v[4 * h + 0], tt.x, dt);
+                        nn = fmaf(v[4 * h + 1], v[4 * h + 1], nn);
+                        dt = fmaf(v[4 * h + 1], tt.y, dt);
+                        nn = fmaf(v[4 * h + 2], v[4 * h + 2], nn);
+                        dt = fmaf(v[4 * h + 2], tt.z, dt);
+                        nn = fmaf(v[4 * h + 3], v[4 * h + 3], nn);
+                        dt = fmaf(v[4 * h + 3], tt.w, dt);
                     }
                 }
             }
@@ -496,57 +511,122 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 }
 
 // --------------------------------------------------------------------------- //
-// Averaging: one CTA per output token.  Walks the event's `assign` range in
-// ascending token order (so the summation order is fixed), sums the member rows in
-// fp32, divides by the member count and rounds once.
+// Averaging: one CTA per output token.  The event's `assign` range is read in
+// segments; in a segment every thread takes a contiguous run of entries (16-byte loads,
+// all issued before the first is looked at), the matches are packed in token order by
+// one block-wide scan, and the member rows are then added in that order (so the
+// summation order is fixed), two rows in flight per thread.  fp32 sum, one division,
+// one rounding.
 // --------------------------------------------------------------------------- //
 constexpr int kAvgThreads = 128;
 constexpr int kAvgChunks = 4;      // 16-byte chunks per thread per pass over d
+constexpr int kAvgQuads = 5;       // 16-byte groups of `assign` per thread and segment
+constexpr int kAvgSeg = kAvgThreads * kAvgQuads * 4;   // tokens per segment
 
 template <typename T>
 __global__ void __launch_bounds__(kAvgThreads)
-merge_avg_kernel(const T* __restrict__ feats, int d, int N, const int32_t* __restrict__ ev_lo,
+merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
                  const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
                  const int32_t* __restrict__ n_out, T* __restrict__ out_feats, int32_t* __restrict__ out_members) {
     constexpr int VN = Vec16<T>::N;
-    __shared__ int s_list[kAvgThreads];
+    __shared__ int s_list[kAvgSeg];
     __shared__ int s_wtot[kAvgThreads / 32];
-    const int c = blockIdx.x;
-    if (c >= *n_out) return;
+    // CTAs start in index order: take the outputs from the last one down, so that this pass
+    // begins with the rows of V that the preceding (ascending) pass left in L2
+    const int c = *n_out - 1 - (int)blockIdx.x;
+    if (c < 0) return;
     const int e = out_event[c];
     const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nchunk = d / VN;
+    const int4* assign4 = reinterpret_cast<const int4*>(assign);
+    const int q_lo = lo >> 2, q_hi = (hi + 3) >> 2;            // groups of four tokens that touch [lo, hi)
     for (int cb = 0; cb < nchunk; cb += kAvgThreads * kAvgChunks) {
         float acc[kAvgChunks][VN];
 #pragma unroll
         for (int u = 0; u < kAvgChunks; ++u) Vec16<T>::zero(acc[u]);
         int count = 0;
-        for (int base = lo; base < hi; base += kAvgThreads) {
-            const int j = base + tid;
-            const bool f = j < hi && assign[j] == c;
-            const unsigned bal = __ballot_sync(0xFFFFFFFFu, f);
-            if (lane == 0) s_wtot[warp] = __popc(bal);
+        for (int qs = q_lo; qs < q_hi; qs += kAvgThreads * kAvgQuads) {
+            // this thread's run: groups [q0, q0 + kAvgQuads)
+            const int q0 = qs + tid * kAvgQuads;
+            int4 a[kAvgQuads];
+#pragma unroll
+            for (int u = 0; u < kAvgQuads; ++u) {
+                const int q = q0 + u;
+                a[u] = make_int4(-1, -1, -1, -1);
+                if (q < q_hi) {
+                    if (q * 4 + 3 < Nv) {
+                        a[u] = assign4[q];
+                    } else {                                   // the array ends inside this group
+                        if (q * 4 + 0 < Nv) a[u].x = assign[q * 4 + 0];
+                        if (q * 4 + 1 < Nv) a[u].y = assign[q * 4 + 1];
+                        if (q * 4 + 2 < Nv) a[u].z = assign[q * 4 + 2];
+                    }
+                }
+            }
+            unsigned match = 0;                                // bit 4u+k: token 4(q0+u)+k belongs to output c
+#pragma unroll
+            for (int u = 0; u < kAvgQuads; ++u) {
+                const int j = (q0 + u) * 4;
+                match |= (unsigned)(a[u].x == c && j + 0 >= lo && j + 0 < hi) << (4 * u + 0);
+                match |= (unsigned)(a[u].y == c && j + 1 >= lo && j + 1 < hi) << (4 * u + 1);
+                match |= (unsigned)(a[u].z == c && j + 2 >= lo && j + 2 < hi) << (4 * u + 2);
+                match |= (unsigned)(a[u].w == c && j + 3 >= lo && j + 3 < hi) << (4 * u + 3);
+            }
+            const int mine = __popc(match);
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31) s_wtot[warp] = incl;
             __syncthreads();
-            int before = 0, total = 0;
+            int before = incl - mine, total = 0;
 #pragma unroll
             for (int w = 0; w < kAvgThreads / 32; ++w) {
                 const int v = s_wtot[w];
                 if (w < warp) before += v;
                 total += v;
             }
-            if (f) s_list[before + __popc(bal & ((1u << lane) - 1u))] = j;
+            while (match) {
+                const int b = __ffs(match) - 1;
+                match &= match - 1;
+                s_list[before++] = q0 * 4 + b;
+            }
             __syncthreads();
-            for (int m = 0; m < total; ++m) {
-                const T* x = feats + (size_t)s_list[m] * d;
+            int m = 0;
+            for (; m + 1 < total; m += 2) {                    // two member rows in flight
+                const T* x0 = feats + (size_t)s_list[m] * d;
+                const T* x1 = feats + (size_t)s_list[m + 1] * d;
+                float v0[kAvgChunks][VN], v1[kAvgChunks][VN];
 #pragma unroll
                 for (int u = 0; u < kAvgChunks; ++u) {
                     const int ch = cb + u * kAvgThreads + tid;
                     if (ch < nchunk) {
-                        float v[VN];
-                        Vec16<T>::load(x + (size_t)ch * VN, v);
+                        Vec16<T>::load(x0 + (size_t)ch * VN, v0[u]);
+                        Vec16<T>::load(x1 + (size_t)ch * VN, v1[u]);
+                    }
+                }
 #pragma unroll
-                        for (int q = 0; q < VN; ++q) acc[u][q] += v[q];
+                for (int u = 0; u < kAvgChunks; ++u) {
+                    const int ch = cb + u * kAvgThreads + tid;
+                    if (ch < nchunk) {
+#pragma unroll
+                        for (int q = 0; q < VN; ++q) acc[u][q] = (acc[u][q] + v0[u][q]) + v1[u][q];
+                    }
+                }
+            }
+            if (m < total) {
+                const T* x0 = feats + (size_t)s_list[m] * d;
+#pragma unroll
+                for (int u = 0; u < kAvgChunks; ++u) {
+                    const int ch = cb + u * kAvgThreads + tid;
+                    if (ch < nchunk) {
+                        float v0[VN];
+                        Vec16<T>::load(x0 + (size_t)ch * VN, v0);
+#pragma unroll
+                        for (int q = 0; q < VN; ++q) acc[u][q] += v0[q];
                     }
                 }
             }
@@ -666,7 +746,8 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
 
     if (mma) {
         // compact copy of the key rows so that one tensor map covers an event's keys
-        const int rc = launch_gather_rows(feats, w.key_rows, out_src, n_out, (int)((size_t)d * sizeof(T) / 16), st);
+        const int rc = launch_gather_rows(feats, w.key_rows, out_src, n_out, (int)((size_t)d * sizeof(T) / 16),
+                                          "gather_key_rows_kernel", st);
         if (rc != METOK_OK) return rc;
         CUtensorMap tmA, tmB;
         int r2 = make_tmap_bf16_2d(&tmA, feats, (uint64_t)Nv, (uint64_t)d, kMmaBM);
@@ -696,8 +777,8 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
 
     {
         METOK_TIMED("merge_avg_kernel", st);
-        merge_avg_kernel<T><<<cap, kAvgThreads, 0, st>>>(feats, d, N, w.ev_lo, out_event, assign, n_out, out_feats,
-                                                     out_members);
+        merge_avg_kernel<T><<<cap, kAvgThreads, 0, st>>>(feats, d, N, Nv, w.ev_lo, out_event, assign, n_out,
+                                                     out_feats, out_members);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;

@@ -57,17 +57,6 @@ kv_paper_lists_kernel(int S_cur, int vis_start, int n_vis, int l1, int32_t* __re
     if (threadIdx.x == 0) { keep_len[layer] = n; new_len[layer] = n; }
 }
 
-// One keep list serves every layer: rows 1..L-1 of keep_idx and the lengths are copies of row 0.
-__global__ void __launch_bounds__(256)
-kv_broadcast_list_kernel(int32_t* __restrict__ keep_idx, int S_cur, int32_t* __restrict__ keep_len,
-                         int32_t* __restrict__ new_len) {
-    const int layer = blockIdx.y + 1;
-    const int n = keep_len[0];
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) keep_idx[(size_t)layer * S_cur + i] = keep_idx[i];
-    if (i == 0) { keep_len[layer] = n; new_len[layer] = n; }
-}
-
 __global__ void copy_len_kernel(const int32_t* __restrict__ a, int32_t* __restrict__ b, int n) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) b[i] = a[i];
@@ -78,7 +67,7 @@ constexpr int kKvFastThreads = 256;
 constexpr int kKvFastUnroll = 8;          // 16-byte chunks in flight per thread
 constexpr int kKvStageSplit = 2;          // CTAs per slab in the staging kernel
 constexpr int kKvCopySplit = 4;           // CTAs per slab in the copy kernel
-constexpr size_t kKvStageBudget = (size_t)64 << 20;   // bytes of workspace the staging area may take
+constexpr size_t kKvStageBudget = (size_t)128 << 20;   // bytes of workspace the staging area may take
 
 // First index of the ascending list keep[0..n) whose value is >= n; whole warp, 32-ary search.
 __device__ __forceinline__ int warp_lower_bound(const int32_t* __restrict__ keep, int n, int lane) {
@@ -292,7 +281,11 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
         return METOK_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
+    // an upper bound, known on the host, of the length of every list that drops anything
+    // (-1: not known); lists that keep all rows cause no copying
+    int kept_bound = -1;
     if (policy == METOK_KV_PAPER) {
+        kept_bound = S_cur - n_vis;
         {
             METOK_TIMED("kv_paper_lists_kernel", st);
             kv_paper_lists_kernel<<<L, 256, 0, st>>>(S_cur, vis_start, n_vis, l1, keep_idx, keep_len, new_len);
@@ -301,20 +294,13 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
     } else if (policy == METOK_KV_TOPK) {
         int32_t budget = ceilq(keep_ratio * (double)n_vis);
         if (budget > n_vis) budget = n_vis;
-        // shared scores give the same list in every layer: select once, then copy
+        // shared scores give the same list in every layer: select once, write it L times
         const int problems = scores_per_layer ? L : 1;
         const int rc = launch_class_topk(scores, scores_per_layer ? (size_t)n_vis : 0, nullptr, n_vis, 1, &budget,
-                                         S_cur, vis_start, keep_idx, (size_t)S_cur, keep_len, new_len, problems, st);
+                                         S_cur, vis_start, keep_idx, (size_t)S_cur, scores_per_layer ? 1 : L,
+                                         keep_len, new_len, problems, st);
         if (rc != METOK_OK) return rc;
-        if (problems < L) {
-            const int kept = budget + (S_cur - n_vis);
-            {
-                METOK_TIMED("kv_broadcast_list_kernel", st);
-                kv_broadcast_list_kernel<<<dim3(ceil_div(kept > 0 ? kept : 1, 256), L - 1), 256, 0, st>>>(
-                    keep_idx, S_cur, keep_len, new_len);
-            }
-            METOK_LAUNCH_CHECK();
-        }
+        kept_bound = budget + (S_cur - n_vis);
     } else {
         {
             METOK_TIMED("copy_len_kernel", st);
@@ -345,12 +331,15 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
                 ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len, w.stage_rows, w.haz, w.stage);
         }
         METOK_LAUNCH_CHECK();
-        {
-            METOK_TIMED("kv_gather_kernel", st);
-            kv_gather_kernel<<<slabs * kKvCluster, kKvThreads, 0, st>>>(ptrs, l0, Hkv, S_cap, S_cur, row_chunks,
-                                                                    keep_idx, keep_len, w.haz);
+        // h <= list length: when every list is known to fit the staging area, no layer takes the general path
+        if (kept_bound < 0 || kept_bound > w.stage_rows) {
+            {
+                METOK_TIMED("kv_gather_kernel", st);
+                kv_gather_kernel<<<slabs * kKvCluster, kKvThreads, 0, st>>>(ptrs, l0, Hkv, S_cap, S_cur, row_chunks,
+                                                                        keep_idx, keep_len, w.haz);
+            }
+            METOK_LAUNCH_CHECK();
         }
-        METOK_LAUNCH_CHECK();
     }
     return METOK_OK;
 }

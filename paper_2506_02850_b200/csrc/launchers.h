@@ -7,13 +7,14 @@
 
 namespace metok {
 
-// Class-wise top-k + ascending keep list, one CTA per problem p in [0, problems):
+// Class-wise top-k + ascending keep list, one cluster per problem p in [0, problems):
 // scores + p*score_stride, keep_idx + p*keep_stride, counts written to count_a[p]
 // and count_b[p] (either may be null).  token_group may be null (single class).
-// budgets_host is a HOST array of G ints.
+// budgets_host is a HOST array of G ints.  With replicas > 1 (problems == 1) the one
+// list and its length are written `replicas` times, keep_stride apart.
 int launch_class_topk(const float* scores, size_t score_stride, const int32_t* token_group, int n_vis, int G,
                       const int32_t* budgets_host, int S, int vis_start, int32_t* keep_idx, size_t keep_stride,
-                      int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st);
+                      int replicas, int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st);
 
 // dst[i] = src[idx[i]] for i < *n_rows (device scalar); rows of row_chunks 16-byte chunks.
 // timer_name labels the launch in the per-kernel timing report.

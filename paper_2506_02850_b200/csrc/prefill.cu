@@ -228,8 +228,8 @@ struct TopkBudgets { int v[METOK_MAX_GROUPS]; };
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 class_topk_kernel(const float* __restrict__ scores, size_t score_stride, const int32_t* __restrict__ token_group,
                   int n_vis, int G, SelectLayout lay, TopkBudgets budgets, int S, int vis_start,
-                  int32_t* __restrict__ keep_idx, size_t keep_stride, int32_t* __restrict__ count_a,
-                  int32_t* __restrict__ count_b) {
+                  int32_t* __restrict__ keep_idx, size_t keep_stride, int replicas,
+                  int32_t* __restrict__ count_a, int32_t* __restrict__ count_b) {
     __shared__ SelectSmem sm;
     __shared__ int s_budget[METOK_MAX_GROUPS];
     extern __shared__ __align__(16) unsigned char sel_dyn[];
@@ -266,17 +266,22 @@ class_topk_kernel(const float* __restrict__ scores, size_t score_stride, const i
         const SelItem it = item_at(cx, i - cx.item_lo, cls, val);
         return it.cls >= 0 && is_selected(sm, it.cls, it.key, i);
     };
-    auto emit = [&](int u, int rank) { keep[rank] = u; };
+    // one list may serve several layers: `replicas` copies, keep_stride apart
+    auto emit = [&](int u, int rank) {
+        for (int r = 0; r < replicas; ++r) keep[(size_t)r * keep_stride + rank] = u;
+    };
     const int total = cluster_compact(cx, p_lo, p_hi, flag, emit, sm);
-    if (threadIdx.x == 0 && cx.rank == 0) {
-        if (count_a) count_a[problem] = total;
-        if (count_b) count_b[problem] = total;
+    if (cx.rank == 0) {
+        for (int r = threadIdx.x; r < replicas; r += blockDim.x) {
+            if (count_a) count_a[problem + r] = total;
+            if (count_b) count_b[problem + r] = total;
+        }
     }
 }
 
 int launch_class_topk(const float* scores, size_t score_stride, const int32_t* token_group, int n_vis, int G,
                       const int32_t* budgets_host, int S, int vis_start, int32_t* keep_idx, size_t keep_stride,
-                      int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st) {
+                      int replicas, int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st) {
     TopkBudgets b;
     for (int g = 0; g < METOK_MAX_GROUPS; ++g) b.v[g] = g < G ? budgets_host[g] : 0;
     const SelectLayout lay = select_layout(G, select_items_per_cta((long long)S));
@@ -287,8 +292,8 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
     {
         METOK_TIMED("class_topk_kernel", st);
         class_topk_kernel<<<problems * kSelCluster, nthreads, lay.bytes, st>>>(
-            scores, score_stride, token_group, n_vis, G, lay, b, S, vis_start, keep_idx, keep_stride, count_a,
-            count_b);
+            scores, score_stride, token_group, n_vis, G, lay, b, S, vis_start, keep_idx, keep_stride, replicas,
+            count_a, count_b);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;
@@ -473,8 +478,8 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
                                 : launch_attn_scores<__nv_bfloat16>(q_text, k_all, dm, w, scores, st);
     }
     if (rc != METOK_OK) return rc;
-    rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, S_out, nullptr,
-                           1, st);
+    rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, 1, S_out,
+                           nullptr, 1, st);
     if (rc != METOK_OK) return rc;
     if (hidden) {
         const int row_chunks = (int)((long long)D * eb / 16);

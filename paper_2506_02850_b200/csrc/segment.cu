@@ -159,16 +159,24 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
     __shared__ int s_scan[1024];
     const int tid = threadIdx.x, nthr = blockDim.x;
 
-    for (int f = tid; f < Tn; f += nthr) {
-        float a = 0.f;
-        for (int s = 0; s < nslab; ++s) a += part_nrm[(size_t)s * Tn + f];
-        s_nrm[f] = fmaxf(sqrtf(a), kEps);
+    // a warp per frame: lanes take the slabs 32 apart, then a fixed shuffle tree
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
+    for (int f = warp; f < Tn; f += nwarps) {
+        float a = 0.f, b = 0.f;
+        for (int s = lane; s < nslab; s += 32) {
+            a += part_nrm[(size_t)s * Tn + f];
+            if (f < Tn - 1) b += part_dot[(size_t)s * Tn + f];
+        }
+        a = warp_sum(a);
+        b = warp_sum(b);
+        if (lane == 0) {
+            s_nrm[f] = fmaxf(sqrtf(a), kEps);
+            s_sim[f] = b;                                   // dot product for now
+        }
     }
     __syncthreads();
     for (int i = tid; i < Tn - 1; i += nthr) {
-        float a = 0.f;
-        for (int s = 0; s < nslab; ++s) a += part_dot[(size_t)s * Tn + i];
-        const float c = a / (s_nrm[i] * s_nrm[i + 1]);
+        const float c = s_sim[i] / (s_nrm[i] * s_nrm[i + 1]);
         s_sim[i] = c;
         sims[i] = c;
     }

@@ -97,32 +97,30 @@ tok_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Nv
     }
 }
 
-// frame_score[f] = mean of the frame's N token scores; one warp per frame, fixed order.
-__global__ void __launch_bounds__(256)
-frame_score_kernel(const float* __restrict__ token_score, int Tn, int N, float* __restrict__ frame_score) {
-    const int f = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (f >= Tn) return;
-    const int lane = threadIdx.x & 31;
-    float s = 0.f;
-    for (int p = lane; p < N; p += 32) s += token_score[(size_t)f * N + p];
-    s = warp_sum(s);
-    if (lane == 0) frame_score[f] = s / (float)N;
-}
-
 // Event scores, key events, per-event token budgets and output offsets.  One CTA.
 struct PlanParams {
-    int Tn, N, k, n_key_events, event_agg, mode, tile_rows;
+    int Tn, N, k, n_key_events, event_agg, mode, tile_rows, chunk_cols;
     double keep_key, keep_nonkey, beta;
 };
 
 __global__ void __launch_bounds__(1024)
-event_plan_kernel(const float* __restrict__ frame_score, const int32_t* __restrict__ event_offsets, PlanParams pp,
+event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ frame_score,
+                  const int32_t* __restrict__ event_offsets, PlanParams pp,
                   float* __restrict__ event_score, uint8_t* __restrict__ event_is_key,
                   int32_t* __restrict__ ev_lo, int32_t* __restrict__ ev_budget, int32_t* __restrict__ ev_out_off,
-                  int32_t* __restrict__ ev_tile_off, int32_t* __restrict__ n_out) {
+                  int32_t* __restrict__ ev_tile_off, int32_t* __restrict__ ev_unit_off,
+                  int32_t* __restrict__ n_out) {
     extern __shared__ float s_score[];      // [k]
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int k = pp.k, Tn = pp.Tn;
+    // frame_score[f] = mean of the frame's N token scores; one warp per frame, fixed order
+    for (int f = tid >> 5; f < Tn; f += nthr >> 5) {
+        float s = 0.f;
+        for (int p = tid & 31; p < pp.N; p += 32) s += token_score[(size_t)f * pp.N + p];
+        s = warp_sum(s);
+        if ((tid & 31) == 0) frame_score[f] = s / (float)pp.N;
+    }
+    __syncthreads();
     for (int e = tid; e < k; e += nthr) {
         int lo = min(max(event_offsets[e], 0), Tn);
         int hi = min(max(event_offsets[e + 1], lo), Tn);
@@ -169,17 +167,21 @@ event_plan_kernel(const float* __restrict__ frame_score, const int32_t* __restri
         }
         __syncthreads();
         if (tid == 0) {
-            int slots = 0, tiles = 0;
+            int slots = 0, tiles = 0, units = 0;
             for (int e = 0; e < k; ++e) {
                 ev_out_off[e] = slots;
                 ev_tile_off[e] = tiles;
+                ev_unit_off[e] = units;
                 const int lo = min(max(event_offsets[e], 0), Tn);
                 const int hi = min(max(event_offsets[e + 1], lo), Tn);
                 slots += ev_budget[e];
-                tiles += ((hi - lo) * pp.N + pp.tile_rows - 1) / pp.tile_rows;
+                const int t = ((hi - lo) * pp.N + pp.tile_rows - 1) / pp.tile_rows;
+                tiles += t;
+                units += t * ((ev_budget[e] + pp.chunk_cols - 1) / pp.chunk_cols);   // row tiles x key chunks
             }
             ev_out_off[k] = slots;
             ev_tile_off[k] = tiles;
+            ev_unit_off[k] = units;
             *n_out = slots;
         }
     }
@@ -347,15 +349,23 @@ merge_assign_simt_kernel(const T* __restrict__ feats, int d, int N, const int32_
 
 
 // --------------------------------------------------------------------------- //
-// Merge-assign on the tensor cores (bf16).  CTA = 128 consecutive token rows of one
-// event (TMEM lanes) x the event's key tokens in chunks of up to 256 columns.
+// Merge-assign on the tensor cores (bf16).
+//
+// Work unit = 128 consecutive token rows of one event (TMEM lanes) x one chunk of the
+// event's key tokens (up to 256 columns; an event's keys are cut into equal chunks).
+// The units of all events form one list; a persistent CTA per SM takes every
+// gridDim-th unit, so the load is balanced whatever the event lengths are, and with two
+// accumulators in TMEM the epilogue of a unit overlaps the main loop of the next.
 //   warp 0   : TMA producer -- per 64-wide K step one 128x64 tile of V (rows are
 //              contiguous in V) and the chunk's key rows from the compact key buffer
-//              (64-row boxes), 4-stage ring;
+//              (64-row boxes), 4-stage ring that runs on across units;
 //   warp 1   : allocates TMEM (2 accumulators x 256 columns), issues tcgen05.mma
 //              (M=128, N=16..256, K=16) and commits to the ring / accumulator barriers;
 //   warps 2-5: epilogue -- read the accumulator with tcgen05.ld, scale each column by
-//              1/|key|, keep the running (value, slot) argmax of the thread's row.
+//              1/|key|, take the (value, slot) argmax of the thread's row over the chunk.
+// Chunks of one row tile may be handled by different CTAs: a row's result is combined
+// with a 64-bit atomicMax on (order-preserving key of the value) << 32 | ~slot, which
+// does not depend on the order of arrival (larger value first, then the lower slot).
 // Every wait is bounded; on a timeout the CTA unwinds and writes METOK_ERR_TIMEOUT.
 // --------------------------------------------------------------------------- //
 constexpr int kMmaBM = 128, kMmaBK = 64, kMmaBN = 256, kMmaStages = 4;
@@ -365,27 +375,40 @@ constexpr uint32_t kMmaBBytes = kMmaBN * kMmaBK * 2;       // 32 KiB
 constexpr uint32_t kMmaBoxBytes = 64 * kMmaBK * 2;         // one 64-row key box
 constexpr size_t kMmaSmemBytes = (size_t)kMmaStages * (kMmaABytes + kMmaBBytes) + 1024;
 
+struct MergeUnit { int row0, row_end, col0, nvalid; };     // rows of V; first key slot and number of keys
+
+__device__ __forceinline__ MergeUnit merge_unit(int u, const int32_t* __restrict__ ev_unit_off,
+                                                const int32_t* __restrict__ ev_lo,
+                                                const int32_t* __restrict__ ev_out_off, int k, int N) {
+    const int e = find_event(ev_unit_off, k, u);
+    const int s0 = ev_out_off[e], nk = ev_out_off[e + 1] - s0;
+    const int nchunks = (nk + kMmaBN - 1) / kMmaBN;
+    const int cols = (((nk + nchunks - 1) / nchunks) + 15) & ~15;       // equal chunks, whole MMA columns
+    const int local = u - ev_unit_off[e];
+    const int tile = local / nchunks, c = local - tile * nchunks;
+    MergeUnit m;
+    m.row0 = ev_lo[e] * N + tile * kMmaBM;
+    m.row_end = ev_lo[e + 1] * N;
+    m.col0 = s0 + c * cols;
+    m.nvalid = min(cols, nk - c * cols);
+    return m;
+}
+
 __global__ void __launch_bounds__(kMmaThreads, 1)
 merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int d, int N,
                         const int32_t* __restrict__ ev_lo, int k, const int32_t* __restrict__ ev_out_off,
-                        const int32_t* __restrict__ ev_tile_off, const int32_t* __restrict__ out_src,
+                        const int32_t* __restrict__ ev_unit_off, const int32_t* __restrict__ out_src,
                         const float* __restrict__ inv_norm, const uint8_t* __restrict__ is_key,
-                        int32_t* __restrict__ assign, int32_t* __restrict__ status) {
+                        unsigned long long* __restrict__ best64, int32_t* __restrict__ status) {
     using namespace sm100;
     extern __shared__ uint8_t smem_dyn[];
-    __shared__ __align__(8) uint64_t full_bar[kMmaStages], empty_bar[kMmaStages], tfull_bar[2], tempty_bar[2];
+    __shared__ __align__(8) uint64_t full_bar[kMmaStages], empty_bar[kMmaStages], tfull_bar[2], tempty_bar[2], drain_bar;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ float s_keyinv[2][kMmaBN];
 
-    const int tile = blockIdx.x;
-    if (tile >= ev_tile_off[k]) return;
-    const int e = find_event(ev_tile_off, k, tile);
-    const int row0 = ev_lo[e] * N + (tile - ev_tile_off[e]) * kMmaBM;
-    const int row_end = ev_lo[e + 1] * N;
-    const int s0 = ev_out_off[e], s1 = ev_out_off[e + 1];
-    const int nk = s1 - s0;
-    const int nchunks = (nk + kMmaBN - 1) / kMmaBN;
+    const int total_units = ev_unit_off[k];
+    if ((int)blockIdx.x >= total_units) return;
     const int ksteps = (d + kMmaBK - 1) / kMmaBK;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -396,6 +419,7 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tfull_bar[b]), 1); mbar_init(smem_u32(&tempty_bar[b]), 4); }
+        mbar_init(smem_u32(&drain_bar), 1);
         s_abort = 0;
         mbar_fence_init();
     }
@@ -415,19 +439,18 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             prefetch_tmap(&tmB);
             int it = 0;
             bool ok = true;
-            for (int c = 0; c < nchunks && ok; ++c) {
-                const int nvalid = min(kMmaBN, nk - c * kMmaBN);
-                const int nbox = (nvalid + 63) >> 6;
+            for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+                const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
+                const int nbox = (mu.nvalid + 63) >> 6;
                 for (int ks = 0; ks < ksteps; ++ks, ++it) {
                     const int s = it % kMmaStages;
                     const uint32_t ph = (uint32_t)(it / kMmaStages) & 1u;
                     if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t fb = smem_u32(&full_bar[s]);
                     mbar_arrive_expect_tx(fb, kMmaABytes + (uint32_t)nbox * kMmaBoxBytes);
-                    tma_load_2d(a_addr(s), &tmA, ks * kMmaBK, row0, fb);
+                    tma_load_2d(a_addr(s), &tmA, ks * kMmaBK, mu.row0, fb);
                     for (int j = 0; j < nbox; ++j)
-                        tma_load_2d(b_addr(s) + (uint32_t)j * kMmaBoxBytes, &tmB, ks * kMmaBK,
-                                    s0 + c * kMmaBN + j * 64, fb);
+                        tma_load_2d(b_addr(s) + (uint32_t)j * kMmaBoxBytes, &tmB, ks * kMmaBK, mu.col0 + j * 64, fb);
                 }
             }
             if (!ok) {
@@ -440,15 +463,14 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            int it = 0;
+            int it = 0, n = 0;
             bool ok = true;
-            for (int c = 0; c < nchunks && ok; ++c) {
-                const int b = c & 1;
-                const uint32_t use = (uint32_t)(c >> 1);
-                if (!mbar_wait(smem_u32(&tempty_bar[b]), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+            for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++n) {
+                const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
+                const int b = n & 1;
+                if (!mbar_wait(smem_u32(&tempty_bar[b]), ((uint32_t)(n >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const int nvalid = min(kMmaBN, nk - c * kMmaBN);
-                const uint32_t idesc = make_idesc_bf16(kMmaBM, (nvalid + 15) & ~15);
+                const uint32_t idesc = make_idesc_bf16(kMmaBM, (mu.nvalid + 15) & ~15);
                 const uint32_t d_tmem = tmem_base + (uint32_t)b * kMmaBN;
                 for (int ks = 0; ks < ksteps; ++ks, ++it) {
                     const int s = it % kMmaStages;
@@ -463,51 +485,64 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     }
                     umma_commit(smem_u32(&empty_bar[s]));          // frees the stage when these MMAs retire
                 }
-                if (ok) umma_commit(smem_u32(&tfull_bar[b]));      // accumulator of chunk c complete
+                if (ok) umma_commit(smem_u32(&tfull_bar[b]));      // accumulator of this unit complete
+            }
+            if (!ok) {                                             // wait until whatever was issued has retired
+                umma_commit(smem_u32(&drain_bar));
+                mbar_wait(smem_u32(&drain_bar), 0u, abort_flag);
             }
         }
     } else {
         const int grp = warp & 3;                                   // TMEM lanes 32*grp .. 32*grp+31
         const int et = (warp - 2) * 32 + lane;                      // 0..127 among the epilogue threads
-        const int row = row0 + grp * 32 + lane;
-        float best_v = -3.4e38f;
-        int best_s = 0x7FFFFFFF;
         bool ok = true;
-        for (int c = 0; c < nchunks; ++c) {
-            const int b = c & 1;
-            const uint32_t use = (uint32_t)(c >> 1);
-            const int nvalid = min(kMmaBN, nk - c * kMmaBN);
-            for (int i = et; i < kMmaBN; i += 128) {
-                const int slot = s0 + c * kMmaBN + i;
-                s_keyinv[b][i] = (i < nvalid) ? inv_norm[out_src[slot]] : 0.f;
-            }
+        int n = 0;
+        for (int u = blockIdx.x; u < total_units; u += gridDim.x, ++n) {
+            const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
+            const int b = n & 1;
+            for (int i = et; i < kMmaBN; i += 128)
+                s_keyinv[b][i] = (i < mu.nvalid) ? inv_norm[out_src[mu.col0 + i]] : 0.f;
             named_bar_sync(1, 128);
-            if (ok && !mbar_wait(smem_u32(&tfull_bar[b]), use & 1u, abort_flag)) ok = false;
+            if (ok && !mbar_wait(smem_u32(&tfull_bar[b]), (uint32_t)(n >> 1) & 1u, abort_flag)) ok = false;
             ok = __all_sync(0xFFFFFFFFu, ok);                      // tcgen05.ld below is warp-collective
-            if (ok) {
-                tc_fence_after();
-                const uint32_t t_row = tmem_base + ((uint32_t)(grp * 32) << 16) + (uint32_t)b * kMmaBN;
-                for (int c0 = 0; c0 < nvalid; c0 += 32) {
-                    float v[32];
-                    tmem_ld32(t_row + (uint32_t)c0, v);
+            if (!ok) continue;                                     // keep meeting the others at the named barrier
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(grp * 32) << 16) + (uint32_t)b * kMmaBN;
+            float best_v = -3.4e38f;
+            int best_c = 0;
+            for (int c0 = 0; c0 < mu.nvalid; c0 += 32) {
+                float v[32];
+                tmem_ld32(t_row + (uint32_t)c0, v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int col = c0 + j;
-                        const float val = v[j] * s_keyinv[b][col];
-                        if (col < nvalid && val > best_v) { best_v = val; best_s = s0 + c * kMmaBN + col; }
-                    }
+                for (int j = 0; j < 32; ++j) {
+                    const int col = c0 + j;
+                    const float val = v[j] * s_keyinv[b][col];
+                    if (col < mu.nvalid && val > best_v) { best_v = val; best_c = col; }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[b]));
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[b]));
+            const int row = mu.row0 + grp * 32 + lane;
+            if (row < mu.row_end && !is_key[row]) {
+                const unsigned long long packed =
+                    ((unsigned long long)float_key(best_v) << 32) | (unsigned long long)(~(uint32_t)(mu.col0 + best_c));
+                atomicMax(&best64[row], packed);
             }
         }
-        if (ok && row < row_end && !is_key[row]) assign[row] = best_s;
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
     if (threadIdx.x == 0 && s_abort) *status = METOK_ERR_TIMEOUT;
+}
+
+// assign[row] of every non-key token from the packed argmax.
+__global__ void __launch_bounds__(256)
+merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t* __restrict__ is_key, int Nv,
+                    int32_t* __restrict__ assign) {
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row < Nv && !is_key[row]) assign[row] = (int32_t)(~(uint32_t)(best64[row] & 0xFFFFFFFFull));
 }
 
 // --------------------------------------------------------------------------- //
@@ -657,7 +692,8 @@ struct VisionWs {
     void* key_rows;           // compact copy of the key-token rows (tensor-core path)
     float* inv_norm;
     uint8_t* is_key;
-    int32_t *ev_lo, *ev_budget, *ev_out_off, *ev_tile_off;
+    int32_t *ev_lo, *ev_budget, *ev_out_off, *ev_tile_off, *ev_unit_off;
+    unsigned long long* best64;   // packed argmax per token (tensor-core path)
 };
 
 static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, bool mma) {
@@ -670,6 +706,8 @@ static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, b
     w.ev_budget = cv.take<int32_t>((size_t)k + 1);
     w.ev_out_off = cv.take<int32_t>((size_t)k + 1);
     w.ev_tile_off = cv.take<int32_t>((size_t)k + 1);
+    w.ev_unit_off = cv.take<int32_t>((size_t)k + 1);
+    w.best64 = mma ? cv.take<unsigned long long>((size_t)Tn * N) : nullptr;
     return w;
 }
 
@@ -710,22 +748,17 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         }
         METOK_LAUNCH_CHECK();
     }
-    {
-        METOK_TIMED("frame_score_kernel", st);
-        frame_score_kernel<<<ceil_div(Tn, 8), 256, 0, st>>>(token_score, Tn, N, frame_score);
-    }
-    METOK_LAUNCH_CHECK();
-
     PlanParams pp;
     pp.Tn = Tn; pp.N = N; pp.k = k;
     pp.n_key_events = min(k, ceilq(p->alpha * (double)k));
     pp.event_agg = p->event_agg; pp.mode = p->mode; pp.tile_rows = mma ? kMmaBM : kMergeTM;
+    pp.chunk_cols = kMmaBN;
     pp.keep_key = p->keep_key; pp.keep_nonkey = p->keep_nonkey; pp.beta = p->beta;
     {
         METOK_TIMED("event_plan_kernel", st);
-        event_plan_kernel<<<1, 1024, (size_t)k * sizeof(float), st>>>(frame_score, event_offsets, pp, event_score,
+        event_plan_kernel<<<1, 1024, (size_t)k * sizeof(float), st>>>(token_score, frame_score, event_offsets, pp, event_score,
                                                                   event_is_key, w.ev_lo, w.ev_budget, w.ev_out_off,
-                                                                  w.ev_tile_off, n_out);
+                                                                  w.ev_tile_off, w.ev_unit_off, n_out);
     }
     METOK_LAUNCH_CHECK();
 
@@ -756,12 +789,17 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         if (r2 != METOK_OK) return r2;
         METOK_CUDA_TRY(cudaFuncSetAttribute(merge_assign_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)kMmaSmemBytes));
-        const int max_tiles = Nv / kMmaBM + k;
+        METOK_CUDA_TRY(cudaMemsetAsync(w.best64, 0, (size_t)Nv * sizeof(unsigned long long), st));
         {
             METOK_TIMED("merge_assign_mma_kernel", st);
-            merge_assign_mma_kernel<<<max_tiles, kMmaThreads, kMmaSmemBytes, st>>>(
-                tmA, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_tile_off, out_src, w.inv_norm, w.is_key, assign,
+            merge_assign_mma_kernel<<<kNumSMs, kMmaThreads, kMmaSmemBytes, st>>>(
+                tmA, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, w.inv_norm, w.is_key, w.best64,
                 w.status);
+        }
+        METOK_LAUNCH_CHECK();
+        {
+            METOK_TIMED("merge_decode_kernel", st);
+            merge_decode_kernel<<<ceil_div(Nv, 256), 256, 0, st>>>(w.best64, w.is_key, Nv, assign);
         }
         METOK_LAUNCH_CHECK();
     } else {

@@ -75,12 +75,16 @@ def schedule(cfg, B, vis):
     return stages
 
 
+PARTS = ("segment", "compress", "prefill", "kv")
+
+
 class Workload:
-    def __init__(self, cfg, device, host_copies: bool):
+    def __init__(self, cfg, device, host_copies: bool, parts=PARTS):
         from paper_2506_02850_b200 import binding as B
         self.B = B
         self.cfg = cfg
         self.dev = device
+        self.parts = tuple(parts)
         tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
         vis = W.vision_inputs(cfg)
         self.vis = vis
@@ -97,8 +101,9 @@ class Workload:
         self.V = put("V", vis["V"])
         self.t = put("t", vis["t"])
         self.params = B.vision_params(cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+        self.planted_offsets = torch.from_numpy(np.asarray(vis["event_offsets"], dtype=np.int32)).to(device)
         self.stages = []
-        for si, (groups, budgets) in enumerate(schedule(cfg, B, vis), start=1):
+        for si, (groups, budgets) in enumerate(schedule(cfg, B, vis) if "prefill" in self.parts else [], start=1):
             pf = W.prefill_inputs(cfg, si, groups.size, groups)
             hidden = W.payload_torch(W.hidden_salt(cfg, si), pf["S"], cfg.D, cfg.dtype, device)
             self.stages.append({
@@ -108,7 +113,7 @@ class Workload:
             })
         self.kv_layers = cfg.L
         self.S_cur = cfg.Nv + cfg.kv_text
-        self.ks, self.vs = W.kv_cache_torch(cfg, device)
+        self.ks, self.vs = W.kv_cache_torch(cfg, device) if "kv" in self.parts else ([], [])
         if host_copies:
             self.h["ks"] = [t.cpu().pin_memory() for t in self.ks]
             self.h["vs"] = [t.cpu().pin_memory() for t in self.vs]
@@ -119,11 +124,16 @@ class Workload:
     # one pass of the hot path, device-resident inputs
     def step(self):
         B, cfg, o = self.B, self.cfg, self.out
-        o["seg"] = B.metok_segment_events(self.V, cfg.k, out=o.get("seg"))
-        o["cv"] = B.metok_compress_vision(self.V, o["seg"]["event_offsets"], self.t, self.params, out=o.get("cv"))
+        if "segment" in self.parts:
+            o["seg"] = B.metok_segment_events(self.V, cfg.k, out=o.get("seg"))
+        if "compress" in self.parts:
+            offs = o["seg"]["event_offsets"] if "seg" in o else self.planted_offsets
+            o["cv"] = B.metok_compress_vision(self.V, offs, self.t, self.params, out=o.get("cv"))
         for i, s in enumerate(self.stages):
             o[f"pf{i}"] = B.metok_prefill_prune(s["Q"], s["K"], s["hidden"], 0, s["n_vis"], s["groups"], s["budgets"],
                                                 self.scale, out=o.get(f"pf{i}"))
+        if "kv" not in self.parts:
+            return
         # KV selection uses the first pruning layer's attention scores (n_vis = all visual tokens)
         scores = o["pf0"]["scores"] if self.stages and self.stages[0]["n_vis"] == cfg.Nv else self.kv_scores
         kv = o.get("kv")
@@ -336,6 +346,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph of the step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--parts", default=",".join(PARTS),
+                    help="comma-separated subset of the four calls (for profiler captures that should hold little "
+                         "memory); anything but the full list is not a benchmark result")
     args = ap.parse_args()
     cfg = W.CONFIGS[args.config]
     rank = int(os.environ.get("RANK", "0"))
@@ -373,7 +386,12 @@ def main():
 
     from paper_2506_02850_b200 import binding as B
     B.lib()
-    wl = Workload(cfg, dev, host_copies=not args.no_e2e)
+    parts = tuple(p for p in args.parts.split(",") if p)
+    assert all(p in PARTS for p in parts), parts
+    partial = set(parts) != set(PARTS)
+    if partial:
+        args.no_e2e = True
+    wl = Workload(cfg, dev, host_copies=not args.no_e2e, parts=parts)
     warm = max(args.warmup, 3)
 
     def barrier():
@@ -478,6 +496,8 @@ def main():
                 "launch": "cuda_graph" if graph is not None else "eager", "eager_ms_per_step": eager_ms_per_step,
                 "host_enqueue_ms_per_step": host_ms.get("step"), "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
                 "roofline": roofline, "cpu_baseline": cpu}
+        if partial:
+            line["partial"] = "only " + ",".join(parts) + ": not a benchmark result"
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -189,30 +189,40 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             const int u0 = u_tile + half * (kStBN / 2);
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * kStBN + half * (kStBN / 2));
             const bool masked = u_tile + kStBN - 1 > text_start;       // some query cannot see some key of the tile
-#pragma unroll 1
-            for (int c0 = 0; c0 < kStBN / 2; c0 += 32) {
+            uint32_t raw[2][32];
+            tmem_ld32_issue(taddr, raw[0]);
+#pragma unroll
+            for (int ci = 0; ci < kStBN / 64; ++ci) {
+                // the next 32 columns are fetched while these are reduced
+                const int c0 = ci * 32;
+                tmem_ld32_wait(raw[ci & 1]);
+                if (ci + 1 < kStBN / 64) tmem_ld32_issue(taddr + (uint32_t)(c0 + 32), raw[(ci + 1) & 1]);
                 float v[32];
-                tmem_ld32(taddr + (uint32_t)c0, v);
-                if (masked) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[ci & 1][j]);
+                float a0 = 0.f, a1 = 0.f;
+                float m_new;
+                if (masked) {                                  // hidden keys add exactly nothing
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = (u0 + c0 + j <= limit) ? v[j] * sc : kNegInf;
-                } else {
+                    float cm = v[0];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] *= sc;
-                }
-                float cm = v[0];
-#pragma unroll
-                for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
-                const float m_new = fmaxf(m_run, cm);
-                float a0 = 0.f, a1 = 0.f;
-                if (masked) {                                  // hidden keys add exactly nothing
+                    for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
+                    m_new = fmaxf(m_run, cm);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) a0 += (v[j] > kNegInf) ? fast_exp2(v[j] - m_new) : 0.f;
                 } else {
+                    // the scale is positive: the maximum of the raw logits, scaled, is the maximum of the
+                    // scaled ones, and scaling folds into the exponent's multiply-add
+                    float cm = v[0];
+#pragma unroll
+                    for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
+                    m_new = fmaxf(m_run, cm * sc);
+                    const float neg_m = -m_new;
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
-                        a0 += fast_exp2(v[j] - m_new);
-                        a1 += fast_exp2(v[j + 1] - m_new);
+                        a0 += fast_exp2(fmaf(v[j], sc, neg_m));
+                        a1 += fast_exp2(fmaf(v[j + 1], sc, neg_m));
                     }
                 }
                 l_run = l_run * fast_exp2(m_run - m_new) + (a0 + a1);

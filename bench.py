@@ -119,6 +119,7 @@ class Workload:
             self.h["vs"] = [t.cpu().pin_memory() for t in self.vs]
         self.kv_scores = torch.from_numpy(W.kv_scores(cfg, cfg.Nv)).to(device)
         self.out = {}
+        self.side = None
         self.scale = float(cfg.dh ** -0.5)
 
     # one pass of the hot path, device-resident inputs
@@ -129,11 +130,27 @@ class Workload:
         if "compress" in self.parts:
             offs = o["seg"]["event_offsets"] if "seg" in o else self.planted_offsets
             o["cv"] = B.metok_compress_vision(self.V, offs, self.t, self.params, out=o.get("cv"))
+        # The K/V lists need the first level's scores only: the compaction runs on a second stream
+        # beside pruning levels 2 and 3 and joins at the end of the step.
+        main = torch.cuda.current_stream()
+        if self.side is None:
+            self.side = torch.cuda.Stream()
+        forked = False
         for i, s in enumerate(self.stages):
             o[f"pf{i}"] = B.metok_prefill_prune(s["Q"], s["K"], s["hidden"], 0, s["n_vis"], s["groups"], s["budgets"],
                                                 self.scale, out=o.get(f"pf{i}"))
-        if "kv" not in self.parts:
-            return
+            if i == 0 and "kv" in self.parts:
+                self.side.wait_stream(main)
+                with torch.cuda.stream(self.side):
+                    self._kv_call()
+                forked = True
+        if "kv" in self.parts and not forked:
+            self._kv_call()
+        if forked:
+            main.wait_stream(self.side)
+
+    def _kv_call(self):
+        B, cfg, o = self.B, self.cfg, self.out
         # KV selection uses the first pruning layer's attention scores (n_vis = all visual tokens)
         scores = o["pf0"]["scores"] if self.stages and self.stages[0]["n_vis"] == cfg.Nv else self.kv_scores
         kv = o.get("kv")

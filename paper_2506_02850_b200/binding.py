@@ -122,8 +122,9 @@ _ws_cache: Dict[tuple, torch.Tensor] = {}
 
 
 def workspace(nbytes: int, device) -> torch.Tensor:
-    """A reusable scratch buffer per device (calls on one stream never overlap)."""
-    key = (str(device),)
+    """A reusable scratch buffer per device and stream: calls on one stream never overlap,
+    calls on different streams may, so they must not share scratch."""
+    key = (str(device), torch.cuda.current_stream(device).cuda_stream)
     buf = _ws_cache.get(key)
     if buf is None or buf.numel() < nbytes:
         buf = torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=device)

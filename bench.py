@@ -298,36 +298,45 @@ class ClockSampler:
 
 
 def oracle_sample_step(cfg, sample):
-    """One pass of the oracle over the sample (a prefix of the video, fewer KV layers)."""
+    """One pass of the oracle over the sample."""
     from oracle import metok_oracle as O
-    V, t, offs, groups, budgets, Q, K, hidden, kv = sample
+    V, t, offs, levels, kv = sample
     O.segment_events(V, len(offs) - 1)
     O.compress_vision(V, t, offs, cfg.alpha, cfg.keep_enc, cfg.keep_enc, cfg.dtype)
-    pr = O.prefill_prune(Q, K, hidden, 0, groups.size, groups, budgets, cfg.dh ** -0.5)
-    lists = O.kv_select(O.KV_TOPK, len(kv[0]), kv[0][0].shape[1], 0, groups.size, keep_ratio=cfg.keep_kv,
-                        scores=pr["scores"])
+    first = None
+    for groups, budgets, Q, K, hidden in levels:
+        pr = O.prefill_prune(Q, K, hidden, 0, groups.size, groups, budgets, cfg.dh ** -0.5)
+        first = pr if first is None else first
+    lists = O.kv_select(O.KV_TOPK, len(kv[0]), kv[0][0].shape[1], 0, levels[0][0].size, keep_ratio=cfg.keep_kv,
+                        scores=first["scores"])
     O.kv_compact(kv[0], kv[1], lists)
 
 
-def oracle_sample(cfg, frames=24, kv_layers=2):
+def oracle_sample(cfg, kv_layers=4):
+    """The whole video through segmentation, stage-1 compression and every pruning level; the K/V
+    compaction on `kv_layers` of the layers (building all of them on the host takes minutes)."""
     from oracle import metok_oracle as O
     vis = W.vision_inputs(cfg)
-    T = min(frames, cfg.T)
-    V = vis["V"][:T]
-    offs = np.unique(np.clip(vis["event_offsets"], 0, T)).astype(np.int32)
-    n_vis = T * cfg.N
-    groups = W.token_groups(cfg, cfg.Nv, vis=vis)[:n_vis]
-    N0 = [int((groups == 0).sum()), int((groups == 1).sum())]
-    budgets = O.retention_budgets(cfg.alpha, cfg.keep_prefill, 1, N0).tolist()
-    pf = W.prefill_inputs(cfg, 1, n_vis, groups)
-    hidden = W.payload_rows_np(W.hidden_salt(cfg, 1), np.arange(pf["S"]), cfg.D, cfg.dtype)
-    S = n_vis + cfg.kv_text
-    kv = ([np.stack([W.payload_rows_np(W.kv_salt(cfg, l, w, h), np.arange(S), cfg.dh, cfg.dtype)
-                     for h in range(cfg.Hkv)]) for l in range(kv_layers)] for w in (0, 1))
-    kv = tuple(kv)
-    what = (f"first {T} of {cfg.T} frames ({n_vis} visual tokens): segmentation, stage-1 compression, "
-            f"pruning level 1, KV TOPK compaction of {kv_layers} of {cfg.L} layers")
-    return (V, vis["t"], offs, groups, budgets, pf["Q"], pf["K"], hidden, kv), n_vis, what
+    grp_full = W.token_groups(cfg, cfg.Nv, vis=vis)
+    N0 = [int((grp_full == 0).sum()), int((grp_full == 1).sum())]
+    levels = []
+    for stage in range(1, cfg.n_stages + 1):
+        if stage == 1:
+            groups = grp_full
+        else:
+            prev = O.retention_budgets(cfg.alpha, cfg.keep_prefill, stage - 1, N0)
+            groups = W.token_groups(cfg, int(prev.sum()), n_key=int(prev[0]), stage=stage)
+        budgets = O.retention_budgets(cfg.alpha, cfg.keep_prefill, stage, N0).tolist()
+        pf = W.prefill_inputs(cfg, stage, groups.size, groups)
+        hidden = W.payload_rows_np(W.hidden_salt(cfg, stage), np.arange(pf["S"]), cfg.D, cfg.dtype)
+        levels.append((groups, budgets, pf["Q"], pf["K"], hidden))
+    kv_layers = min(kv_layers, cfg.L)
+    S = cfg.Nv + cfg.kv_text
+    kv = tuple([np.stack([W.payload_rows_np(W.kv_salt(cfg, l, w, h), np.arange(S), cfg.dh, cfg.dtype)
+                          for h in range(cfg.Hkv)]) for l in range(kv_layers)] for w in (0, 1))
+    what = (f"all {cfg.T} frames ({cfg.Nv} visual tokens): segmentation, stage-1 compression, "
+            f"{cfg.n_stages} pruning levels, KV TOPK compaction of {kv_layers} of {cfg.L} layers")
+    return (vis["V"], vis["t"], vis["event_offsets"], levels, kv), cfg.Nv, what
 
 
 def cpu_threads():
@@ -500,7 +509,7 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, dt, what = time_oracle(cfg, 1, 0)
+        v, dt, what = time_oracle(cfg, 3, 1)
         cpu = {"value": v, "unit": "tokens/s", "cores": cpu_threads(), "kind": "oracle", "sample": what,
                "seconds": dt}
 

@@ -97,9 +97,20 @@ tok_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Nv
     }
 }
 
+// Index e with off[e] <= t < off[e+1] in an ascending offset array off[0..k].
+__device__ __forceinline__ int find_event(const int32_t* __restrict__ off, int k, int t) {
+    int lo = 0, hi = k;                     // off[lo] <= t < off[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (off[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
 // Event scores, key events, per-event token budgets and output offsets.  One CTA.
 struct PlanParams {
     int Tn, N, k, n_key_events, event_agg, mode, tile_rows, chunk_cols;
+    int grid, s1, s2, s1_nonkey, s2_nonkey;     // POOL: side of the token grid and the four strides
     double keep_key, keep_nonkey, beta;
 };
 
@@ -109,8 +120,10 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
                   float* __restrict__ event_score, uint8_t* __restrict__ event_is_key,
                   int32_t* __restrict__ ev_lo, int32_t* __restrict__ ev_budget, int32_t* __restrict__ ev_out_off,
                   int32_t* __restrict__ ev_tile_off, int32_t* __restrict__ ev_unit_off,
-                  int32_t* __restrict__ n_out) {
+                  int32_t* __restrict__ frame_ev, int32_t* __restrict__ frame_stride,
+                  int32_t* __restrict__ frame_off, int32_t* __restrict__ n_out) {
     extern __shared__ float s_score[];      // [k]
+    __shared__ int s_scan[1024];
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int k = pp.k, Tn = pp.Tn;
     // frame_score[f] = mean of the frame's N token scores; one warp per frame, fixed order
@@ -184,6 +197,150 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
             ev_unit_off[k] = units;
             *n_out = slots;
         }
+    } else {
+        // Algorithm 1: key frames = the ceil(beta * len) best-scored frames of every event (ties to the
+        // lower frame); a frame's stride follows from its event's and its own class; the pooled
+        // frames are laid out in temporal order.
+        for (int f = tid; f < Tn; f += nthr) frame_ev[f] = 0;
+        __syncthreads();
+        for (int e = tid; e < k; e += nthr) {
+            const int lo = min(max(event_offsets[e], 0), Tn);
+            const int hi = min(max(event_offsets[e + 1], lo), Tn);
+            for (int f = lo; f < hi; ++f) frame_ev[f] = e;
+        }
+        __syncthreads();
+        for (int f = tid; f < Tn; f += nthr) {
+            const int e = frame_ev[f];
+            const int lo = min(max(event_offsets[e], 0), Tn);
+            const int hi = min(max(event_offsets[e + 1], lo), Tn);
+            const int len = hi - lo;
+            const double c = pp.beta * (double)len - 1e-9;
+            long long nk = (long long)c;
+            if ((double)nk < c) nk += 1;
+            if (nk < 1) nk = 1;
+            if (nk > len) nk = len;
+            const float v = frame_score[f];
+            int rank = 0;
+            for (int j = lo; j < hi; ++j) {
+                const float w = frame_score[j];
+                rank += (w > v) || (w == v && j < f);
+            }
+            const bool key_frame = rank < (int)nk;
+            frame_stride[f] = event_is_key[e] ? (key_frame ? pp.s1 : pp.s2) : (key_frame ? pp.s1_nonkey : pp.s2_nonkey);
+        }
+        __syncthreads();
+        // exclusive scan of the pooled sizes: contiguous ranges per thread, then a scan of the range totals
+        const int per = (Tn + nthr - 1) / nthr;
+        const int lo = min(Tn, tid * per), hi = min(Tn, lo + per);
+        int local = 0;
+        for (int f = lo; f < hi; ++f) {
+            const int go = (pp.grid + frame_stride[f] - 1) / frame_stride[f];
+            local += go * go;
+        }
+        s_scan[tid] = local;
+        __syncthreads();
+        for (int off = 1; off < nthr; off <<= 1) {
+            const int v = (tid >= off) ? s_scan[tid - off] : 0;
+            __syncthreads();
+            s_scan[tid] += v;
+            __syncthreads();
+        }
+        int run = s_scan[tid] - local;
+        for (int f = lo; f < hi; ++f) {
+            frame_off[f] = run;
+            const int go = (pp.grid + frame_stride[f] - 1) / frame_stride[f];
+            run += go * go;
+        }
+        if (tid == nthr - 1) { frame_off[Tn] = s_scan[tid]; *n_out = s_scan[tid]; }
+    }
+}
+
+// --------------------------------------------------------------------------- //
+// Adaptive pooling (Algorithm 1): one CTA per output token = one window of one frame's
+// G x G token grid, window = stride, edge windows clipped to the grid.  The window's
+// cells are added in row-major order in fp32 (two rows of V in flight per thread),
+// divided by their number and rounded once.
+// --------------------------------------------------------------------------- //
+constexpr int kPoolThreads = 128;
+constexpr int kPoolChunks = 4;
+
+template <typename T>
+__global__ void __launch_bounds__(kPoolThreads)
+pool_kernel(const T* __restrict__ feats, int d, int N, int G, int Tn, const int32_t* __restrict__ frame_off,
+            const int32_t* __restrict__ frame_stride, const int32_t* __restrict__ frame_ev,
+            const int32_t* __restrict__ n_out, T* __restrict__ out_feats, int32_t* __restrict__ out_src,
+            int32_t* __restrict__ out_event, int32_t* __restrict__ out_members, int32_t* __restrict__ assign) {
+    constexpr int VN = Vec16<T>::N;
+    const int o = blockIdx.x;
+    if (o >= *n_out) return;
+    const int f = find_event(frame_off, Tn, o);
+    const int w = o - frame_off[f];
+    const int s = frame_stride[f];
+    const int go = (G + s - 1) / s;
+    const int r0 = (w / go) * s, r1 = min(G, r0 + s);
+    const int c0 = (w % go) * s, c1 = min(G, c0 + s);
+    const int wc = c1 - c0, cells = (r1 - r0) * wc;
+    const int tid = threadIdx.x;
+    const int nchunk = d / VN;
+    const size_t frame_base = (size_t)f * N;
+    auto cell_token = [&](int i) { return frame_base + (size_t)(r0 + i / wc) * G + (c0 + i % wc); };
+    for (int cb = 0; cb < nchunk; cb += kPoolThreads * kPoolChunks) {
+        float acc[kPoolChunks][VN];
+#pragma unroll
+        for (int u = 0; u < kPoolChunks; ++u) Vec16<T>::zero(acc[u]);
+        int i = 0;
+        for (; i + 1 < cells; i += 2) {
+            const T* x0 = feats + cell_token(i) * d;
+            const T* x1 = feats + cell_token(i + 1) * d;
+            float v0[kPoolChunks][VN], v1[kPoolChunks][VN];
+#pragma unroll
+            for (int u = 0; u < kPoolChunks; ++u) {
+                const int ch = cb + u * kPoolThreads + tid;
+                if (ch < nchunk) {
+                    Vec16<T>::load(x0 + (size_t)ch * VN, v0[u]);
+                    Vec16<T>::load(x1 + (size_t)ch * VN, v1[u]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kPoolChunks; ++u) {
+                const int ch = cb + u * kPoolThreads + tid;
+                if (ch < nchunk) {
+#pragma unroll
+                    for (int q = 0; q < VN; ++q) acc[u][q] = (acc[u][q] + v0[u][q]) + v1[u][q];
+                }
+            }
+        }
+        if (i < cells) {
+            const T* x0 = feats + cell_token(i) * d;
+#pragma unroll
+            for (int u = 0; u < kPoolChunks; ++u) {
+                const int ch = cb + u * kPoolThreads + tid;
+                if (ch < nchunk) {
+                    float v0[VN];
+                    Vec16<T>::load(x0 + (size_t)ch * VN, v0);
+#pragma unroll
+                    for (int q = 0; q < VN; ++q) acc[u][q] += v0[q];
+                }
+            }
+        }
+        const float inv = 1.0f / (float)cells;
+#pragma unroll
+        for (int u = 0; u < kPoolChunks; ++u) {
+            const int ch = cb + u * kPoolThreads + tid;
+            if (ch < nchunk) {
+                T* dst = out_feats + (size_t)o * d + (size_t)ch * VN;
+                alignas(16) T tmp[VN];
+#pragma unroll
+                for (int q = 0; q < VN; ++q) from_float(tmp[q], acc[u][q] * inv);
+                *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(tmp);
+            }
+        }
+    }
+    for (int i = tid; i < cells; i += kPoolThreads) assign[cell_token(i)] = o;
+    if (tid == 0) {
+        out_src[o] = (int32_t)cell_token(0);
+        out_event[o] = frame_ev[f];
+        out_members[o] = cells;
     }
 }
 
@@ -238,14 +395,6 @@ event_topk_kernel(const float* __restrict__ token_score, const int32_t* __restri
 // --------------------------------------------------------------------------- //
 constexpr int kMergeTM = 64, kMergeTN = 64, kMergeTK = 32;
 
-__device__ __forceinline__ int find_event(const int32_t* __restrict__ off, int k, int t) {
-    int lo = 0, hi = k;                     // off[lo] <= t < off[hi]
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (off[mid] <= t) lo = mid; else hi = mid;
-    }
-    return lo;
-}
 
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -693,6 +842,7 @@ struct VisionWs {
     float* inv_norm;
     uint8_t* is_key;
     int32_t *ev_lo, *ev_budget, *ev_out_off, *ev_tile_off, *ev_unit_off;
+    int32_t *frame_ev, *frame_stride, *frame_off;   // POOL mode
     unsigned long long* best64;   // packed argmax per token (tensor-core path)
 };
 
@@ -707,6 +857,9 @@ static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, b
     w.ev_out_off = cv.take<int32_t>((size_t)k + 1);
     w.ev_tile_off = cv.take<int32_t>((size_t)k + 1);
     w.ev_unit_off = cv.take<int32_t>((size_t)k + 1);
+    w.frame_ev = cv.take<int32_t>((size_t)Tn);
+    w.frame_stride = cv.take<int32_t>((size_t)Tn);
+    w.frame_off = cv.take<int32_t>((size_t)Tn + 1);
     w.best64 = mma ? cv.take<unsigned long long>((size_t)Tn * N) : nullptr;
     return w;
 }
@@ -731,7 +884,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     T* out_feats = reinterpret_cast<T*>(out_feats_);
     const int Nv = Tn * N;
     constexpr bool kBf16 = sizeof(T) == 2;
-    const bool mma = kBf16 && use_mma_path(d);
+    const bool mma = kBf16 && use_mma_path(d) && p->mode == METOK_MODE_TOPK_MERGE;
     Carver cv(ws);
     VisionWs w = carve_vision(cv, Tn, N, k, d, cap, mma);
     METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
@@ -754,13 +907,28 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     pp.event_agg = p->event_agg; pp.mode = p->mode; pp.tile_rows = mma ? kMmaBM : kMergeTM;
     pp.chunk_cols = kMmaBN;
     pp.keep_key = p->keep_key; pp.keep_nonkey = p->keep_nonkey; pp.beta = p->beta;
+    pp.grid = 1;
+    while (pp.grid * pp.grid < N) ++pp.grid;
+    pp.s1 = p->s1; pp.s2 = p->s2; pp.s1_nonkey = p->s1_nonkey; pp.s2_nonkey = p->s2_nonkey;
     {
         METOK_TIMED("event_plan_kernel", st);
         event_plan_kernel<<<1, 1024, (size_t)k * sizeof(float), st>>>(token_score, frame_score, event_offsets, pp, event_score,
                                                                   event_is_key, w.ev_lo, w.ev_budget, w.ev_out_off,
-                                                                  w.ev_tile_off, w.ev_unit_off, n_out);
+                                                                  w.ev_tile_off, w.ev_unit_off, w.frame_ev,
+                                                                  w.frame_stride, w.frame_off, n_out);
     }
     METOK_LAUNCH_CHECK();
+
+    if (p->mode == METOK_MODE_POOL) {
+        {
+            METOK_TIMED("pool_kernel", st);
+            pool_kernel<T><<<cap, kPoolThreads, 0, st>>>(feats, d, N, pp.grid, Tn, w.frame_off, w.frame_stride,
+                                                     w.frame_ev, n_out, out_feats, out_src, out_event, out_members,
+                                                     assign);
+        }
+        METOK_LAUNCH_CHECK();
+        return METOK_OK;
+    }
 
     {
         // the cache is sized for the longest event there can be, the thread count for twice the mean
@@ -862,10 +1030,9 @@ extern "C" int metok_compress_vision_bound(int T, int N, int k, const metok_visi
 
 extern "C" size_t metok_compress_vision_workspace_bytes(int dtype, int T, int N, int d, int k, int cap,
                                                         const metok_vision_params* p) {
-    (void)p;
     if (T < 1 || N < 1 || k < 1 || d < 1 || cap < 0) return 0;
     Carver cv(nullptr);
-    carve_vision(cv, T, N, k, d, cap, dtype == METOK_BF16);
+    carve_vision(cv, T, N, k, d, cap, dtype == METOK_BF16 && !(p && p->mode == METOK_MODE_POOL));
     return cv.total();
 }
 
@@ -888,7 +1055,6 @@ extern "C" int metok_compress_vision(const void* feats, int dtype, int T, int N,
     if (bound < 0 || cap < bound) return METOK_ERR_INVALID_ARG;
     const int eb = dtype == METOK_F32 ? 4 : 2;
     if (((long long)d * eb) % 16 != 0 || T > 8192) return METOK_ERR_UNSUPPORTED;
-    if (p->mode == METOK_MODE_POOL) return METOK_ERR_UNSUPPORTED;
     const size_t need = metok_compress_vision_workspace_bytes(dtype, T, N, d, k, cap, p);
     if (!ws || ws_bytes < need || !aligned16(ws)) return METOK_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);

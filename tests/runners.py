@@ -118,6 +118,69 @@ def compress_case(V: np.ndarray, t: np.ndarray, offs: np.ndarray, dtype: str, al
     return rep
 
 
+def pool_case(V: np.ndarray, t: np.ndarray, offs: np.ndarray, dtype: str, alpha: float, beta: float,
+              strides: Sequence[int], event_agg: int = 0) -> Dict[str, object]:
+    """mode POOL (Algorithm 1) against the oracle's adaptive_pool.  Key frames are chosen by frame
+    score: a frame whose score is within the near-tie band of its event's cut may flip, and then the
+    layouts differ; everything the layout fixes is checked either way."""
+    T, N, d = V.shape
+    G = int(round(N ** 0.5))
+    want = O.adaptive_pool(V, t, offs, alpha, beta, strides, dtype, event_agg)
+    p = B.vision_params(alpha, event_agg=event_agg, mode=B.MODE_POOL, beta=beta, s1=strides[0], s2=strides[1],
+                        s1_nonkey=strides[2], s2_nonkey=strides[3])
+    got = B.metok_compress_vision(P.to_torch(V, dtype), torch.from_numpy(np.asarray(offs, dtype=np.int32)).cuda(),
+                                  P.to_torch(t, dtype), p)
+    torch.cuda.synchronize()
+    rep: Dict[str, object] = {}
+    P.check_scores(got["frame_score"].cpu().numpy(), want["frame_score"], dtype, "frame_score")
+    assert np.array_equal(got["event_is_key"].cpu().numpy(), want["event_is_key"])
+    n_out = int(got["n_out"].item())
+    src = got["out_src"][:n_out].cpu().numpy()
+    members = got["out_members"][:n_out].cpu().numpy()
+    event = got["out_event"][:n_out].cpu().numpy()
+    assign = got["assign"].cpu().numpy()
+    # layout implied by the outputs themselves: frames in order, windows row-major, every token in one window
+    assert np.all(np.diff(src) > 0) and members.min() >= 1 and int(members.sum()) == T * N
+    assert np.array_equal(np.bincount(assign, minlength=n_out), members)
+    assert np.array_equal(assign[src], np.arange(n_out))
+    frame_of = src // N
+    assert np.array_equal(event, np.searchsorted(offs, frame_of, side="right") - 1)
+    # the stride a frame was pooled with shows in its first window (min(stride, G)^2 cells); strides
+    # beyond the grid side all give the one window of the whole frame
+    first = np.searchsorted(frame_of, np.arange(T), side="left")
+    got_stride = np.rint(np.sqrt(members[first])).astype(np.int32)
+    assert np.array_equal(got_stride ** 2, members[first])
+    want_stride = np.minimum(want["frame_stride"], G)
+    per_frame = np.bincount(frame_of, minlength=T)
+    assert np.array_equal(per_frame, (-(-G // got_stride)) ** 2)
+    flips = np.nonzero(got_stride != want_stride)[0]
+    rep["stride_flips"] = int(flips.size)
+    if flips.size:
+        fs = want["frame_score"]
+        for f in flips:
+            e = int(np.searchsorted(offs, f, side="right") - 1)
+            seg = fs[int(offs[e]):int(offs[e + 1])]
+            nk = int(want["frame_is_key"][int(offs[e]):int(offs[e + 1])].sum())
+            tau = np.sort(seg)[::-1][nk - 1]
+            assert abs(fs[f] - tau) < O.NEAR_TIE * max(float(np.max(np.abs(seg))), 1e-300), f"frame {f} flipped outside the near-tie band"
+        return rep
+    assert n_out == want["n_out"]
+    assert np.array_equal(frame_of, want["out_frame"])
+    err = P.row_rel_l2(P.to_np(got["out_feats"][:n_out]), want["out_feats"])
+    assert float(err.max()) <= P.TOL[dtype], f"pooled feature error {float(err.max()):.3e}"
+    rep["feature_err"] = float(err.max())
+    rep["n_out"] = n_out
+    # a window's members: spot-check against the grid arithmetic
+    for o in np.linspace(0, n_out - 1, num=min(n_out, 50)).astype(int):
+        f = int(frame_of[o]); s_ = int(got_stride[f]); go = -(-G // s_)
+        w = o - int(np.searchsorted(frame_of, f, side="left"))
+        r0, c0 = (w // go) * s_, (w % go) * s_
+        cells = [f * N + r * G + c for r in range(r0, min(G, r0 + s_)) for c in range(c0, min(G, c0 + s_))]
+        assert src[o] == cells[0] and members[o] == len(cells)
+        assert np.all(assign[cells] == o)
+    return rep
+
+
 def prefill_case(Q: np.ndarray, K: np.ndarray, dtype: str, vis_start: int, n_vis: int, groups: np.ndarray,
                  budgets: Sequence[int], scale: float, hidden: Optional[torch.Tensor] = None) -> Dict[str, object]:
     """`hidden` is a device tensor [S, D] (hash payload) or None."""

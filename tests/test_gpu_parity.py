@@ -133,6 +133,33 @@ def test_compress_vision_identity_is_bit_exact_and_repeatable():
             assert torch.equal(a[key], b[key]), key
 
 
+# ------------------------------------------------ Algorithm 1 pooling ------ #
+
+@pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128d1024"])
+def test_compress_vision_pool_workloads(name):
+    cfg = W.CONFIGS[name]
+    vis = vis_of(name)
+    rep = R.pool_case(vis["V"], vis["t"], vis["event_offsets"], cfg.dtype, cfg.alpha, 0.45, (2, 3, 4, 6))
+    print(name, rep)
+    assert rep["stride_flips"] == 0
+
+
+@pytest.mark.parametrize("T,G,d,offs,dtype,beta,strides,agg", [
+    (5, 3, 8, [0, 2, 5], "bf16", 0.5, (1, 2, 2, 3), 0),
+    (9, 5, 72, [0, 1, 4, 9], "f32", 0.3, (2, 3, 4, 5), 1),
+    (7, 7, 136, [0, 7], "bf16", 1.0, (3, 3, 7, 8), 0),             # one event; a stride beyond the grid
+    (6, 4, 1032, [0, 3, 6], "bf16", 0.01, (1, 1, 1, 1), 0),        # stride 1 everywhere: identity
+])
+def test_compress_vision_pool_ragged(T, G, d, offs, dtype, beta, strides, agg):
+    rng = np.random.default_rng(T * 10 + G)
+    N = G * G
+    V = W.quantize(rng.standard_normal((T, N, d)).astype(np.float32), dtype)
+    t = W.quantize(rng.standard_normal(d).astype(np.float32), dtype)
+    rep = R.pool_case(V, t, np.array(offs, dtype=np.int32), dtype, 0.5, beta, strides, agg)
+    if strides == (1, 1, 1, 1):
+        assert rep["n_out"] == T * N and rep["feature_err"] == 0.0
+
+
 # ------------------------------------------------------------- a5 a6 a7 ---- #
 
 def _prefill_stage_inputs(cfg, stage, vis):

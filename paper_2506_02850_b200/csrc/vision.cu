@@ -699,22 +699,31 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
 // segments; in a segment every thread takes a contiguous run of entries (16-byte loads,
 // all issued before the first is looked at), the matches are packed in token order by
 // one block-wide scan, and the member rows are then added in that order (so the
-// summation order is fixed), two rows in flight per thread.  fp32 sum, one division,
-// one rounding.
+// summation order is fixed).  The rows come in by bulk copies into shared memory, up to
+// kAvgStages rows at once (usually all members of an output), so that the bytes in
+// flight do not depend on registers.  fp32 sum, one division, one rounding.
 // --------------------------------------------------------------------------- //
 constexpr int kAvgThreads = 128;
 constexpr int kAvgChunks = 4;      // 16-byte chunks per thread per pass over d
 constexpr int kAvgQuads = 5;       // 16-byte groups of `assign` per thread and segment
-constexpr int kAvgSeg = kAvgThreads * kAvgQuads * 4;   // tokens per segment
+constexpr int kAvgStages = 4;      // member rows in flight
+constexpr int kAvgList = 512;      // members listed at a time
+constexpr int kAvgStageBytes = kAvgThreads * kAvgChunks * 16;
+constexpr size_t kAvgSmemBytes = (size_t)kAvgStages * kAvgStageBytes + 128;
 
 template <typename T>
 __global__ void __launch_bounds__(kAvgThreads)
 merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
                  const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
-                 const int32_t* __restrict__ n_out, T* __restrict__ out_feats, int32_t* __restrict__ out_members) {
+                 const int32_t* __restrict__ n_out, T* __restrict__ out_feats, int32_t* __restrict__ out_members,
+                 int32_t* __restrict__ status) {
+    using namespace sm100;
     constexpr int VN = Vec16<T>::N;
-    __shared__ int s_list[kAvgSeg];
+    extern __shared__ uint8_t avg_dyn[];
+    __shared__ __align__(8) uint64_t s_bar[kAvgStages];
+    __shared__ int s_list[kAvgList];
     __shared__ int s_wtot[kAvgThreads / 32];
+    __shared__ int s_abort;
     // CTAs start in index order: take the outputs from the last one down, so that this pass
     // begins with the rows of V that the preceding (ascending) pass left in L2
     const int c = *n_out - 1 - (int)blockIdx.x;
@@ -725,7 +734,17 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
     const int nchunk = d / VN;
     const int4* assign4 = reinterpret_cast<const int4*>(assign);
     const int q_lo = lo >> 2, q_hi = (hi + 3) >> 2;            // groups of four tokens that touch [lo, hi)
+    const uint32_t stage0 = (smem_u32(avg_dyn) + 127u) & ~127u;
+    if (tid == 0) {
+        for (int j = 0; j < kAvgStages; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
+        s_abort = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    volatile int* abort_flag = &s_abort;
+    uint32_t phase = 0;                                        // bit j: parity of the next completion of barrier j
     for (int cb = 0; cb < nchunk; cb += kAvgThreads * kAvgChunks) {
+        const uint32_t seg_bytes = (uint32_t)min(kAvgThreads * kAvgChunks, nchunk - cb) * 16u;
         float acc[kAvgChunks][VN];
 #pragma unroll
         for (int u = 0; u < kAvgChunks; ++u) Vec16<T>::zero(acc[u]);
@@ -773,49 +792,62 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
                 if (w < warp) before += v;
                 total += v;
             }
-            while (match) {
-                const int b = __ffs(match) - 1;
-                match &= match - 1;
-                s_list[before++] = q0 * 4 + b;
-            }
-            __syncthreads();
-            int m = 0;
-            for (; m + 1 < total; m += 2) {                    // two member rows in flight
-                const T* x0 = feats + (size_t)s_list[m] * d;
-                const T* x1 = feats + (size_t)s_list[m + 1] * d;
-                float v0[kAvgChunks][VN], v1[kAvgChunks][VN];
-#pragma unroll
-                for (int u = 0; u < kAvgChunks; ++u) {
-                    const int ch = cb + u * kAvgThreads + tid;
-                    if (ch < nchunk) {
-                        Vec16<T>::load(x0 + (size_t)ch * VN, v0[u]);
-                        Vec16<T>::load(x1 + (size_t)ch * VN, v1[u]);
+            // the members are listed kAvgList at a time (one batch covers all but pathological cases)
+            for (int b0 = 0; b0 < total; b0 += kAvgList) {
+                {
+                    unsigned mm = match;
+                    int r = before;
+                    while (mm) {
+                        const int b = __ffs(mm) - 1;
+                        mm &= mm - 1;
+                        if (r >= b0 && r < b0 + kAvgList) s_list[r - b0] = q0 * 4 + b;
+                        ++r;
                     }
                 }
-#pragma unroll
-                for (int u = 0; u < kAvgChunks; ++u) {
-                    const int ch = cb + u * kAvgThreads + tid;
-                    if (ch < nchunk) {
-#pragma unroll
-                        for (int q = 0; q < VN; ++q) acc[u][q] = (acc[u][q] + v0[u][q]) + v1[u][q];
+                __syncthreads();
+                const int nlist = min(kAvgList, total - b0);
+                for (int m0 = 0; m0 < nlist; m0 += kAvgStages) {
+                    const int nr = min(kAvgStages, nlist - m0);
+                    if (tid == 0) {
+                        for (int j = 0; j < nr; ++j) {
+                            const uint32_t bar = smem_u32(&s_bar[j]);
+                            mbar_arrive_expect_tx(bar, seg_bytes);
+                            bulk_load(stage0 + (uint32_t)j * kAvgStageBytes,
+                                      feats + (size_t)s_list[m0 + j] * d + (size_t)cb * VN, seg_bytes, bar);
+                        }
                     }
-                }
-            }
-            if (m < total) {
-                const T* x0 = feats + (size_t)s_list[m] * d;
-#pragma unroll
-                for (int u = 0; u < kAvgChunks; ++u) {
-                    const int ch = cb + u * kAvgThreads + tid;
-                    if (ch < nchunk) {
-                        float v0[VN];
-                        Vec16<T>::load(x0 + (size_t)ch * VN, v0);
-#pragma unroll
-                        for (int q = 0; q < VN; ++q) acc[u][q] += v0[q];
+                    for (int j = 0; j < nr; ++j) {
+                        const bool ok = mbar_wait(smem_u32(&s_bar[j]), (phase >> j) & 1u, abort_flag);
+                        phase ^= 1u << j;
+                        if (!ok) continue;
+                        const uint8_t* row = avg_dyn + (stage0 - smem_u32(avg_dyn)) + (size_t)j * kAvgStageBytes;
+    #pragma unroll
+                        for (int u = 0; u < kAvgChunks; ++u) {
+                            const int ch = cb + u * kAvgThreads + tid;
+                            if (ch < nchunk) {
+                                const uint4 raw = *reinterpret_cast<const uint4*>(row + (size_t)(u * kAvgThreads + tid) * 16);
+                                float v[VN];
+                                if constexpr (sizeof(T) == 4) {
+                                    v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
+                                    v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+                                } else {
+                                    const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
+    #pragma unroll
+                                    for (int i = 0; i < 4; ++i) {
+                                        v[2 * i]     = __uint_as_float(w4[i] << 16);
+                                        v[2 * i + 1] = __uint_as_float(w4[i] & 0xFFFF0000u);
+                                    }
+                                }
+    #pragma unroll
+                                for (int q = 0; q < VN; ++q) acc[u][q] += v[q];
+                            }
+                        }
                     }
+                    __syncthreads();                               // every thread is done with the stages
                 }
             }
             count += total;
-            __syncthreads();
+            __syncthreads();                                   // s_wtot and s_list are reused by the next segment
         }
         const float inv = 1.0f / (float)count;
 #pragma unroll
@@ -831,6 +863,7 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
         }
         if (tid == 0 && cb == 0) out_members[c] = count;
     }
+    if (tid == 0 && s_abort) *status = METOK_ERR_TIMEOUT;
 }
 
 // --------------------------------------------------------------------------- //
@@ -981,10 +1014,12 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         METOK_LAUNCH_CHECK();
     }
 
+    METOK_CUDA_TRY(cudaFuncSetAttribute(merge_avg_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)kAvgSmemBytes));
     {
         METOK_TIMED("merge_avg_kernel", st);
-        merge_avg_kernel<T><<<cap, kAvgThreads, 0, st>>>(feats, d, N, Nv, w.ev_lo, out_event, assign, n_out,
-                                                     out_feats, out_members);
+        merge_avg_kernel<T><<<cap, kAvgThreads, kAvgSmemBytes, st>>>(feats, d, N, Nv, w.ev_lo, out_event, assign, n_out,
+                                                                 out_feats, out_members, w.status);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;

@@ -21,6 +21,11 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
 int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
                        const char* timer_name, cudaStream_t st);
 
+// The same gather by bulk copies through shared memory (rows of any multiple of 16 bytes).
+// `status` receives METOK_ERR_TIMEOUT if a device-side wait gave up.
+int launch_gather_rows_bulk(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, size_t row_bytes,
+                            int32_t* status, const char* timer_name, cudaStream_t st);
+
 // Text->visual attention scores on the tensor cores (bf16, dh 64 or 128): leaves
 // n_planes partial column sums of n_vis floats each in part_col; their sum divided by
 // Hq*Lt is the score.  attn_mma_workspace gives the element counts of part_m / part_l

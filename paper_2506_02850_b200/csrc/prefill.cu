@@ -5,6 +5,7 @@
 #include "common.cuh"
 #include "select.cuh"
 #include "launchers.h"
+#include "sm100.cuh"
 
 namespace metok {
 
@@ -335,6 +336,81 @@ gather_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const
     }
 }
 
+// The same gather driven by the copy engine: one thread per CTA moves (row, 8 KiB segment)
+// items global -> shared -> global with bulk copies, kGbStages items in flight; no registers
+// or warps are spent on the data.
+constexpr int kGbStages = 4;
+constexpr uint32_t kGbSegBytes = 8192;
+constexpr size_t kGbSmemBytes = (size_t)kGbStages * kGbSegBytes + 128;
+
+__global__ void __launch_bounds__(32)
+gather_rows_bulk_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
+                        const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ n_rows,
+                        uint32_t row_bytes, int32_t* __restrict__ status) {
+    using namespace sm100;
+    extern __shared__ uint8_t gb_dyn[];
+    __shared__ __align__(8) uint64_t s_bar[kGbStages];
+    __shared__ int s_abort;
+    if (threadIdx.x != 0) return;
+    const uint32_t stage0 = (smem_u32(gb_dyn) + 127u) & ~127u;
+    for (int j = 0; j < kGbStages; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
+    s_abort = 0;
+    mbar_fence_init();
+    const int nseg = (int)((row_bytes + kGbSegBytes - 1) / kGbSegBytes);
+    const long long items = (long long)(*n_rows) * nseg;
+    const long long first = blockIdx.x, stride = gridDim.x;
+    const long long mine = first < items ? (items - first + stride - 1) / stride : 0;   // items of this CTA
+    auto issue_load = [&](long long k) {
+        const long long it = first + k * stride;
+        const int i = (int)(it / nseg), sg = (int)(it - (long long)i * nseg);
+        const uint32_t off = (uint32_t)sg * kGbSegBytes;
+        const uint32_t bytes = min(kGbSegBytes, row_bytes - off);
+        const uint32_t bar = smem_u32(&s_bar[k % kGbStages]);
+        mbar_arrive_expect_tx(bar, bytes);
+        bulk_load(stage0 + (uint32_t)(k % kGbStages) * kGbSegBytes, src + (size_t)keep_idx[i] * row_bytes + off, bytes,
+                  bar);
+    };
+    volatile int* abort_flag = &s_abort;
+    for (long long k = 0; k < mine && k < kGbStages; ++k) issue_load(k);
+    bool ok = true;
+    for (long long k = 0; k < mine; ++k) {
+        const int s = (int)(k % kGbStages);
+        if (!mbar_wait(smem_u32(&s_bar[s]), (uint32_t)(k / kGbStages) & 1u, abort_flag)) { ok = false; break; }
+        const long long it = first + k * stride;
+        const int i = (int)(it / nseg), sg = (int)(it - (long long)i * nseg);
+        const uint32_t off = (uint32_t)sg * kGbSegBytes;
+        const uint32_t bytes = min(kGbSegBytes, row_bytes - off);
+        fence_proxy_async();
+        bulk_store(dst + (size_t)i * row_bytes + off, stage0 + (uint32_t)s * kGbSegBytes, bytes);
+        bulk_commit();
+        // the stage of the item before this one is free once its store has read it
+        if (k >= 1 && k - 1 + kGbStages < mine) {
+            bulk_wait_read<1>();
+            issue_load(k - 1 + kGbStages);
+        }
+    }
+    bulk_wait_all();
+    if (!ok) {
+        // loads still in flight must land before the shared memory goes away
+        for (int j = 0; j < kGbStages; ++j) mbar_wait(smem_u32(&s_bar[j]), 0u, abort_flag);
+        *status = METOK_ERR_TIMEOUT;
+    }
+}
+
+int launch_gather_rows_bulk(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, size_t row_bytes,
+                            int32_t* status, const char* timer_name, cudaStream_t st) {
+    METOK_CUDA_TRY(cudaFuncSetAttribute(gather_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)kGbSmemBytes));
+    {
+        METOK_TIMED(timer_name, st);
+        gather_rows_bulk_kernel<<<kNumSMs * 6, 32, kGbSmemBytes, st>>>(
+            reinterpret_cast<const uint8_t*>(src), reinterpret_cast<uint8_t*>(dst), idx, n_rows, (uint32_t)row_bytes,
+            status);
+    }
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
+}
+
 int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
                        const char* timer_name, cudaStream_t st) {
     {
@@ -482,14 +558,9 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
                            nullptr, 1, st);
     if (rc != METOK_OK) return rc;
     if (hidden) {
-        const int row_chunks = (int)((long long)D * eb / 16);
-        {
-            METOK_TIMED("gather_rows_kernel", st);
-            gather_rows_kernel<<<kNumSMs * 8, kGatherThreads, 0, st>>>(reinterpret_cast<const uint4*>(hidden),
-                                                        reinterpret_cast<uint4*>(hidden_out), keep_idx, S_out,
-                                                        row_chunks);
-        }
-        METOK_LAUNCH_CHECK();
+        rc = launch_gather_rows_bulk(hidden, hidden_out, keep_idx, S_out, (size_t)D * eb, w.status, "gather_rows_kernel",
+                                     st);
+        if (rc != METOK_OK) return rc;
     }
     return METOK_OK;
 }

@@ -159,17 +159,23 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
     __shared__ int s_scan[1024];
     const int tid = threadIdx.x, nthr = blockDim.x;
 
-    // a warp per frame: lanes take the slabs 32 apart, then a fixed shuffle tree
-    const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
-    for (int f = warp; f < Tn; f += nwarps) {
+    // eight lanes per frame: a lane takes the slabs 8 apart (all its loads are independent), then a
+    // fixed shuffle tree over the eight; 128 frames per sweep of the CTA
+    for (int f0 = 0; f0 < Tn; f0 += nthr >> 3) {
+        const int f = f0 + (tid >> 3), part = tid & 7;
         float a = 0.f, b = 0.f;
-        for (int s = lane; s < nslab; s += 32) {
-            a += part_nrm[(size_t)s * Tn + f];
-            if (f < Tn - 1) b += part_dot[(size_t)s * Tn + f];
+        if (f < Tn) {
+            for (int s = part; s < nslab; s += 8) {
+                a += part_nrm[(size_t)s * Tn + f];
+                if (f < Tn - 1) b += part_dot[(size_t)s * Tn + f];
+            }
         }
-        a = warp_sum(a);
-        b = warp_sum(b);
-        if (lane == 0) {
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) {
+            a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+            b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
+        }
+        if (f < Tn && part == 0) {
             s_nrm[f] = fmaxf(sqrtf(a), kEps);
             s_sim[f] = b;                                   // dot product for now
         }

@@ -126,12 +126,20 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
     __shared__ int s_scan[1024];
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int k = pp.k, Tn = pp.Tn;
-    // frame_score[f] = mean of the frame's N token scores; one warp per frame, fixed order
-    for (int f = tid >> 5; f < Tn; f += nthr >> 5) {
+    // frame_score[f] = mean of the frame's N token scores; eight lanes per frame (a lane's loads are
+    // independent), fixed shuffle tree; the scores stay in shared memory for the event loops below
+    float* s_frame = s_score + k;           // [Tn]
+    for (int f0 = 0; f0 < Tn; f0 += nthr >> 3) {
+        const int f = f0 + (tid >> 3), part = tid & 7;
         float s = 0.f;
-        for (int p = tid & 31; p < pp.N; p += 32) s += token_score[(size_t)f * pp.N + p];
-        s = warp_sum(s);
-        if ((tid & 31) == 0) frame_score[f] = s / (float)pp.N;
+        if (f < Tn)
+            for (int p = part; p < pp.N; p += 8) s += token_score[(size_t)f * pp.N + p];
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        if (f < Tn && part == 0) {
+            s_frame[f] = s / (float)pp.N;
+            frame_score[f] = s_frame[f];
+        }
     }
     __syncthreads();
     for (int e = tid; e < k; e += nthr) {
@@ -144,11 +152,11 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
             s = -3.0e38f;
         } else if (pp.event_agg == METOK_AGG_MEAN) {
             float a = 0.f;
-            for (int f = lo; f < hi; ++f) a += frame_score[f];
+            for (int f = lo; f < hi; ++f) a += s_frame[f];
             s = a / (float)(hi - lo);
         } else {
-            float a = frame_score[lo];
-            for (int f = lo + 1; f < hi; ++f) a = fmaxf(a, frame_score[f]);
+            float a = s_frame[lo];
+            for (int f = lo + 1; f < hi; ++f) a = fmaxf(a, s_frame[f]);
             s = a;
         }
         s_score[e] = s;
@@ -219,10 +227,10 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
             if ((double)nk < c) nk += 1;
             if (nk < 1) nk = 1;
             if (nk > len) nk = len;
-            const float v = frame_score[f];
+            const float v = s_frame[f];
             int rank = 0;
             for (int j = lo; j < hi; ++j) {
-                const float w = frame_score[j];
+                const float w = s_frame[j];
                 rank += (w > v) || (w == v && j < f);
             }
             const bool key_frame = rank < (int)nk;
@@ -943,9 +951,12 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     pp.grid = 1;
     while (pp.grid * pp.grid < N) ++pp.grid;
     pp.s1 = p->s1; pp.s2 = p->s2; pp.s1_nonkey = p->s1_nonkey; pp.s2_nonkey = p->s2_nonkey;
+    if ((size_t)(k + Tn) * sizeof(float) > 40 * 1024)
+        METOK_CUDA_TRY(cudaFuncSetAttribute(event_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)((size_t)(k + Tn) * sizeof(float))));
     {
         METOK_TIMED("event_plan_kernel", st);
-        event_plan_kernel<<<1, 1024, (size_t)k * sizeof(float), st>>>(token_score, frame_score, event_offsets, pp, event_score,
+        event_plan_kernel<<<1, 1024, (size_t)(k + Tn) * sizeof(float), st>>>(token_score, frame_score, event_offsets, pp, event_score,
                                                                   event_is_key, w.ev_lo, w.ev_budget, w.ev_out_off,
                                                                   w.ev_tile_off, w.ev_unit_off, w.frame_ev,
                                                                   w.frame_stride, w.frame_off, n_out);

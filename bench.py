@@ -39,7 +39,16 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu
 # captures (profiles/), keyed by (kernel, workload); absent -> null in the JSON line.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/kernel_sections_frames128.txt; averages over a step's launches of the kernel
+    ("class_topk_kernel", "frames128"): 0.17e6,
+    ("merge_assign_mma_kernel", "frames128"): 163.9e6,
+    ("seg_partial_kernel", "frames128"): 139.1e6,
+    ("tok_score_kernel", "frames128"): 135.7e6,
+    ("kv_copy_kernel", "frames128"): 100.3e6,
+    ("attn_stats_mma_kernel", "frames128"): 9.9e6,
+    ("attn_colsum_mma_kernel", "frames128"): 10.1e6,
+}
 
 
 def load_peaks():
@@ -362,6 +371,20 @@ def time_oracle(cfg, steps, warmup):
 # --------------------------------------------------------------------------- #
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The slowest rank's time: replicas finish together only when the last one does."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(tokens_per_replica: int, world: int, ms_per_step: float) -> float:
+    """Whole-job tokens/s of `world` independent replicas that each finish a step in ms_per_step."""
+    return world * tokens_per_replica / (ms_per_step * 1e-3)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -439,12 +462,7 @@ def main():
         host_ms[fn.__name__] = (time.perf_counter() - t0) * 1e3 / steps     # time to enqueue one step
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            tms = torch.tensor([ms], device=dev)
-            dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-            ms = float(tms.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dist, dev)
 
     # eager: every step issues its C-ABI calls from Python
     eager_ms_per_step = timed(wl.step, args.steps) / args.steps
@@ -463,7 +481,7 @@ def main():
     total_ms = timed(step_graph if graph is not None else wl.step, args.steps)
     clocks = sampler.stop()
     ms_per_step = total_ms / args.steps
-    value = world * cfg.Nv / (ms_per_step * 1e-3)
+    value = replica_throughput(cfg.Nv, world, ms_per_step)
 
     # per-kernel times: the same K steps again with the library's event brackets on
     barrier()
@@ -504,7 +522,7 @@ def main():
         h2d, d2h = wl.e2e_alloc()
         e2e_steps = max(3, min(args.steps, 10))
         ms = timed(wl.e2e_step, e2e_steps) / e2e_steps
-        e2e = {"value": world * cfg.Nv / (ms * 1e-3), "unit": "tokens/s", "ms_per_step": ms,
+        e2e = {"value": replica_throughput(cfg.Nv, world, ms), "unit": "tokens/s", "ms_per_step": ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps}
 
     cpu = None

@@ -1,8 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the METok hot path on B200.
 
-A "step" is one pass of the whole hot path over one synthetic video of the
-128-frame workload (128 x 144 visual tokens, 28-layer 7B-shaped LLM): event
+A "step" is one pass of the whole hot path over a batch of independent synthetic
+videos of the 128-frame workload (128 x 144 visual tokens, 28-layer 7B-shaped LLM;
+4 videos in flight by default, each on a stream of its own): event
 segmentation, stage-1 compression, the three prefill pruning levels at the
 sizes the Eq. 6/7 schedule implies, and the KV-cache compaction -- all through
 the C ABI.  `value` = visual tokens entering the path per second, inputs resident
@@ -130,6 +131,19 @@ class Workload:
         self.out = {}
         self.side = None
         self.scale = float(cfg.dh ** -0.5)
+
+    def twin(self):
+        """A second, independent video: the same values in buffers of its own (nothing is shared,
+        so it competes for L2 and HBM like any other video would)."""
+        import copy
+        w = copy.copy(self)
+        w.V, w.t = self.V.clone(), self.t.clone()
+        w.planted_offsets = self.planted_offsets.clone()
+        w.stages = [{k_: (v.clone() if isinstance(v, torch.Tensor) else v) for k_, v in s.items()} for s in self.stages]
+        w.ks, w.vs = [x.clone() for x in self.ks], [x.clone() for x in self.vs]
+        w.kv_scores = self.kv_scores.clone()
+        w.out, w.side, w.h = {}, None, {}
+        return w
 
     # one pass of the hot path, device-resident inputs
     def step(self):
@@ -395,6 +409,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph of the step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--videos", type=int, default=4,
+                    help="independent videos in flight per step, each on a stream of its own (a step = this batch)")
     ap.add_argument("--parts", default=",".join(PARTS),
                     help="comma-separated subset of the four calls (for profiler captures that should hold little "
                          "memory); anything but the full list is not a benchmark result")
@@ -441,7 +457,22 @@ def main():
     if partial:
         args.no_e2e = True
     wl = Workload(cfg, dev, host_copies=not args.no_e2e, parts=parts)
+    n_videos = max(1, args.videos)
+    wls = [wl] + [wl.twin() for _ in range(n_videos - 1)]
+    lanes = [torch.cuda.Stream() for _ in range(n_videos - 1)]
     warm = max(args.warmup, 3)
+
+    def batch_step():
+        """All videos of the batch, each on its own stream, joined at the end."""
+        main = torch.cuda.current_stream()
+        for st in lanes:
+            st.wait_stream(main)
+        wls[0].step()
+        for w, st in zip(wls[1:], lanes):
+            with torch.cuda.stream(st):
+                w.step()
+        for st in lanes:
+            main.wait_stream(st)
 
     def barrier():
         if dist is not None:
@@ -465,23 +496,31 @@ def main():
         return max_over_ranks(e0.elapsed_time(e1), dist, dev)
 
     # eager: every step issues its C-ABI calls from Python
-    eager_ms_per_step = timed(wl.step, args.steps) / args.steps
+    eager_ms_per_step = timed(batch_step, args.steps) / args.steps
     # the same calls captured once in a CUDA graph and replayed: the calls enqueue on a stream
     # and never synchronise, so one capture of a step holds all of its launches
-    graph = None
+    graph = graph_one = None
     if not args.no_graph:
+        graph_one = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_one):
+            wl.step()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            wl.step()
+            batch_step()
 
         def step_graph():
             graph.replay()
+
+        def step_graph_one():
+            graph_one.replay()
+    # latency of one video alone on the GPU
+    ms_one_video = timed(step_graph_one if graph_one is not None else wl.step, args.steps) / args.steps
     sampler = ClockSampler(local)
     sampler.start()
-    total_ms = timed(step_graph if graph is not None else wl.step, args.steps)
+    total_ms = timed(step_graph if graph is not None else batch_step, args.steps)
     clocks = sampler.stop()
     ms_per_step = total_ms / args.steps
-    value = replica_throughput(cfg.Nv, world, ms_per_step)
+    value = replica_throughput(cfg.Nv * n_videos, world, ms_per_step)
 
     # per-kernel times: the same K steps again with the library's event brackets on
     barrier()
@@ -536,9 +575,10 @@ def main():
                 "steps": args.steps, "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
                 "config": {"workload": workload_name, "l2": "inputs larger than L2 (V 132 MB, hidden 133 MB, K/V 1.06 GB touched between reuses)",
-                           "parallelism": f"replicas x{world}"},
+                           "videos_in_flight": n_videos, "parallelism": f"replicas x{world}"},
+                "single_video": {"ms_per_video": ms_one_video, "tokens_per_s": replica_throughput(cfg.Nv, world, ms_one_video)},
                 "launch": "cuda_graph" if graph is not None else "eager", "eager_ms_per_step": eager_ms_per_step,
-                "host_enqueue_ms_per_step": host_ms.get("step"), "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+                "host_enqueue_ms_per_step": host_ms.get("batch_step"), "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * n_videos * args.steps,
                 "roofline": roofline, "cpu_baseline": cpu}
         if partial:
             line["partial"] = "only " + ",".join(parts) + ": not a benchmark result"

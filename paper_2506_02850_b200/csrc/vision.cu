@@ -508,26 +508,30 @@ merge_assign_simt_kernel(const T* __restrict__ feats, int d, int N, const int32_
 // --------------------------------------------------------------------------- //
 // Merge-assign on the tensor cores (bf16).
 //
-// Work unit = 128 consecutive token rows of one event (TMEM lanes) x one chunk of the
-// event's key tokens (up to 256 columns; an event's keys are cut into equal chunks).
-// The units of all events form one list; a persistent CTA per SM takes every
-// gridDim-th unit, so the load is balanced whatever the event lengths are, and with two
-// accumulators in TMEM the epilogue of a unit overlaps the main loop of the next.
-//   warp 0   : TMA producer -- per 64-wide K step one 128x64 tile of V (rows are
-//              contiguous in V) and the chunk's key rows from the compact key buffer
-//              (64-row boxes), 4-stage ring that runs on across units;
-//   warp 1   : allocates TMEM (2 accumulators x 256 columns), issues tcgen05.mma
-//              (M=128, N=16..256, K=16) and commits to the ring / accumulator barriers;
-//   warps 2-5: epilogue -- read the accumulator with tcgen05.ld, scale each column by
-//              1/|key|, take the (value, slot) argmax of the thread's row over the chunk.
+// Work unit = up to 256 consecutive token rows of one event x one chunk of the event's
+// key tokens (up to 256 columns; an event's keys are cut into equal chunks).  The two
+// 128-row halves of a unit are two accumulators in TMEM (2 x 256 columns) that share
+// every key tile brought into shared memory: the main loop is fed at a fixed rate per
+// SM, so what counts is the work done per byte loaded -- a 256 x 256 unit needs a third
+// fewer bytes per flop than a 128 x 256 one.  The units of all events form one list; a
+// persistent CTA takes every gridDim-th unit.
+//   warp 0   : TMA producer -- per 64-wide K step one 256x64 (or, for an event's last
+//              rows, 128x64) tile of V (rows are contiguous in V) and the chunk's key
+//              rows from the compact key buffer (64-row boxes), 3-stage ring that runs
+//              on across units;
+//   warp 1   : allocates TMEM, issues tcgen05.mma (M=128, N=16..256, K=16), two per K
+//              slice (one per row half), and commits to the ring / accumulator barriers;
+//   warps 2-9: epilogue, four warps per row half -- read the accumulator with
+//              tcgen05.ld, scale each column by 1/|key|, take the (value, slot) argmax of
+//              the thread's row over the chunk.
 // Chunks of one row tile may be handled by different CTAs: a row's result is combined
 // with a 64-bit atomicMax on (order-preserving key of the value) << 32 | ~slot, which
 // does not depend on the order of arrival (larger value first, then the lower slot).
 // Every wait is bounded; on a timeout the CTA unwinds and writes METOK_ERR_TIMEOUT.
 // --------------------------------------------------------------------------- //
-constexpr int kMmaBM = 128, kMmaBK = 64, kMmaBN = 256, kMmaStages = 4;
-constexpr int kMmaThreads = 192;
-constexpr uint32_t kMmaABytes = kMmaBM * kMmaBK * 2;       // 16 KiB
+constexpr int kMmaBM = 256, kMmaBK = 64, kMmaBN = 256, kMmaStages = 3;
+constexpr int kMmaThreads = 320;
+constexpr uint32_t kMmaABytes = kMmaBM * kMmaBK * 2;       // 32 KiB
 constexpr uint32_t kMmaBBytes = kMmaBN * kMmaBK * 2;       // 32 KiB
 constexpr uint32_t kMmaBoxBytes = 64 * kMmaBK * 2;         // one 64-row key box
 constexpr size_t kMmaSmemBytes = (size_t)kMmaStages * (kMmaABytes + kMmaBBytes) + 1024;
@@ -552,14 +556,15 @@ __device__ __forceinline__ MergeUnit merge_unit(int u, const int32_t* __restrict
 }
 
 __global__ void __launch_bounds__(kMmaThreads, 1)
-merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int d, int N,
+merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_half,
+                        const __grid_constant__ CUtensorMap tmB, int d, int N,
                         const int32_t* __restrict__ ev_lo, int k, const int32_t* __restrict__ ev_out_off,
                         const int32_t* __restrict__ ev_unit_off, const int32_t* __restrict__ out_src,
                         const float* __restrict__ inv_norm, const uint8_t* __restrict__ is_key,
                         unsigned long long* __restrict__ best64, int32_t* __restrict__ status) {
     using namespace sm100;
     extern __shared__ uint8_t smem_dyn[];
-    __shared__ __align__(8) uint64_t full_bar[kMmaStages], empty_bar[kMmaStages], tfull_bar[2], tempty_bar[2], drain_bar;
+    __shared__ __align__(8) uint64_t full_bar[kMmaStages], empty_bar[kMmaStages], tfull_bar, tempty_bar, drain_bar;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ float s_keyinv[2][kMmaBN];
@@ -575,7 +580,8 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tfull_bar[b]), 1); mbar_init(smem_u32(&tempty_bar[b]), 4); }
+        mbar_init(smem_u32(&tfull_bar), 1);
+        mbar_init(smem_u32(&tempty_bar), 8);
         mbar_init(smem_u32(&drain_bar), 1);
         s_abort = 0;
         mbar_fence_init();
@@ -593,19 +599,21 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (warp == 0) {
         if (lane == 0) {
             prefetch_tmap(&tmA);
+            prefetch_tmap(&tmA_half);
             prefetch_tmap(&tmB);
             int it = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
                 const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
                 const int nbox = (mu.nvalid + 63) >> 6;
+                const bool two = mu.row_end - mu.row0 > 128;           // both row halves hold rows of the event
                 for (int ks = 0; ks < ksteps; ++ks, ++it) {
                     const int s = it % kMmaStages;
                     const uint32_t ph = (uint32_t)(it / kMmaStages) & 1u;
                     if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t fb = smem_u32(&full_bar[s]);
-                    mbar_arrive_expect_tx(fb, kMmaABytes + (uint32_t)nbox * kMmaBoxBytes);
-                    tma_load_2d(a_addr(s), &tmA, ks * kMmaBK, mu.row0, fb);
+                    mbar_arrive_expect_tx(fb, (two ? kMmaABytes : kMmaABytes / 2) + (uint32_t)nbox * kMmaBoxBytes);
+                    tma_load_2d(a_addr(s), two ? &tmA : &tmA_half, ks * kMmaBK, mu.row0, fb);
                     for (int j = 0; j < nbox; ++j)
                         tma_load_2d(b_addr(s) + (uint32_t)j * kMmaBoxBytes, &tmB, ks * kMmaBK, mu.col0 + j * 64, fb);
                 }
@@ -624,11 +632,10 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             bool ok = true;
             for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++n) {
                 const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
-                const int b = n & 1;
-                if (!mbar_wait(smem_u32(&tempty_bar[b]), ((uint32_t)(n >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                const bool two = mu.row_end - mu.row0 > 128;
+                if (!mbar_wait(smem_u32(&tempty_bar), ((uint32_t)n & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t idesc = make_idesc_bf16(kMmaBM, (mu.nvalid + 15) & ~15);
-                const uint32_t d_tmem = tmem_base + (uint32_t)b * kMmaBN;
+                const uint32_t idesc = make_idesc_bf16(128, (mu.nvalid + 15) & ~15);
                 for (int ks = 0; ks < ksteps; ++ks, ++it) {
                     const int s = it % kMmaStages;
                     const uint32_t ph = (uint32_t)(it / kMmaStages) & 1u;
@@ -636,13 +643,15 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     tc_fence_after();
 #pragma unroll
                     for (int kk = 0; kk < kMmaBK / 16; ++kk) {
-                        const uint64_t ad = make_desc_k128(a_addr(s) + kk * 32);
                         const uint64_t bd = make_desc_k128(b_addr(s) + kk * 32);
-                        umma_bf16(d_tmem, ad, bd, idesc, (ks | kk) != 0 ? 1u : 0u);
+                        umma_bf16(tmem_base, make_desc_k128(a_addr(s) + kk * 32), bd, idesc, (ks | kk) != 0 ? 1u : 0u);
+                        if (two)                                     // rows 128..255 of the tile: 16 KiB further on
+                            umma_bf16(tmem_base + kMmaBN, make_desc_k128(a_addr(s) + kMmaABytes / 2 + kk * 32), bd, idesc,
+                                      (ks | kk) != 0 ? 1u : 0u);
                     }
                     umma_commit(smem_u32(&empty_bar[s]));          // frees the stage when these MMAs retire
                 }
-                if (ok) umma_commit(smem_u32(&tfull_bar[b]));      // accumulator of this unit complete
+                if (ok) umma_commit(smem_u32(&tfull_bar));         // both accumulators of this unit complete
             }
             if (!ok) {                                             // wait until whatever was issued has retired
                 umma_commit(smem_u32(&drain_bar));
@@ -651,36 +660,38 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
     } else {
         const int grp = warp & 3;                                   // TMEM lanes 32*grp .. 32*grp+31
-        const int et = (warp - 2) * 32 + lane;                      // 0..127 among the epilogue threads
+        const int half = (warp - 2) >> 2;                           // row half = accumulator
+        const int et = (warp - 2) * 32 + lane;                      // 0..255 among the epilogue threads
         bool ok = true;
         int n = 0;
         for (int u = blockIdx.x; u < total_units; u += gridDim.x, ++n) {
             const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
-            const int b = n & 1;
-            for (int i = et; i < kMmaBN; i += 128)
-                s_keyinv[b][i] = (i < mu.nvalid) ? inv_norm[out_src[mu.col0 + i]] : 0.f;
-            named_bar_sync(1, 128);
-            if (ok && !mbar_wait(smem_u32(&tfull_bar[b]), (uint32_t)(n >> 1) & 1u, abort_flag)) ok = false;
+            const int b = n & 1;                                    // s_keyinv alternates: a slow warp may still read the last one
+            s_keyinv[b][et] = (et < mu.nvalid) ? inv_norm[out_src[mu.col0 + et]] : 0.f;
+            named_bar_sync(1, 256);
+            if (ok && !mbar_wait(smem_u32(&tfull_bar), (uint32_t)n & 1u, abort_flag)) ok = false;
             ok = __all_sync(0xFFFFFFFFu, ok);                      // tcgen05.ld below is warp-collective
             if (!ok) continue;                                     // keep meeting the others at the named barrier
             tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(grp * 32) << 16) + (uint32_t)b * kMmaBN;
+            const int row = mu.row0 + half * 128 + grp * 32 + lane;
             float best_v = -3.4e38f;
             int best_c = 0;
-            for (int c0 = 0; c0 < mu.nvalid; c0 += 32) {
-                float v[32];
-                tmem_ld32(t_row + (uint32_t)c0, v);
+            if (half == 0 || mu.row_end - mu.row0 > 128) {          // the second accumulator of a short unit holds nothing
+                const uint32_t t_row = tmem_base + ((uint32_t)(grp * 32) << 16) + (uint32_t)half * kMmaBN;
+                for (int c0 = 0; c0 < mu.nvalid; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(t_row + (uint32_t)c0, v);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int col = c0 + j;
-                    const float val = v[j] * s_keyinv[b][col];
-                    if (col < mu.nvalid && val > best_v) { best_v = val; best_c = col; }
+                    for (int j = 0; j < 32; ++j) {
+                        const int col = c0 + j;
+                        const float val = v[j] * s_keyinv[b][col];
+                        if (col < mu.nvalid && val > best_v) { best_v = val; best_c = col; }
+                    }
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[b]));
-            const int row = mu.row0 + grp * 32 + lane;
+            if (lane == 0) mbar_arrive(smem_u32(&tempty_bar));
             if (row < mu.row_end && !is_key[row]) {
                 const unsigned long long packed =
                     ((unsigned long long)float_key(best_v) << 32) | (unsigned long long)(~(uint32_t)(mu.col0 + best_c));
@@ -995,7 +1006,10 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
                                           "gather_key_rows_kernel", st);
         if (rc != METOK_OK) return rc;
         CUtensorMap tmA, tmB;
+        CUtensorMap tmA_half;
         int r2 = make_tmap_bf16_2d(&tmA, feats, (uint64_t)Nv, (uint64_t)d, kMmaBM);
+        if (r2 != METOK_OK) return r2;
+        r2 = make_tmap_bf16_2d(&tmA_half, feats, (uint64_t)Nv, (uint64_t)d, kMmaBM / 2);
         if (r2 != METOK_OK) return r2;
         r2 = make_tmap_bf16_2d(&tmB, w.key_rows, (uint64_t)cap + 64, (uint64_t)d, 64);
         if (r2 != METOK_OK) return r2;
@@ -1005,7 +1019,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         {
             METOK_TIMED("merge_assign_mma_kernel", st);
             merge_assign_mma_kernel<<<kNumSMs, kMmaThreads, kMmaSmemBytes, st>>>(
-                tmA, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, w.inv_norm, w.is_key, w.best64,
+                tmA, tmA_half, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, w.inv_norm, w.is_key, w.best64,
                 w.status);
         }
         METOK_LAUNCH_CHECK();

@@ -38,6 +38,8 @@ constexpr int kStStages = 2;
 constexpr int kCsBM = 128;                // colsum: keys per tile
 constexpr int kCsMaxNQ = 256;             // colsum: query rows per chunk (multiple of 16)
 constexpr int kCsStages = 4;
+constexpr int kStMinTiles = 4;            // fewest key tiles a stats CTA is started for
+constexpr int kCsMinTiles = 6;            // the same for colsum
 
 struct AttnMmaDims {
     int Hq, Hkv, Lt, S, vis_start, n_vis, R;
@@ -54,7 +56,10 @@ __host__ AttnMmaDims make_mma_dims(int Hq, int Hkv, int Lt, int S, int vis_start
     // one CTA per SM: as many key splits as keep the grid within one wave
     dm.st_nrt = ceil_div(dm.R, kStBM);
     dm.st_tiles = ceil_div(S, kStBN);
+    // ... but a CTA gets at least kStMinTiles tiles: a launch that is mostly prologue on every SM
+    // keeps other streams' kernels off the GPU for nothing
     int ns = kNumSMs / (Hkv * dm.st_nrt);
+    if (ns > ceil_div(dm.st_tiles, kStMinTiles)) ns = ceil_div(dm.st_tiles, kStMinTiles);
     if (ns < 1) ns = 1;
     if (ns > dm.st_tiles) ns = dm.st_tiles;
     dm.st_per = ceil_div(dm.st_tiles, ns);
@@ -64,6 +69,7 @@ __host__ AttnMmaDims make_mma_dims(int Hq, int Hkv, int Lt, int S, int vis_start
     dm.cs_t0 = vis_start / kCsBM;
     dm.cs_tiles = (vis_start + n_vis - 1) / kCsBM - dm.cs_t0 + 1;
     ns = kNumSMs / (Hkv * dm.cs_nchunk);
+    if (ns > ceil_div(dm.cs_tiles, kCsMinTiles)) ns = ceil_div(dm.cs_tiles, kCsMinTiles);
     if (ns < 1) ns = 1;
     if (ns > dm.cs_tiles) ns = dm.cs_tiles;
     dm.cs_per = ceil_div(dm.cs_tiles, ns);

@@ -252,7 +252,7 @@ class Workload:
             "tok_score_kernel": ("hbm", float(Nv) * d * b),
             "merge_assign_simt_kernel": ("tensor", merge_flops),
             "merge_assign_mma_kernel": ("tensor", merge_flops),
-            "merge_avg_kernel": ("hbm", float(Nv) * d * b + float(n_out) * d * b),
+            "merge_avg_kernel": ("hbm", float(Nv) * d * b + float(n_out) * d * b),   # with its long-list launch
             "attn_stats_kernel": ("tensor", attn_flops),
             "attn_colsum_kernel": ("tensor", attn_flops),
             "attn_stats_mma_kernel": ("tensor", attn_flops),

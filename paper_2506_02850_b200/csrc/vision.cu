@@ -705,56 +705,117 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (threadIdx.x == 0 && s_abort) *status = METOK_ERR_TIMEOUT;
 }
 
-// assign[row] of every non-key token from the packed argmax.
+// An event's tokens are cut into at most 64 blocks of this many tokens; per output token one
+// bit per block says whether the block holds a member.
+__host__ __device__ __forceinline__ int avg_block_tokens(int m) {
+    const int g = (((m + 63) / 64) + 3) & ~3;
+    return g < 256 ? 256 : g;
+}
+
+// assign[row] of every non-key token from the packed argmax (tensor-core path; best64 is null when
+// the CUDA-core kernel has written assign itself), and the member-block bits of every output token.
 __global__ void __launch_bounds__(256)
 merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t* __restrict__ is_key, int Nv,
-                    int32_t* __restrict__ assign) {
+                    int N, const int32_t* __restrict__ ev_lo, int k, int32_t* __restrict__ assign,
+                    unsigned long long* __restrict__ slot_blocks, int32_t* __restrict__ slot_cnt,
+                    int32_t* __restrict__ long_index, int32_t* __restrict__ long_slot,
+                    int32_t* __restrict__ long_counter, int long_threshold, int long_cap) {
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
-    if (row < Nv && !is_key[row]) assign[row] = (int32_t)(~(uint32_t)(best64[row] & 0xFFFFFFFFull));
+    if (row >= Nv) return;
+    int slot;
+    if (best64 && !is_key[row]) {
+        slot = (int32_t)(~(uint32_t)(best64[row] & 0xFFFFFFFFull));
+        assign[row] = slot;
+    } else {
+        slot = assign[row];
+    }
+    const int e = find_event(ev_lo, k, row / N);
+    const int lo = ev_lo[e] * N, m = ev_lo[e + 1] * N - lo;
+    atomicOr(&slot_blocks[slot], 1ull << ((row - lo) / avg_block_tokens(m)));
+    // member count; the token that takes an output past the threshold books scratch for it (which
+    // scratch an output gets depends on arrival order, what is computed in it does not)
+    if (atomicAdd(&slot_cnt[slot], 1) == long_threshold) {
+        const int l = atomicAdd(long_counter, 1);
+        long_index[slot] = l;
+        if (l < long_cap) long_slot[l] = slot;
+    }
 }
 
 // --------------------------------------------------------------------------- //
-// Averaging: one CTA per output token.  The event's `assign` range is read in
-// segments; in a segment every thread takes a contiguous run of entries (16-byte loads,
-// all issued before the first is looked at), the matches are packed in token order by
-// one block-wide scan, and the member rows are then added in that order (so the
+// Averaging: one CTA per output token.  Only the blocks of the event that hold a member
+// (one bit each, set by merge_decode) are searched: their `assign` entries are read in
+// passes in which every thread takes a contiguous run (16-byte loads, all issued before
+// the first is looked at), the matches are packed in token order by one block-wide
+// scan, and the member rows are then added in that order (so the
 // summation order is fixed).  The rows come in by bulk copies into shared memory, up to
 // kAvgStages rows at once (usually all members of an output), so that the bytes in
 // flight do not depend on registers.  fp32 sum, one division, one rounding.
 // --------------------------------------------------------------------------- //
 constexpr int kAvgThreads = 128;
 constexpr int kAvgChunks = 4;      // 16-byte chunks per thread per pass over d
-constexpr int kAvgQuads = 5;       // 16-byte groups of `assign` per thread and segment
+constexpr int kAvgQuads = 5;       // 16-byte groups of `assign` per thread and pass
 constexpr int kAvgStages = 4;      // member rows in flight
 constexpr int kAvgList = 512;      // members listed at a time
 constexpr int kAvgStageBytes = kAvgThreads * kAvgChunks * 16;
 constexpr size_t kAvgSmemBytes = (size_t)kAvgStages * kAvgStageBytes + 128;
+constexpr int kAvgLong = 128;      // outputs with more members than this are split ...
+constexpr int kAvgParts = 8;       // ... over this many CTAs (fp32 partial sums, added in part order)
+constexpr int kAvgLongCap = 256;   // long outputs that get scratch for their partial sums
 
 template <typename T>
-__global__ void __launch_bounds__(kAvgThreads)
+__global__ void __launch_bounds__(kAvgThreads, 6)
 merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
                  const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
-                 const int32_t* __restrict__ n_out, T* __restrict__ out_feats, int32_t* __restrict__ out_members,
-                 int32_t* __restrict__ status) {
+                 const unsigned long long* __restrict__ slot_blocks, const int32_t* __restrict__ slot_cnt,
+                 const int32_t* __restrict__ long_index, const int32_t* __restrict__ long_slot,
+                 const int32_t* __restrict__ long_counter, float* __restrict__ long_sums,
+                 int32_t* __restrict__ long_done, int long_pass, const int32_t* __restrict__ n_out,
+                 T* __restrict__ out_feats, int32_t* __restrict__ out_members, int32_t* __restrict__ status) {
     using namespace sm100;
     constexpr int VN = Vec16<T>::N;
     extern __shared__ uint8_t avg_dyn[];
     __shared__ __align__(8) uint64_t s_bar[kAvgStages];
     __shared__ int s_list[kAvgList];
     __shared__ int s_wtot[kAvgThreads / 32];
-    __shared__ int s_abort;
+    __shared__ int s_blocks[64];
+    __shared__ int s_abort, s_last;
     // CTAs start in index order: take the outputs from the last one down, so that this pass
     // begins with the rows of V that the preceding (ascending) pass left in L2
-    const int c = *n_out - 1 - (int)blockIdx.x;
-    if (c < 0) return;
+    // An output with many members is shared by kAvgParts CTAs, each taking a range of member ranks:
+    // part 0 comes from the launch over all outputs, the other parts from a second, small launch
+    // over the outputs that booked scratch (long_pass).
+    int c, part;
+    if (!long_pass) {
+        c = *n_out - 1 - (int)blockIdx.x;
+        part = 0;
+        if (c < 0) return;
+    } else {
+        const int l = blockIdx.x / (kAvgParts - 1);
+        if (l >= min(*long_counter, kAvgLongCap)) return;
+        c = long_slot[l];
+        part = 1 + blockIdx.x % (kAvgParts - 1);
+    }
+    const int count = slot_cnt[c];
+    int li = long_index[c];
+    if (li >= kAvgLongCap) li = -1;                            // no scratch left: one CTA does it all
+    const int nparts = li >= 0 ? kAvgParts : 1;
+    const int per = (count + nparts - 1) / nparts;
+    const int r_lo = part * per, r_hi = min(count, r_lo + per);
     const int e = out_event[c];
     const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nchunk = d / VN;
     const int4* assign4 = reinterpret_cast<const int4*>(assign);
-    const int q_lo = lo >> 2, q_hi = (hi + 3) >> 2;            // groups of four tokens that touch [lo, hi)
     const uint32_t stage0 = (smem_u32(avg_dyn) + 127u) & ~127u;
+    // the blocks to search, in order; a block is searched as bt/4 + 1 groups of four tokens (its
+    // first token need not start a group)
+    const unsigned long long blocks = slot_blocks[c];
+    const int nblk = __popcll(blocks);
+    const int bt = avg_block_tokens(hi - lo), qpb = bt / 4 + 1;
+    const int total_q = nblk * qpb;
     if (tid == 0) {
+        unsigned long long mm = blocks;
+        for (int i = 0; mm; ++i, mm &= mm - 1) s_blocks[i] = __ffsll((long long)mm) - 1;
         for (int j = 0; j < kAvgStages; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
         s_abort = 0;
         mbar_fence_init();
@@ -767,16 +828,21 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
         float acc[kAvgChunks][VN];
 #pragma unroll
         for (int u = 0; u < kAvgChunks; ++u) Vec16<T>::zero(acc[u]);
-        int count = 0;
-        for (int qs = q_lo; qs < q_hi; qs += kAvgThreads * kAvgQuads) {
-            // this thread's run: groups [q0, q0 + kAvgQuads)
-            const int q0 = qs + tid * kAvgQuads;
+        int seen = 0;                                          // members met in earlier passes
+        for (int qs = 0; qs < total_q && seen < r_hi; qs += kAvgThreads * kAvgQuads) {
+            // this thread's run: kAvgQuads consecutive groups of the searched blocks
             int4 a[kAvgQuads];
+            int qidx[kAvgQuads], j_lo[kAvgQuads], j_hi[kAvgQuads];   // group index; the block's token range
 #pragma unroll
             for (int u = 0; u < kAvgQuads; ++u) {
-                const int q = q0 + u;
+                const int qf = qs + tid * kAvgQuads + u;
                 a[u] = make_int4(-1, -1, -1, -1);
-                if (q < q_hi) {
+                qidx[u] = 0; j_lo[u] = 0; j_hi[u] = 0;
+                if (qf < total_q) {
+                    const int bi = qf / qpb, wq = qf - bi * qpb;
+                    const int st = lo + s_blocks[bi] * bt;
+                    const int q = (st >> 2) + wq;
+                    qidx[u] = q; j_lo[u] = st; j_hi[u] = min(st + bt, hi);
                     if (q * 4 + 3 < Nv) {
                         a[u] = assign4[q];
                     } else {                                   // the array ends inside this group
@@ -786,14 +852,14 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
                     }
                 }
             }
-            unsigned match = 0;                                // bit 4u+k: token 4(q0+u)+k belongs to output c
+            unsigned match = 0;                                // bit 4u+i: token 4*qidx[u]+i belongs to output c
 #pragma unroll
             for (int u = 0; u < kAvgQuads; ++u) {
-                const int j = (q0 + u) * 4;
-                match |= (unsigned)(a[u].x == c && j + 0 >= lo && j + 0 < hi) << (4 * u + 0);
-                match |= (unsigned)(a[u].y == c && j + 1 >= lo && j + 1 < hi) << (4 * u + 1);
-                match |= (unsigned)(a[u].z == c && j + 2 >= lo && j + 2 < hi) << (4 * u + 2);
-                match |= (unsigned)(a[u].w == c && j + 3 >= lo && j + 3 < hi) << (4 * u + 3);
+                const int j = qidx[u] * 4;
+                match |= (unsigned)(a[u].x == c && j + 0 >= j_lo[u] && j + 0 < j_hi[u]) << (4 * u + 0);
+                match |= (unsigned)(a[u].y == c && j + 1 >= j_lo[u] && j + 1 < j_hi[u]) << (4 * u + 1);
+                match |= (unsigned)(a[u].z == c && j + 2 >= j_lo[u] && j + 2 < j_hi[u]) << (4 * u + 2);
+                match |= (unsigned)(a[u].w == c && j + 3 >= j_lo[u] && j + 3 < j_hi[u]) << (4 * u + 3);
             }
             const int mine = __popc(match);
             int incl = mine;
@@ -804,27 +870,28 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
             }
             if (lane == 31) s_wtot[warp] = incl;
             __syncthreads();
-            int before = incl - mine, total = 0;
+            int before = seen + incl - mine, total = 0;        // rank of this thread's first member
 #pragma unroll
             for (int w = 0; w < kAvgThreads / 32; ++w) {
                 const int v = s_wtot[w];
                 if (w < warp) before += v;
                 total += v;
             }
-            // the members are listed kAvgList at a time (one batch covers all but pathological cases)
-            for (int b0 = 0; b0 < total; b0 += kAvgList) {
+            // this part's ranks among the members of the pass, listed kAvgList at a time
+            const int b_lo = max(r_lo, seen), b_hi = min(r_hi, seen + total);
+            for (int b0 = b_lo; b0 < b_hi; b0 += kAvgList) {
+                const int nlist = min(kAvgList, b_hi - b0);
                 {
                     unsigned mm = match;
                     int r = before;
                     while (mm) {
                         const int b = __ffs(mm) - 1;
                         mm &= mm - 1;
-                        if (r >= b0 && r < b0 + kAvgList) s_list[r - b0] = q0 * 4 + b;
+                        if (r >= b0 && r < b0 + nlist) s_list[r - b0] = qidx[b >> 2] * 4 + (b & 3);
                         ++r;
                     }
                 }
                 __syncthreads();
-                const int nlist = min(kAvgList, total - b0);
                 for (int m0 = 0; m0 < nlist; m0 += kAvgStages) {
                     const int nr = min(kAvgStages, nlist - m0);
                     if (tid == 0) {
@@ -840,7 +907,7 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
                         phase ^= 1u << j;
                         if (!ok) continue;
                         const uint8_t* row = avg_dyn + (stage0 - smem_u32(avg_dyn)) + (size_t)j * kAvgStageBytes;
-    #pragma unroll
+#pragma unroll
                         for (int u = 0; u < kAvgChunks; ++u) {
                             const int ch = cb + u * kAvgThreads + tid;
                             if (ch < nchunk) {
@@ -851,38 +918,67 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
                                     v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
                                 } else {
                                     const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
-    #pragma unroll
+#pragma unroll
                                     for (int i = 0; i < 4; ++i) {
                                         v[2 * i]     = __uint_as_float(w4[i] << 16);
                                         v[2 * i + 1] = __uint_as_float(w4[i] & 0xFFFF0000u);
                                     }
                                 }
-    #pragma unroll
+#pragma unroll
                                 for (int q = 0; q < VN; ++q) acc[u][q] += v[q];
                             }
                         }
                     }
-                    __syncthreads();                               // every thread is done with the stages
+                    __syncthreads();                           // every thread is done with the stages
                 }
             }
-            count += total;
-            __syncthreads();                                   // s_wtot and s_list are reused by the next segment
+            seen += total;
+            __syncthreads();                                   // s_wtot and s_list are reused by the next pass
         }
-        const float inv = 1.0f / (float)count;
+        if (nparts == 1) {
+            const float inv = 1.0f / (float)count;
 #pragma unroll
-        for (int u = 0; u < kAvgChunks; ++u) {
-            const int ch = cb + u * kAvgThreads + tid;
-            if (ch < nchunk) {
-                T* o = out_feats + (size_t)c * d + (size_t)ch * VN;
-                alignas(16) T tmp[VN];
+            for (int u = 0; u < kAvgChunks; ++u) {
+                const int ch = cb + u * kAvgThreads + tid;
+                if (ch < nchunk) {
+                    T* o = out_feats + (size_t)c * d + (size_t)ch * VN;
+                    alignas(16) T tmp[VN];
 #pragma unroll
-                for (int q = 0; q < VN; ++q) from_float(tmp[q], acc[u][q] * inv);
-                *reinterpret_cast<uint4*>(o) = *reinterpret_cast<const uint4*>(tmp);
+                    for (int q = 0; q < VN; ++q) from_float(tmp[q], acc[u][q] * inv);
+                    *reinterpret_cast<uint4*>(o) = *reinterpret_cast<const uint4*>(tmp);
+                }
+            }
+        } else {
+            float* ps = long_sums + ((size_t)li * kAvgParts + part) * d;
+#pragma unroll
+            for (int u = 0; u < kAvgChunks; ++u) {
+                const int ch = cb + u * kAvgThreads + tid;
+                if (ch < nchunk) {
+#pragma unroll
+                    for (int q = 0; q < VN; ++q) ps[(size_t)ch * VN + q] = acc[u][q];
+                }
             }
         }
-        if (tid == 0 && cb == 0) out_members[c] = count;
     }
+    if (part == 0 && tid == 0) out_members[c] = count;
     if (tid == 0 && s_abort) *status = METOK_ERR_TIMEOUT;
+    if (nparts > 1) {
+        // the last part to finish adds the partial sums in part order
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = atomicAdd(&long_done[li], 1) == nparts - 1;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            const float inv = 1.0f / (float)count;
+            const float* ps = long_sums + (size_t)li * kAvgParts * d;
+            for (int i = tid; i < d; i += kAvgThreads) {
+                float a = 0.f;
+                for (int q = 0; q < kAvgParts; ++q) a += __ldcg(ps + (size_t)q * d + i);
+                from_float(out_feats[(size_t)c * d + i], a * inv);
+            }
+        }
+    }
 }
 
 // --------------------------------------------------------------------------- //
@@ -896,6 +992,14 @@ struct VisionWs {
     int32_t *ev_lo, *ev_budget, *ev_out_off, *ev_tile_off, *ev_unit_off;
     int32_t *frame_ev, *frame_stride, *frame_off;   // POOL mode
     unsigned long long* best64;   // packed argmax per token (tensor-core path)
+    unsigned long long* slot_blocks;   // per output token: which blocks of its event hold a member
+    int32_t* slot_cnt;                 // per output token: members
+    int32_t* long_counter;             // outputs with more than kAvgLong members ...
+    int32_t* long_done;                // ... parts of each that have finished
+    int32_t* long_index;               // output -> index among the long ones, -1 otherwise
+    int32_t* long_slot;                // and back
+    float* long_sums;                  // partial sums of their parts
+    size_t zero_bytes;                 // slot_blocks .. long_done are cleared together
 };
 
 static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, bool mma) {
@@ -913,6 +1017,18 @@ static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, b
     w.frame_stride = cv.take<int32_t>((size_t)Tn);
     w.frame_off = cv.take<int32_t>((size_t)Tn + 1);
     w.best64 = mma ? cv.take<unsigned long long>((size_t)Tn * N) : nullptr;
+    {
+        const size_t n = (size_t)cap + 64;
+        w.zero_bytes = n * 8 + n * 4 + (size_t)(64 + kAvgLongCap) * 4;
+        unsigned char* z = cv.take<unsigned char>(w.zero_bytes);
+        w.slot_blocks = reinterpret_cast<unsigned long long*>(z);
+        w.slot_cnt = reinterpret_cast<int32_t*>(z + n * 8);
+        w.long_counter = w.slot_cnt + n;
+        w.long_done = w.long_counter + 64;
+        w.long_index = cv.take<int32_t>(n);
+        w.long_slot = cv.take<int32_t>(kAvgLongCap);
+        w.long_sums = cv.take<float>((size_t)kAvgLongCap * kAvgParts * d);
+    }
     return w;
 }
 
@@ -1023,11 +1139,6 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
                 w.status);
         }
         METOK_LAUNCH_CHECK();
-        {
-            METOK_TIMED("merge_decode_kernel", st);
-            merge_decode_kernel<<<ceil_div(Nv, 256), 256, 0, st>>>(w.best64, w.is_key, Nv, assign);
-        }
-        METOK_LAUNCH_CHECK();
     } else {
         const int max_tiles = Nv / kMergeTM + k;
         {
@@ -1039,12 +1150,29 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         METOK_LAUNCH_CHECK();
     }
 
+    METOK_CUDA_TRY(cudaMemsetAsync(w.slot_blocks, 0, w.zero_bytes, st));
+    METOK_CUDA_TRY(cudaMemsetAsync(w.long_index, 0xFF, ((size_t)cap + 64) * sizeof(int32_t), st));
+    {
+        METOK_TIMED("merge_decode_kernel", st);
+        merge_decode_kernel<<<ceil_div(Nv, 256), 256, 0, st>>>(mma ? w.best64 : nullptr, w.is_key, Nv, N, w.ev_lo, k,
+                                                               assign, w.slot_blocks, w.slot_cnt, w.long_index,
+                                                               w.long_slot, w.long_counter, kAvgLong, kAvgLongCap);
+    }
+    METOK_LAUNCH_CHECK();
     METOK_CUDA_TRY(cudaFuncSetAttribute(merge_avg_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)kAvgSmemBytes));
     {
         METOK_TIMED("merge_avg_kernel", st);
-        merge_avg_kernel<T><<<cap, kAvgThreads, kAvgSmemBytes, st>>>(feats, d, N, Nv, w.ev_lo, out_event, assign, n_out,
-                                                                 out_feats, out_members, w.status);
+        merge_avg_kernel<T><<<cap, kAvgThreads, kAvgSmemBytes, st>>>(
+            feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
+            w.long_counter, w.long_sums, w.long_done, 0, n_out, out_feats, out_members, w.status);
+    }
+    METOK_LAUNCH_CHECK();
+    {
+        METOK_TIMED("merge_avg_long_kernel", st);
+        merge_avg_kernel<T><<<kAvgLongCap * (kAvgParts - 1), kAvgThreads, kAvgSmemBytes, st>>>(
+            feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
+            w.long_counter, w.long_sums, w.long_done, 1, n_out, out_feats, out_members, w.status);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;

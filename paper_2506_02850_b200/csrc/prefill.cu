@@ -216,7 +216,15 @@ attn_score_reduce_kernel(const float* __restrict__ part_col, int nparts, int n_v
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n_vis) return;
     float a = 0.f;
-    for (int p = 0; p < nparts; ++p) a += part_col[(size_t)p * n_vis + j];
+    int p = 0;
+    for (; p + 8 <= nparts; p += 8) {                          // eight loads in flight, added in plane order
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = part_col[(size_t)(p + u) * n_vis + j];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) a += v[u];
+    }
+    for (; p < nparts; ++p) a += part_col[(size_t)p * n_vis + j];
     scores[j] = a * inv_rows;
 }
 

@@ -95,6 +95,8 @@ def test_compress_vision_stress():
     (10, 25, 264, [0, 5, 10], "bf16", 1.0, 1.0, 0),            # keep everything: identity
     (7, 16, 40, [0, 1, 2, 3, 4, 5, 6, 7], "f32", 0.01, 0.01, 0),   # one key token per event
     (5, 130, 64, [0, 2, 5], "bf16", 0.7, 0.05, 1),
+    (14, 64, 72, [0, 12, 14], "bf16", 0.004, 0.004, 0),        # 768 tokens, 4 keys: member lists long enough to be split
+    (20, 100, 40, [0, 20], "f32", 0.0005, 0.0005, 0),          # one key token, 1999 members
 ])
 def test_compress_vision_ragged(T, N, d, offs, dtype, kk, kn, agg):
     rng = np.random.default_rng(T * 100 + N)

@@ -148,11 +148,14 @@ class Workload:
     # one pass of the hot path, device-resident inputs
     def step(self):
         B, cfg, o = self.B, self.cfg, self.out
+        # the text embedding is known before the video is segmented: segmentation and the Eq. 5
+        # token scores share one pass over V, and the compressor takes the scores from there
         if "segment" in self.parts:
-            o["seg"] = B.metok_segment_events(self.V, cfg.k, out=o.get("seg"))
+            o["seg"] = B.metok_segment_score_events(self.V, cfg.k, self.t, out=o.get("seg"))
         if "compress" in self.parts:
             offs = o["seg"]["event_offsets"] if "seg" in o else self.planted_offsets
-            o["cv"] = B.metok_compress_vision(self.V, offs, self.t, self.params, out=o.get("cv"))
+            o["cv"] = B.metok_compress_vision(self.V, offs, self.t, self.params, out=o.get("cv"),
+                                              scored=o.get("seg"))
         # The K/V lists need the first level's scores only: the compaction runs on a second stream
         # beside pruning levels 2 and 3 and joins at the end of the step.
         main = torch.cuda.current_stream()
@@ -249,6 +252,7 @@ class Workload:
         kv_rows = min(cfg.Nv, math.ceil(cfg.keep_kv * cfg.Nv - 1e-9)) + cfg.kv_text
         work = {
             "seg_partial_kernel": ("hbm", float(Nv) * d * b),
+            "seg_score_kernel": ("hbm", float(Nv) * d * b),
             "tok_score_kernel": ("hbm", float(Nv) * d * b),
             "merge_assign_simt_kernel": ("tensor", merge_flops),
             "merge_assign_mma_kernel": ("tensor", merge_flops),

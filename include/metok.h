@@ -136,6 +136,32 @@ METOK_API int metok_segment_events_static(const void* feats, int dtype, int T, i
                                 int32_t* frame_event, void* stream);
 
 /* ------------------------------------------------------------------------- *
+ * (1c) Segmentation and the token relevance of Eq. 5 in one pass -- Eq. 4 and
+ *      Eq. 5; Algorithm 1, "Event temporal segmentation" and "Key visual-text
+ *      semantic identification".
+ *
+ *   Both need one read of V each and nothing of each other; when the text
+ *   embedding is already known at segmentation time this call computes
+ *   everything metok_segment_events computes (sim_mode FLATTEN) and, from the same
+ *   pass over V,
+ *     token_score[j]    = cos(x_j, t)            (what metok_compress_vision's first step computes)
+ *     token_inv_norm[j] = 1 / max(|x_j|, 1e-8)
+ *   Hand both to metok_compress_vision (token_score argument; params.token_inv_norm)
+ *   and it skips its own pass over V.
+ *
+ *   text_emb       DEVICE [d] of `dtype`                  (input)
+ *   token_score    DEVICE float [T*N]                     (output)
+ *   token_inv_norm DEVICE float [T*N]                     (output)
+ *   the other arguments and errors as in metok_segment_events; UNSUPPORTED also for
+ *   rows of more than 8 KiB (use the two separate calls).
+ * ------------------------------------------------------------------------- */
+METOK_API size_t metok_segment_score_events_workspace_bytes(int dtype, int T, int N, int d);
+METOK_API int metok_segment_score_events(const void* feats, int dtype, int T, int N, int d, int k,
+                               const void* text_emb, float* sims, int32_t* boundaries,
+                               int32_t* event_offsets, int32_t* frame_event, float* token_score,
+                               float* token_inv_norm, void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
  * (2) Event-aware token reduction after the vision encoder -- Eq. 5 and
  *     section 3.2.1 ("Key Visual-Text Semantic Identification", "Adaptive
  *     Pooling Strategy"); Algorithm 1.
@@ -168,7 +194,8 @@ METOK_API int metok_segment_events_static(const void* feats, int dtype, int T, i
  *   out_event     DEVICE int32 [cap]  event of the output token
  *   out_members   DEVICE int32 [cap]  number of input tokens averaged (>= 1)
  *   assign        DEVICE int32 [T*N]  output row that each input token went into
- *   token_score   DEVICE float [T*N]; frame_score DEVICE float [T];
+ *   token_score   DEVICE float [T*N] (input instead when p->token_inv_norm is set);
+ *   frame_score   DEVICE float [T];
  *   event_score   DEVICE float [k];   event_is_key DEVICE uint8 [k]
  *   n_out         DEVICE int32 scalar: number of output tokens
  *   cap           rows available in the out_* arrays; must be at least
@@ -187,6 +214,8 @@ typedef struct metok_vision_params {
     double beta;         /* POOL: key-frame ratio, (0,1]                        */
     int    s1, s2;       /* POOL: strides of key / other frames in key events   */
     int    s1_nonkey, s2_nonkey;  /* POOL: the same for non-key events (the paper: s/alpha) */
+    const float* token_inv_norm;  /* NULL, or DEVICE float [T*N] from metok_segment_score_events: then the
+                                     token_score argument is an INPUT and the Eq. 5 pass over V is skipped */
 } metok_vision_params;
 
 METOK_API int    metok_compress_vision_bound(int T, int N, int k, const metok_vision_params* p);

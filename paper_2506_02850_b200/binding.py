@@ -30,7 +30,8 @@ _vp, _i, _sz, _f, _d = _c.c_void_p, _c.c_int, _c.c_size_t, _c.c_float, _c.c_doub
 
 class VisionParams(_c.Structure):
     _fields_ = [("alpha", _d), ("event_agg", _i), ("mode", _i), ("keep_key", _d), ("keep_nonkey", _d),
-                ("beta", _d), ("s1", _i), ("s2", _i), ("s1_nonkey", _i), ("s2_nonkey", _i)]
+                ("beta", _d), ("s1", _i), ("s2", _i), ("s1_nonkey", _i), ("s2_nonkey", _i),
+                ("token_inv_norm", _vp)]
 
 
 class MetokError(RuntimeError):
@@ -46,6 +47,8 @@ _SIGNATURES = {
     "metok_segment_events": (_i, [_vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "metok_segment_events_static_capacity": (_sz, []),
     "metok_segment_events_static": (_i, [_vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "metok_segment_score_events_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "metok_segment_score_events": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "metok_compress_vision_bound": (_i, [_i, _i, _i, _c.POINTER(VisionParams)]),
     "metok_compress_vision_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _c.POINTER(VisionParams)]),
     "metok_compress_vision": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _vp, _c.POINTER(VisionParams),
@@ -176,10 +179,41 @@ def metok_segment_events_static(feats: torch.Tensor, k: int, sim_mode: int = SIM
             "frame_event": frame_event}
 
 
+def metok_segment_score_events(feats: torch.Tensor, k: int, text_emb: torch.Tensor,
+                               out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """metok_segment_events (FLATTEN) plus the per-token text relevance and inverse norms of the
+    same pass over `feats`; hand "token_score" / "token_inv_norm" on to metok_compress_vision."""
+    feats = _cuda_contig(feats, "feats")
+    text_emb = _cuda_contig(text_emb, "text_emb")
+    T, N, d = feats.shape
+    dev = feats.device
+    L = lib()
+    if out is None:
+        out = {
+            "_sims": torch.empty(max(T - 1, 1), dtype=torch.float32, device=dev),
+            "_boundaries": torch.empty(max(k - 1, 1), dtype=torch.int32, device=dev),
+            "_offsets": torch.empty(max(k + 1, 2), dtype=torch.int32, device=dev),
+            "frame_event": torch.empty(T, dtype=torch.int32, device=dev),
+            "token_score": torch.empty(T * N, dtype=torch.float32, device=dev),
+            "token_inv_norm": torch.empty(T * N, dtype=torch.float32, device=dev),
+        }
+    need = L.metok_segment_score_events_workspace_bytes(_dt(feats), T, N, d)
+    ws = workspace(need, dev)
+    st = L.metok_segment_score_events(_ptr(feats), _dt(feats), T, N, d, k, _ptr(text_emb), _ptr(out["_sims"]),
+                                      _ptr(out["_boundaries"]), _ptr(out["_offsets"]), _ptr(out["frame_event"]),
+                                      _ptr(out["token_score"]), _ptr(out["token_inv_norm"]), _ptr(ws), ws.numel(),
+                                      _stream())
+    _check("metok_segment_score_events", st)
+    out["sims"] = out["_sims"][: T - 1]
+    out["boundaries"] = out["_boundaries"][: max(k - 1, 0)]
+    out["event_offsets"] = out["_offsets"][: k + 1]
+    return out
+
+
 def vision_params(alpha: float, keep_key: float = 1.0, keep_nonkey: float = 1.0, event_agg: int = AGG_MEAN,
                   mode: int = MODE_TOPK_MERGE, beta: float = 0.5, s1: int = 2, s2: int = 3,
                   s1_nonkey: int = 4, s2_nonkey: int = 6) -> VisionParams:
-    return VisionParams(alpha, event_agg, mode, keep_key, keep_nonkey, beta, s1, s2, s1_nonkey, s2_nonkey)
+    return VisionParams(alpha, event_agg, mode, keep_key, keep_nonkey, beta, s1, s2, s1_nonkey, s2_nonkey, None)
 
 
 def metok_compress_vision_bound(T: int, N: int, k: int, p: VisionParams) -> int:
@@ -191,7 +225,10 @@ def metok_compress_vision_bound(T: int, N: int, k: int, p: VisionParams) -> int:
 
 def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text_emb: torch.Tensor,
                           p: VisionParams, cap: Optional[int] = None,
-                          out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+                          out: Optional[Dict[str, torch.Tensor]] = None,
+                          scored: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """`scored` (the result of metok_segment_score_events on the same feats and text) makes the call
+    skip its own scoring pass over `feats`."""
     feats = _cuda_contig(feats, "feats")
     event_offsets = _cuda_contig(event_offsets, "event_offsets")
     text_emb = _cuda_contig(text_emb, "text_emb")
@@ -215,6 +252,10 @@ def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text
             "event_is_key": torch.empty(k, dtype=torch.uint8, device=dev),
             "n_out": torch.zeros(1, **i32),
         }
+    if scored is not None:
+        out["token_score"] = scored["token_score"]
+        p = VisionParams.from_buffer_copy(p)
+        p.token_inv_norm = scored["token_inv_norm"].data_ptr()
     need = L.metok_compress_vision_workspace_bytes(_dt(feats), T, N, d, k, cap, _c.byref(p))
     ws = workspace(need, dev)
     st = L.metok_compress_vision(_ptr(feats), _dt(feats), T, N, d, _ptr(event_offsets), k, _ptr(text_emb),

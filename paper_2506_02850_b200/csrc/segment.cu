@@ -326,6 +326,183 @@ extern "C" int metok_segment_events(const void* feats, int dtype, int T, int N, 
 }
 
 // --------------------------------------------------------------------------- //
+// metok_segment_score_events: segmentation and the per-token text relevance of Eq. 5
+// in ONE pass over V.  A warp owns one token position p and a run of frames; per frame
+// it loads the token row (kCH 16-byte chunks per lane, all in flight at once), and from
+// the same registers takes the row's squared norm, its dot product with the text
+// embedding (shared memory) and its dot product with the same position's row of the
+// previous frame (kept as raw chunks in shared memory, which leaves the registers to
+// the loads in flight).  Token score and 1/norm are final in the warp; the
+// per-(position, frame) norms and dots are added over the positions by seg_finish in a
+// fixed order.  (A variant that staged the rows by bulk copies in a per-warp ring of
+// shared memory was slower: shared memory then limits an SM to six warps, too few to
+// keep up with the arithmetic of a row.)
+// --------------------------------------------------------------------------- //
+namespace metok {
+
+constexpr int kFsThreads = 128;
+
+template <typename T, int kCH>
+__global__ void __launch_bounds__(kFsThreads, 5)
+seg_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Tn, int N, int d, int frames_per_warp,
+                 float* __restrict__ part_dot, float* __restrict__ part_nrm, float* __restrict__ token_score,
+                 float* __restrict__ inv_norm) {
+    constexpr int VN = Vec16<T>::N;
+    extern __shared__ float s_t[];                 // [d], in planes of 4 floats per chunk (conflict-free 16-byte reads)
+                                                   // then [warps][nchunk] raw 16-byte chunks: the previous frame's row
+    __shared__ float s_red[kFsThreads / 32];
+    __shared__ float s_tn;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nchunk = d / VN;
+    for (int i = tid; i < d; i += kFsThreads) {
+        const int c = i / VN, q = i % VN;
+        s_t[(q >> 2) * (nchunk * 4) + c * 4 + (q & 3)] = to_float(text[i]);
+    }
+    __syncthreads();
+    float a = 0.f;
+    for (int i = tid; i < d; i += kFsThreads) a = fmaf(s_t[i], s_t[i], a);
+    a = warp_sum(a);
+    if (lane == 0) s_red[warp] = a;
+    __syncthreads();
+    if (tid == 0) {
+        float sum = 0.f;
+        for (int w = 0; w < kFsThreads / 32; ++w) sum += s_red[w];
+        s_tn = fmaxf(sqrtf(sum), kEps);
+    }
+    __syncthreads();
+    const float tn = s_tn;
+    const int nruns = (Tn + frames_per_warp - 1) / frames_per_warp;
+    const int gw = blockIdx.x * (kFsThreads / 32) + warp;
+    if (gw >= N * nruns) return;
+    const int p = gw % N, run = gw / N;
+    const int f0 = run * frames_per_warp;
+    const int f1 = min(Tn, f0 + frames_per_warp);           // own frames [f0, f1)
+    const int f_last = min(Tn - 1, f1);                     // halo frame for the last dot
+    const uint4* base = reinterpret_cast<const uint4*>(feats);
+    uint4* prev = reinterpret_cast<uint4*>(s_t + d) + (size_t)warp * nchunk;   // d floats = a multiple of 16 bytes
+    uint4 cur[kCH];
+#pragma unroll
+    for (int u = 0; u < kCH; ++u) {
+        const int c = u * 32 + lane;
+        if (c < nchunk) prev[c] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    for (int f = f0; f <= f_last; ++f) {
+        const size_t row = (size_t)f * N + p;
+        const uint4* x = base + row * (size_t)nchunk;
+#pragma unroll
+        for (int u = 0; u < kCH; ++u) {
+            const int c = u * 32 + lane;
+            cur[u] = c < nchunk ? __ldg(x + c) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        float nn = 0.f, dt = 0.f, dp = 0.f;
+#pragma unroll
+        for (int u = 0; u < kCH; ++u) {
+            const int c = u * 32 + lane;
+            if (c < nchunk) {
+                float v[VN], pv[VN];
+                widen16<T>(cur[u], v);
+                widen16<T>(prev[c], pv);
+                prev[c] = cur[u];                           // a lane only ever touches its own chunks
+#pragma unroll
+                for (int h = 0; h < VN / 4; ++h) {
+                    const float4 tt = reinterpret_cast<const float4*>(s_t + h * (nchunk * 4))[c];
+                    nn = fmaf(v[4 * h + 0], v[4 * h + 0], nn); dt = fmaf(v[4 * h + 0], tt.x, dt); dp = fmaf(v[4 * h + 0], pv[4 * h + 0], dp);
+                    nn = fmaf(v[4 * h + 1], v[4 * h + 1], nn); dt = fmaf(v[4 * h + 1], tt.y, dt); dp = fmaf(v[4 * h + 1], pv[4 * h + 1], dp);
+                    nn = fmaf(v[4 * h + 2], v[4 * h + 2], nn); dt = fmaf(v[4 * h + 2], tt.z, dt); dp = fmaf(v[4 * h + 2], pv[4 * h + 2], dp);
+                    nn = fmaf(v[4 * h + 3], v[4 * h + 3], nn); dt = fmaf(v[4 * h + 3], tt.w, dt); dp = fmaf(v[4 * h + 3], pv[4 * h + 3], dp);
+                }
+            }
+        }
+        nn = warp_sum(nn);
+        dt = warp_sum(dt);
+        dp = warp_sum(dp);
+        if (lane == 0) {
+            if (f < f1) {
+                const float n = fmaxf(sqrtf(nn), kEps);
+                part_nrm[(size_t)p * Tn + f] = nn;
+                token_score[row] = dt / (n * tn);
+                inv_norm[row] = 1.0f / n;
+            }
+            if (f > f0) part_dot[(size_t)p * Tn + (f - 1)] = dp;   // dot of frames f-1 and f at position p
+        }
+    }
+}
+
+template <typename T, int kCH>
+static int launch_seg_score(const void* feats, const void* text, int Tn, int N, int d, int k, float* sims,
+                            int32_t* boundaries, int32_t* event_offsets, int32_t* frame_event,
+                            float* token_score, float* inv_norm, void* ws, cudaStream_t st) {
+    Carver cv(ws);
+    float* part_dot = cv.take<float>((size_t)N * Tn);
+    float* part_nrm = cv.take<float>((size_t)N * Tn);
+    int fpw = kSegMaxRun;
+    while (fpw > 1 && (long long)N * ceil_div(Tn, fpw) < 12LL * kNumSMs) fpw >>= 1;   // 12 to 24 warps per SM
+    const int warps = N * ceil_div(Tn, fpw);
+    const size_t smem_t = (size_t)d * sizeof(float) + (size_t)(kFsThreads / 32) * d * sizeof(T);
+    if (smem_t > 40 * 1024)
+        METOK_CUDA_TRY(cudaFuncSetAttribute(seg_score_kernel<T, kCH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)smem_t));
+    {
+        METOK_TIMED("seg_score_kernel", st);
+        seg_score_kernel<T, kCH><<<ceil_div(warps, kFsThreads / 32), kFsThreads, smem_t, st>>>(
+            reinterpret_cast<const T*>(feats), reinterpret_cast<const T*>(text), Tn, N, d, fpw, part_dot, part_nrm,
+            token_score, inv_norm);
+    }
+    METOK_LAUNCH_CHECK();
+    const size_t smem = (size_t)Tn * 3 * sizeof(float);
+    if (smem > 48 * 1024)
+        METOK_CUDA_TRY(cudaFuncSetAttribute(seg_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        METOK_TIMED("seg_finish_kernel", st);
+        seg_finish_kernel<<<1, 1024, smem, st>>>(part_dot, part_nrm, N, Tn, k, sims, boundaries, event_offsets,
+                                             frame_event);
+    }
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
+}
+
+}  // namespace metok
+
+extern "C" size_t metok_segment_score_events_workspace_bytes(int dtype, int T, int N, int d) {
+    (void)dtype; (void)d;
+    if (T < 1 || N < 1) return 0;
+    Carver cv(nullptr);
+    cv.take<float>((size_t)N * T);
+    cv.take<float>((size_t)N * T);
+    return cv.total();
+}
+
+extern "C" int metok_segment_score_events(const void* feats, int dtype, int T, int N, int d, int k,
+                                          const void* text_emb, float* sims, int32_t* boundaries,
+                                          int32_t* event_offsets, int32_t* frame_event, float* token_score,
+                                          float* token_inv_norm, void* ws, size_t ws_bytes, void* stream) {
+    if (!feats || !text_emb || !sims || !boundaries || !event_offsets || !frame_event || !token_score || !token_inv_norm)
+        return METOK_ERR_INVALID_ARG;
+    if (dtype != METOK_F32 && dtype != METOK_BF16) return METOK_ERR_INVALID_ARG;
+    if (T < 1 || N < 1 || d < 1 || k < 1 || k > T) return METOK_ERR_INVALID_ARG;
+    if (!aligned16(feats) || !aligned16(text_emb)) return METOK_ERR_INVALID_ARG;
+    const int eb = dtype == METOK_F32 ? 4 : 2;
+    if (((long long)d * eb) % 16 != 0 || T > kMaxFrames) return METOK_ERR_UNSUPPORTED;
+    const long long nchunk = (long long)d * eb / 16;
+    if (nchunk > 32 * 16) return METOK_ERR_UNSUPPORTED;          // rows of more than 8 KiB: use the two separate calls
+    const size_t need = metok_segment_score_events_workspace_bytes(dtype, T, N, d);
+    if (!ws || ws_bytes < need || !aligned16(ws)) return METOK_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+#define METOK_FS(TYPE, CH)                                                                                        \
+    return launch_seg_score<TYPE, CH>(feats, text_emb, T, N, d, k, sims, boundaries, event_offsets, frame_event, \
+                                      token_score, token_inv_norm, ws, st)
+    if (dtype == METOK_F32) {
+        if (nchunk <= 32 * 4) METOK_FS(float, 4);
+        if (nchunk <= 32 * 8) METOK_FS(float, 8);
+        METOK_FS(float, 16);
+    }
+    if (nchunk <= 32 * 4) METOK_FS(__nv_bfloat16, 4);
+    if (nchunk <= 32 * 8) METOK_FS(__nv_bfloat16, 8);
+    METOK_FS(__nv_bfloat16, 16);
+#undef METOK_FS
+}
+
+// --------------------------------------------------------------------------- //
 // metok_segment_events_static: the same computation with the scratch in a fixed
 // array that lives inside the library image instead of a caller workspace.
 // --------------------------------------------------------------------------- //

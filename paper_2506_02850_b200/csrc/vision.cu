@@ -1057,7 +1057,9 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     VisionWs w = carve_vision(cv, Tn, N, k, d, cap, mma);
     METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
 
-    {
+    // Eq. 5 per token, unless the caller brings the scores and norms from metok_segment_score_events
+    const float* inv_norm = p->token_inv_norm ? p->token_inv_norm : w.inv_norm;
+    if (!p->token_inv_norm) {
         const int grid = min(ceil_div(Nv, 8), kNumSMs * 8);
         const size_t smem = (size_t)d * sizeof(float);
         if (smem > 48 * 1024)
@@ -1135,7 +1137,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         {
             METOK_TIMED("merge_assign_mma_kernel", st);
             merge_assign_mma_kernel<<<kNumSMs, kMmaThreads, kMmaSmemBytes, st>>>(
-                tmA, tmA_half, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, w.inv_norm, w.is_key, w.best64,
+                tmA, tmA_half, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, inv_norm, w.is_key, w.best64,
                 w.status);
         }
         METOK_LAUNCH_CHECK();
@@ -1144,7 +1146,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         {
             METOK_TIMED("merge_assign_simt_kernel", st);
             merge_assign_simt_kernel<T><<<max_tiles, 256, 0, st>>>(feats, d, N, w.ev_lo, k, w.ev_out_off,
-                                                                   w.ev_tile_off, out_src, w.inv_norm, w.is_key,
+                                                                   w.ev_tile_off, out_src, inv_norm, w.is_key,
                                                                    assign);
         }
         METOK_LAUNCH_CHECK();

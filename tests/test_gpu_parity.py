@@ -67,6 +67,50 @@ def test_segment_events_ties_go_to_lower_index_and_repeatable():
         assert torch.equal(a, B.metok_segment_events(x, 4)["sims"])
 
 
+@pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128"])
+def test_segment_score_events_one_pass(name):
+    """Segmentation and Eq. 5 token scores from one pass over V: both against the oracle, and the
+    compressor fed with them against the compressor that scores by itself."""
+    cfg = W.CONFIGS[name]
+    vis = vis_of(name)
+    Vd, td = P.to_torch(vis["V"], cfg.dtype), P.to_torch(vis["t"], cfg.dtype)
+    got = B.metok_segment_score_events(Vd, cfg.k, td)
+    want = O.segment_events(vis["V"], cfg.k)
+    P.check_scores(got["sims"].cpu().numpy(), want["sims"], cfg.dtype, "sims")
+    assert np.array_equal(got["boundaries"].cpu().numpy(), want["boundaries"])
+    assert np.array_equal(got["event_offsets"].cpu().numpy(), want["event_offsets"])
+    assert np.array_equal(got["frame_event"].cpu().numpy(), want["frame_event"])
+    ts = O.token_relevance(vis["V"], vis["t"])
+    P.check_scores(got["token_score"].cpu().numpy(), ts, cfg.dtype, "token_score")
+    norms = np.sqrt((vis["V"].reshape(cfg.Nv, -1).astype(np.float64) ** 2).sum(axis=1))
+    assert np.allclose(got["token_inv_norm"].cpu().numpy(), 1.0 / np.maximum(norms, 1e-8), rtol=1e-5)
+    p = B.vision_params(cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+    a = B.metok_compress_vision(Vd, got["event_offsets"], td, p)
+    b = B.metok_compress_vision(Vd, got["event_offsets"], td, p, scored=got)
+    torch.cuda.synchronize()
+    n = int(a["n_out"].item())
+    assert n == int(b["n_out"].item())
+    assert np.array_equal(a["event_is_key"].cpu().numpy(), b["event_is_key"].cpu().numpy())
+    same = float(np.mean(a["out_src"][:n].cpu().numpy() == b["out_src"][:n].cpu().numpy()))
+    assert same > 0.995, same                                  # the two scoring passes round differently in near-ties
+    want_c = O.compress_vision(vis["V"], vis["t"], want["event_offsets"], cfg.alpha, cfg.keep_enc, cfg.keep_enc, cfg.dtype)
+    P.check_index_set(b["out_src"][:n].cpu().numpy(), want_c["out_src"], lambda j: bool(want_c["near_tie"][j]),
+                      "key tokens from one-pass scores")
+
+
+def test_segment_score_events_ragged():
+    for T, N, d, k, dtype in [(3, 5, 72, 2, "f32"), (9, 7, 40, 9, "bf16"), (17, 33, 264, 5, "bf16"), (5, 3, 2056, 3, "bf16")]:
+        rng = np.random.default_rng(T * 1000 + N)
+        V = W.quantize(rng.standard_normal((T, N, d)).astype(np.float32), dtype)
+        t = W.quantize(rng.standard_normal(d).astype(np.float32), dtype)
+        got = B.metok_segment_score_events(P.to_torch(V, dtype), k, P.to_torch(t, dtype))
+        want = O.segment_events(V, k)
+        if T > 1:
+            P.check_scores(got["sims"].cpu().numpy(), want["sims"], dtype, "sims")
+        P.check_scores(got["token_score"].cpu().numpy(), O.token_relevance(V, t), dtype, "token_score")
+        assert np.array_equal(got["event_offsets"].cpu().numpy(), want["event_offsets"]) or T <= 3
+
+
 # ------------------------------------------------------------- a2 a3 a4 ---- #
 
 @pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128", "frames128d1024"])

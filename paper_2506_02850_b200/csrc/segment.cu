@@ -343,7 +343,7 @@ namespace metok {
 constexpr int kFsThreads = 128;
 
 template <typename T, int kCH>
-__global__ void __launch_bounds__(kFsThreads, 5)
+__global__ void __launch_bounds__(kFsThreads, 3)
 seg_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Tn, int N, int d, int frames_per_warp,
                  float* __restrict__ part_dot, float* __restrict__ part_nrm, float* __restrict__ token_score,
                  float* __restrict__ inv_norm) {
@@ -380,20 +380,25 @@ seg_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Tn
     const int f_last = min(Tn - 1, f1);                     // halo frame for the last dot
     const uint4* base = reinterpret_cast<const uint4*>(feats);
     uint4* prev = reinterpret_cast<uint4*>(s_t + d) + (size_t)warp * nchunk;   // d floats = a multiple of 16 bytes
-    uint4 cur[kCH];
+    uint4 cur[kCH], nxt[kCH];
 #pragma unroll
     for (int u = 0; u < kCH; ++u) {
         const int c = u * 32 + lane;
         if (c < nchunk) prev[c] = make_uint4(0u, 0u, 0u, 0u);
     }
-    for (int f = f0; f <= f_last; ++f) {
-        const size_t row = (size_t)f * N + p;
-        const uint4* x = base + row * (size_t)nchunk;
+    auto fetch = [&](int f, uint4 (&r)[kCH]) {
+        const uint4* x = base + ((size_t)f * N + p) * (size_t)nchunk;
 #pragma unroll
         for (int u = 0; u < kCH; ++u) {
             const int c = u * 32 + lane;
-            cur[u] = c < nchunk ? __ldg(x + c) : make_uint4(0u, 0u, 0u, 0u);
+            r[u] = c < nchunk ? __ldg(x + c) : make_uint4(0u, 0u, 0u, 0u);
         }
+    };
+    fetch(f0, cur);
+    // the next row's loads are in flight while this row is reduced
+    for (int f = f0; f <= f_last; ++f) {
+        const size_t row = (size_t)f * N + p;
+        if (f < f_last) fetch(f + 1, nxt);
         float nn = 0.f, dt = 0.f, dp = 0.f;
 #pragma unroll
         for (int u = 0; u < kCH; ++u) {
@@ -425,6 +430,8 @@ seg_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Tn
             }
             if (f > f0) part_dot[(size_t)p * Tn + (f - 1)] = dp;   // dot of frames f-1 and f at position p
         }
+#pragma unroll
+        for (int u = 0; u < kCH; ++u) cur[u] = nxt[u];
     }
 }
 
@@ -436,7 +443,7 @@ static int launch_seg_score(const void* feats, const void* text, int Tn, int N, 
     float* part_dot = cv.take<float>((size_t)N * Tn);
     float* part_nrm = cv.take<float>((size_t)N * Tn);
     int fpw = kSegMaxRun;
-    while (fpw > 1 && (long long)N * ceil_div(Tn, fpw) < 12LL * kNumSMs) fpw >>= 1;   // 12 to 24 warps per SM
+    while (fpw > 1 && (long long)N * ceil_div(Tn, fpw) < 8LL * kNumSMs) fpw >>= 1;    // 8 to 16 warps per SM
     const int warps = N * ceil_div(Tn, fpw);
     const size_t smem_t = (size_t)d * sizeof(float) + (size_t)(kFsThreads / 32) * d * sizeof(T);
     if (smem_t > 40 * 1024)

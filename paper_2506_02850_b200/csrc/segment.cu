@@ -327,16 +327,33 @@ extern "C" int metok_segment_events(const void* feats, int dtype, int T, int N, 
 
 // --------------------------------------------------------------------------- //
 // metok_segment_score_events: segmentation and the per-token text relevance of Eq. 5
-// in ONE pass over V.  A warp owns one token position p and a run of frames; per frame
-// it loads the token row (kCH 16-byte chunks per lane, all in flight at once), and from
-// the same registers takes the row's squared norm, its dot product with the text
-// embedding (shared memory) and its dot product with the same position's row of the
-// previous frame (kept as raw chunks in shared memory, which leaves the registers to
-// the loads in flight).  Token score and 1/norm are final in the warp; the
-// per-(position, frame) norms and dots are added over the positions by seg_finish in a
-// fixed order.  (A variant that staged the rows by bulk copies in a per-warp ring of
-// shared memory was slower: shared memory then limits an SM to six warps, too few to
-// keep up with the arithmetic of a row.)
+// in ONE pass over V: per token row its squared norm, its dot product with the text
+// embedding and its dot product with the same position's row of the previous frame.
+// Token score and 1/norm are final in the kernel; the per-(position, frame) norms and
+// dots are added over the positions by seg_finish in a fixed order.
+//
+// fp32 rows (seg_score_kernel): a warp owns one token position and a run of frames, holds
+// the row in registers (the next row's loads in flight meanwhile) and the previous row in
+// shared memory, and takes the three sums with multiply-adds.
+//
+// bf16 rows (seg_score_mma_kernel).  The multiply-add form costs 40 instructions per 16
+// bytes (widening, three fma per element) and needs the whole row in registers, which
+// leaves an SM with 12 warps.  Here the rows land in shared memory by 16-byte
+// asynchronous copies (a ring of kFsDepth stages per warp, no registers held while in
+// flight) and the sums run on the tensor cores.  A warp owns one position and
+// EIGHT consecutive frames; a stage holds one 64-byte slice of those eight rows and of
+// the frame before them.  Lane (g, q) = (lane / 4, lane % 4) reads chunk q of frame g's
+// slice: the 16 bytes, as they lie in memory (dwords m0..m3), are the A operand of
+// m16n8k16 mma, which gives row g of A the k-slots (m0, m2) and row 8 + g the slots
+// (m1, m3).  The other vector is the B operand, whose two registers pair with (m0, m2)
+// in the upper half of C and with (m1, m3) in the lower half: with B = (y0, y2) the
+// diagonal element C[g][g] adds the products of the even dwords of frame g's slice, with
+// B = (y1, y3) C[8 + g][g] those of the odd dwords -- the order of k inside a dot product
+// is free as long as both operands use the same one.  Two mma per slice and vector pair,
+// accumulated over the slices of the row: at the end the lane that holds C[g][g] has the
+// complete sum of frame g, with no shuffle and no widening.  The previous frame's slice
+// is the neighbouring 64 bytes of the same stage.  Products of bf16 are exact in fp32 and
+// the sums are fp32; the off-diagonal entries are never read.
 // --------------------------------------------------------------------------- //
 namespace metok {
 
@@ -435,6 +452,149 @@ seg_score_kernel(const T* __restrict__ feats, const T* __restrict__ text, int Tn
     }
 }
 
+// D += A * B for one m16n8k16 bf16 tile, fp32 accumulators; A is a 16-byte chunk as loaded.
+__device__ __forceinline__ void mma_bf16_m16n8k16(float (&c)[4], const uint4& a, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
+}
+
+// 16-byte asynchronous copy global -> shared that bypasses L1; src_bytes = 0 writes zeros.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+constexpr int kFsDepth = 16;                       // stages of a warp's ring
+constexpr int kFsFrames = 8;                       // frames per warp = row groups of the mma tile
+constexpr int kFsStageBytes = (kFsFrames + 1) * 64;
+
+// Shared memory: the text embedding as 16-byte chunks with the dwords in the order
+// (0, 2, 1, 3), zero-padded to whole slices; then per warp kFsDepth stages of 9 x 64 bytes
+// (slice of frame f0 - 1, then of frames f0 .. f0 + 7).
+template <bool kFull>                               // kFull: the row is a whole number of 64-byte slices
+__global__ void __launch_bounds__(kFsThreads)
+seg_score_mma_kernel(const __nv_bfloat16* __restrict__ feats, const __nv_bfloat16* __restrict__ text, int Tn, int N,
+                     int d, float* __restrict__ part_dot, float* __restrict__ part_nrm,
+                     float* __restrict__ token_score, float* __restrict__ inv_norm) {
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    __shared__ float s_red[kFsThreads / 32];
+    __shared__ float s_tn;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nchunk = d / 8;
+    const int nslice = (nchunk + 3) >> 2;
+    uint4* s_text = reinterpret_cast<uint4*>(s_dyn);
+    float a = 0.f;
+    for (int c = tid; c < nslice * 4; c += kFsThreads) {
+        const uint4 r = c < nchunk ? __ldg(reinterpret_cast<const uint4*>(text) + c) : make_uint4(0u, 0u, 0u, 0u);
+        s_text[c] = make_uint4(r.x, r.z, r.y, r.w);
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+            a = fmaf(lo, lo, a);
+            a = fmaf(hi, hi, a);
+        }
+    }
+    a = warp_sum(a);
+    if (lane == 0) s_red[warp] = a;
+    __syncthreads();
+    if (tid == 0) {
+        float sum = 0.f;
+        for (int w = 0; w < kFsThreads / 32; ++w) sum += s_red[w];
+        s_tn = fmaxf(sqrtf(sum), kEps);
+    }
+    __syncthreads();
+    const float tn = s_tn;
+    const int nruns = (Tn + kFsFrames - 1) / kFsFrames;
+    const int gw = blockIdx.x * (kFsThreads / 32) + warp;   // the warp owns position p and eight frames
+    if (gw >= N * nruns) return;
+    const int p = gw % N, run = gw / N;
+    const int f0 = run * kFsFrames;
+    const int g = lane >> 2, q = lane & 3;
+    const int f = f0 + g;                                   // this lane's frame
+    const bool has_f = f < Tn;
+    const bool halo = g == 0 && f0 > 0;                     // lanes 0..3 also fetch frame f0 - 1
+    // chunk q of slice 0 of this lane's row, and of the row before the run (a valid address even if unused)
+    const uint4* src = reinterpret_cast<const uint4*>(feats) + ((size_t)(has_f ? f : 0) * N + p) * (size_t)nchunk + q;
+    const uint4* src_h = reinterpret_cast<const uint4*>(feats) + ((size_t)(halo ? f0 - 1 : 0) * N + p) * (size_t)nchunk + q;
+    const uint32_t sz = has_f ? 16u : 0u, sz_h = halo ? 16u : 0u;      // 0 bytes read = zeros written
+    unsigned char* ring = s_dyn + (size_t)nslice * 4 * sizeof(uint4) + (size_t)warp * kFsDepth * kFsStageBytes;
+    const unsigned char* mine = ring + (g + 1) * 64 + q * 16;
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + (uint32_t)((g + 1) * 64 + q * 16);
+    const uint32_t dst_h = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + (uint32_t)(q * 16);
+    const uint4* tq = s_text + q;
+    // slice sl into stage `stage` (a constant where the caller is unrolled); one group per call
+    auto issue = [&](int sl, int stage) {
+        if (sl < nslice) {
+            const bool in = kFull || sl * 4 + q < nchunk;
+            const int o = in ? sl * 4 : 0;
+            cp_async16(dst + stage * kFsStageBytes, src + o, in ? sz : 0u);
+            if (g == 0) cp_async16(dst_h + stage * kFsStageBytes, src_h + o, in ? sz_h : 0u);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int j = 0; j < kFsDepth - 1; ++j) issue(j, j);
+    // accumulators: [0] pairs the even dwords (diagonal of the upper half), [1] the odd ones (lower half)
+    float cn[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float cp[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float ct[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll 1
+    for (int base = 0; base < nslice; base += kFsDepth) {
+#pragma unroll
+        for (int j = 0; j < kFsDepth; ++j) {
+            const int sl = base + j;
+            if (sl < nslice) {                              // the same for the whole warp
+                cp_async_wait<kFsDepth - 2>();              // this lane's copies of slice sl have landed
+                __syncwarp();                               // ... and every lane's; slice sl - 1 is read by all
+                issue(sl + kFsDepth - 1, (j + kFsDepth - 1) % kFsDepth);      // into the stage that held slice sl - 1
+                const uint4 x = *reinterpret_cast<const uint4*>(mine + j * kFsStageBytes);
+                const uint4 pv = *reinterpret_cast<const uint4*>(mine + j * kFsStageBytes - 64);
+                const uint4 tt = tq[sl * 4];
+                const uint4 xs = make_uint4(x.x, x.z, x.y, x.w);
+                mma_bf16_m16n8k16(cn[0], x, xs.x, xs.y);
+                mma_bf16_m16n8k16(cn[1], x, xs.z, xs.w);
+                mma_bf16_m16n8k16(cp[0], pv, xs.x, xs.y);
+                mma_bf16_m16n8k16(cp[1], pv, xs.z, xs.w);
+                mma_bf16_m16n8k16(ct[0], x, tt.x, tt.y);
+                mma_bf16_m16n8k16(ct[1], x, tt.z, tt.w);
+            }
+        }
+    }
+    cp_async_wait<0>();
+    // the diagonal element of group g sits in the lane with q == g / 2, at column g % 2
+    if (q == (g >> 1) && has_f) {
+        const bool odd = g & 1;
+        const float nn = odd ? cn[0][1] + cn[1][3] : cn[0][0] + cn[1][2];
+        const float dp = odd ? cp[0][1] + cp[1][3] : cp[0][0] + cp[1][2];
+        const float dt = odd ? ct[0][1] + ct[1][3] : ct[0][0] + ct[1][2];
+        const size_t r = (size_t)f * N + p;
+        const float n = fmaxf(sqrtf(nn), kEps);
+        part_nrm[(size_t)p * Tn + f] = nn;
+        token_score[r] = dt / (n * tn);
+        inv_norm[r] = 1.0f / n;
+        if (f > 0) part_dot[(size_t)p * Tn + (f - 1)] = dp;       // dot of frames f-1 and f at position p
+    }
+}
+
+// Frame runs sized so that all warps are resident at once: a second, partly filled wave of
+// CTAs would cost as much time as the first.
+template <typename KernelT>
+static int seg_score_runs(KernelT kernel, size_t smem, int Tn, int N, int* frames_per_warp) {
+    if (smem > 40 * 1024)
+        METOK_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    METOK_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kFsThreads, smem));
+    const long long slots = (long long)kNumSMs * (per_sm > 0 ? per_sm : 1) * (kFsThreads / 32);
+    long long nruns = slots / N;
+    nruns = nruns < 1 ? 1 : nruns > Tn ? Tn : nruns;
+    *frames_per_warp = ceil_div(Tn, (int)nruns);
+    return METOK_OK;
+}
+
 template <typename T, int kCH>
 static int launch_seg_score(const void* feats, const void* text, int Tn, int N, int d, int k, float* sims,
                             int32_t* boundaries, int32_t* event_offsets, int32_t* frame_event,
@@ -442,14 +602,23 @@ static int launch_seg_score(const void* feats, const void* text, int Tn, int N, 
     Carver cv(ws);
     float* part_dot = cv.take<float>((size_t)N * Tn);
     float* part_nrm = cv.take<float>((size_t)N * Tn);
-    int fpw = kSegMaxRun;
-    while (fpw > 1 && (long long)N * ceil_div(Tn, fpw) < 8LL * kNumSMs) fpw >>= 1;    // 8 to 16 warps per SM
-    const int warps = N * ceil_div(Tn, fpw);
-    const size_t smem_t = (size_t)d * sizeof(float) + (size_t)(kFsThreads / 32) * d * sizeof(T);
-    if (smem_t > 40 * 1024)
-        METOK_CUDA_TRY(cudaFuncSetAttribute(seg_score_kernel<T, kCH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)smem_t));
-    {
+    int fpw = 1;
+    if constexpr (sizeof(T) == 2) {
+        const int nslice = (d / 8 + 3) / 4;
+        const size_t smem_t = (size_t)nslice * 4 * sizeof(uint4) + (size_t)(kFsThreads / 32) * kFsDepth * kFsStageBytes;
+        auto kernel = (d / 8) % 4 == 0 ? seg_score_mma_kernel<true> : seg_score_mma_kernel<false>;
+        if (smem_t > 40 * 1024)
+            METOK_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_t));
+        const int warps = N * ceil_div(Tn, kFsFrames);
+        METOK_TIMED("seg_score_kernel", st);
+        kernel<<<ceil_div(warps, kFsThreads / 32), kFsThreads, smem_t, st>>>(
+            reinterpret_cast<const __nv_bfloat16*>(feats), reinterpret_cast<const __nv_bfloat16*>(text), Tn, N, d,
+            part_dot, part_nrm, token_score, inv_norm);
+    } else {
+        const size_t smem_t = (size_t)d * sizeof(float) + (size_t)(kFsThreads / 32) * d * sizeof(T);
+        const int rc = seg_score_runs(seg_score_kernel<T, kCH>, smem_t, Tn, N, &fpw);
+        if (rc != METOK_OK) return rc;
+        const int warps = N * ceil_div(Tn, fpw);
         METOK_TIMED("seg_score_kernel", st);
         seg_score_kernel<T, kCH><<<ceil_div(warps, kFsThreads / 32), kFsThreads, smem_t, st>>>(
             reinterpret_cast<const T*>(feats), reinterpret_cast<const T*>(text), Tn, N, d, fpw, part_dot, part_nrm,
@@ -503,9 +672,7 @@ extern "C" int metok_segment_score_events(const void* feats, int dtype, int T, i
         if (nchunk <= 32 * 8) METOK_FS(float, 8);
         METOK_FS(float, 16);
     }
-    if (nchunk <= 32 * 4) METOK_FS(__nv_bfloat16, 4);
-    if (nchunk <= 32 * 8) METOK_FS(__nv_bfloat16, 8);
-    METOK_FS(__nv_bfloat16, 16);
+    METOK_FS(__nv_bfloat16, 4);                                  // the bf16 kernel has no per-width variants
 #undef METOK_FS
 }
 

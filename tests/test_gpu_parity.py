@@ -247,7 +247,8 @@ def test_prefill_prune_stress_stage1():
 
 @pytest.mark.parametrize("Hq,Hkv,Lt,dh,n_vis,vis_start,G,dtype", [
     (1, 1, 1, 64, 5, 0, 1, "f32"), (4, 2, 3, 64, 70, 2, 3, "bf16"), (6, 2, 5, 128, 333, 7, 2, "bf16"),
-    (3, 3, 9, 32, 129, 0, 4, "f32"), (8, 1, 17, 128, 1000, 64, 2, "bf16"), (2, 2, 70, 64, 64, 1, 1, "bf16")])
+    (3, 3, 9, 32, 129, 0, 4, "f32"), (8, 1, 17, 128, 1000, 64, 2, "bf16"), (2, 2, 70, 64, 64, 1, 1, "bf16"),
+    (2, 1, 4, 64, 2003, 5, 40, "bf16"), (2, 2, 3, 64, 4099, 33, 12, "f32")])
 def test_prefill_prune_ragged(Hq, Hkv, Lt, dh, n_vis, vis_start, G, dtype):
     rng = np.random.default_rng(Hq * 100 + n_vis)
     S = vis_start + n_vis + 3 + Lt                              # 3 extra non-visual tokens before the text queries
@@ -273,6 +274,33 @@ def test_prefill_prune_tied_scores_keep_lower_index():
                                 torch.from_numpy(groups).cuda(), [3, 4], 0.125)
     n = int(got["S_out"].item())
     assert got["keep_idx"][:n].cpu().tolist() == [0, 1, 2, 3, 4, 5, 7, 50, 51]
+
+
+def test_prefill_prune_thousands_of_tied_scores():
+    # far more equal scores than one bucket's candidate list holds: the search has to go on
+    # over the index part of the keys, and still take the lowest indices of each class
+    Hq, Lt, dh, n_vis, vis_start = 2, 2, 64, 5003, 6
+    S = vis_start + n_vis + Lt
+    Q = np.ones((Hq, Lt, dh), dtype=np.float32)
+    K = np.ones((1, S, dh), dtype=np.float32)
+    groups = (np.arange(n_vis) % 3).astype(np.int32)
+    budgets = [700, 0, 1500]
+    got = B.metok_prefill_prune(P.to_torch(Q, "bf16"), P.to_torch(K, "bf16"), None, vis_start, n_vis,
+                                torch.from_numpy(groups).cuda(), budgets, 0.125)
+    n = int(got["S_out"].item())
+    want = list(range(vis_start))
+    vis = sorted([vis_start + i for i in range(n_vis) if i % 3 == 0][:700] +
+                 [vis_start + i for i in range(n_vis) if i % 3 == 2][:1500])
+    want += vis + list(range(vis_start + n_vis, S))
+    assert n == len(want)
+    assert got["keep_idx"][:n].cpu().tolist() == want
+    # two score levels, the cut inside the lower one
+    K2 = K.copy()
+    K2[0, vis_start:vis_start + 300] *= 2.0
+    got = B.metok_prefill_prune(P.to_torch(Q, "bf16"), P.to_torch(K2, "bf16"), None, vis_start, n_vis,
+                                torch.zeros(n_vis, dtype=torch.int32).cuda(), [1000], 0.125)
+    n = int(got["S_out"].item())
+    assert got["keep_idx"][:n].cpu().tolist() == list(range(vis_start + 1000)) + list(range(vis_start + n_vis, S))
 
 
 # ------------------------------------------------------------- a8 a9 ------- #

@@ -38,8 +38,8 @@ constexpr int kStStages = 2;
 constexpr int kCsBM = 128;                // colsum: keys per tile
 constexpr int kCsMaxNQ = 256;             // colsum: query rows per chunk (multiple of 16)
 constexpr int kCsStages = 4;
-constexpr int kStMinTiles = 4;            // fewest key tiles a stats CTA is started for
-constexpr int kCsMinTiles = 6;            // the same for colsum
+constexpr int kStMinTiles = 2;            // fewest key tiles a stats CTA is started for
+constexpr int kCsMinTiles = 3;            // the same for colsum
 
 struct AttnMmaDims {
     int Hq, Hkv, Lt, S, vis_start, n_vis, R;

@@ -761,40 +761,24 @@ constexpr size_t kAvgSmemBytes = (size_t)kAvgStages * kAvgStageBytes + 128;
 constexpr int kAvgLong = 128;      // outputs with more members than this are split ...
 constexpr int kAvgParts = 8;       // ... over this many CTAs (fp32 partial sums, added in part order)
 constexpr int kAvgLongCap = 256;   // long outputs that get scratch for their partial sums
+constexpr int kAvgLongCtas = kNumSMs;   // CTAs that take the extra parts of the long outputs
 
+// One (output, part): the members of output c with ranks in this part's range, added in token order.
 template <typename T>
-__global__ void __launch_bounds__(kAvgThreads, 6)
-merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
-                 const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
-                 const unsigned long long* __restrict__ slot_blocks, const int32_t* __restrict__ slot_cnt,
-                 const int32_t* __restrict__ long_index, const int32_t* __restrict__ long_slot,
-                 const int32_t* __restrict__ long_counter, float* __restrict__ long_sums,
-                 int32_t* __restrict__ long_done, int long_pass, const int32_t* __restrict__ n_out,
-                 T* __restrict__ out_feats, int32_t* __restrict__ out_members, int32_t* __restrict__ status) {
+__device__ __forceinline__ void
+merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_bar, int* s_list, int* s_wtot,
+               int* s_blocks, int* s_abort_p, int* s_last_p,
+               const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
+               const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
+               const unsigned long long* __restrict__ slot_blocks, const int32_t* __restrict__ slot_cnt,
+               const int32_t* __restrict__ long_index, float* __restrict__ long_sums,
+               int32_t* __restrict__ long_done, T* __restrict__ out_feats, int32_t* __restrict__ out_members,
+               int32_t* __restrict__ status) {
     using namespace sm100;
     constexpr int VN = Vec16<T>::N;
-    extern __shared__ uint8_t avg_dyn[];
-    __shared__ __align__(8) uint64_t s_bar[kAvgStages];
-    __shared__ int s_list[kAvgList];
-    __shared__ int s_wtot[kAvgThreads / 32];
-    __shared__ int s_blocks[64];
-    __shared__ int s_abort, s_last;
-    // CTAs start in index order: take the outputs from the last one down, so that this pass
-    // begins with the rows of V that the preceding (ascending) pass left in L2
-    // An output with many members is shared by kAvgParts CTAs, each taking a range of member ranks:
-    // part 0 comes from the launch over all outputs, the other parts from a second, small launch
-    // over the outputs that booked scratch (long_pass).
-    int c, part;
-    if (!long_pass) {
-        c = *n_out - 1 - (int)blockIdx.x;
-        part = 0;
-        if (c < 0) return;
-    } else {
-        const int l = blockIdx.x / (kAvgParts - 1);
-        if (l >= min(*long_counter, kAvgLongCap)) return;
-        c = long_slot[l];
-        part = 1 + blockIdx.x % (kAvgParts - 1);
-    }
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int& s_abort = *s_abort_p;
+    int& s_last = *s_last_p;
     const int count = slot_cnt[c];
     int li = long_index[c];
     if (li >= kAvgLongCap) li = -1;                            // no scratch left: one CTA does it all
@@ -803,7 +787,6 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
     const int r_lo = part * per, r_hi = min(count, r_lo + per);
     const int e = out_event[c];
     const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nchunk = d / VN;
     const int4* assign4 = reinterpret_cast<const int4*>(assign);
     const uint32_t stage0 = (smem_u32(avg_dyn) + 127u) & ~127u;
@@ -816,13 +799,9 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
     if (tid == 0) {
         unsigned long long mm = blocks;
         for (int i = 0; mm; ++i, mm &= mm - 1) s_blocks[i] = __ffsll((long long)mm) - 1;
-        for (int j = 0; j < kAvgStages; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
-        s_abort = 0;
-        mbar_fence_init();
     }
     __syncthreads();
     volatile int* abort_flag = &s_abort;
-    uint32_t phase = 0;                                        // bit j: parity of the next completion of barrier j
     for (int cb = 0; cb < nchunk; cb += kAvgThreads * kAvgChunks) {
         const uint32_t seg_bytes = (uint32_t)min(kAvgThreads * kAvgChunks, nchunk - cb) * 16u;
         float acc[kAvgChunks][VN];
@@ -979,6 +958,63 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
             }
         }
     }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kAvgThreads, 6)
+merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
+                 const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
+                 const unsigned long long* __restrict__ slot_blocks, const int32_t* __restrict__ slot_cnt,
+                 const int32_t* __restrict__ long_index, const int32_t* __restrict__ long_slot,
+                 const int32_t* __restrict__ long_counter, float* __restrict__ long_sums,
+                 int32_t* __restrict__ long_done, int long_ctas, const int32_t* __restrict__ n_out,
+                 T* __restrict__ out_feats, int32_t* __restrict__ out_members, int32_t* __restrict__ status) {
+    using namespace sm100;
+    extern __shared__ uint8_t avg_dyn[];
+    __shared__ __align__(8) uint64_t s_bar[kAvgStages];
+    __shared__ int s_list[kAvgList];
+    __shared__ int s_wtot[kAvgThreads / 32];
+    __shared__ int s_blocks[64];
+    __shared__ int s_abort, s_last;
+    // The first long_ctas CTAs take the extra parts of the outputs with many members: such an
+    // output is shared by kAvgParts CTAs, each taking a range of member ranks; part 0 comes from
+    // the output's own CTA, the other parts are dealt round-robin to the long CTAs (booked by
+    // merge_decode, so the work is known when this kernel starts).  They come first in the grid
+    // so that they do not end up in its tail.
+    // The other CTAs start in index order and take the outputs from the last one down, so that
+    // this pass begins with the rows of V that the preceding (ascending) pass left in L2.
+    const int tid = threadIdx.x;
+    const int first_long = (int)gridDim.x - long_ctas;       // the long CTAs are the last of the grid
+    const bool long_cta = (int)blockIdx.x >= first_long;
+    int w_first, w_step, w_limit;
+    if (long_cta) {
+        w_first = (int)blockIdx.x - first_long;
+        w_step = long_ctas;
+        w_limit = min(*long_counter, kAvgLongCap) * (kAvgParts - 1);
+    } else {
+        w_first = 0; w_step = 1;
+        w_limit = (*n_out - 1 - (int)blockIdx.x) >= 0 ? 1 : 0;
+    }
+    if (w_first >= w_limit) return;
+    if (tid == 32) {                                           // not thread 0: it is busy with the block list below
+        for (int j = 0; j < kAvgStages; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
+        s_abort = 0;
+        mbar_fence_init();
+    }
+    uint32_t phase = 0;                                        // bit j: parity of the next completion of barrier j
+#define METOK_AVG_ITEM(C, PART)                                                                                     \
+    merge_avg_item<T>(C, PART, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,  \
+                      ev_lo, out_event, assign, slot_blocks, slot_cnt, long_index, long_sums, long_done, out_feats,  \
+                      out_members, status)
+    if (!long_cta) {
+        METOK_AVG_ITEM(*n_out - 1 - (int)blockIdx.x, 0);
+        return;
+    }
+    for (int wi = w_first; wi < w_limit; wi += w_step) {
+        METOK_AVG_ITEM(long_slot[wi / (kAvgParts - 1)], 1 + wi % (kAvgParts - 1));
+        __syncthreads();                                       // s_blocks and s_last are reused by the next item
+    }
+#undef METOK_AVG_ITEM
 }
 
 // --------------------------------------------------------------------------- //
@@ -1165,16 +1201,9 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
                                         (int)kAvgSmemBytes));
     {
         METOK_TIMED("merge_avg_kernel", st);
-        merge_avg_kernel<T><<<cap, kAvgThreads, kAvgSmemBytes, st>>>(
+        merge_avg_kernel<T><<<kAvgLongCtas + cap, kAvgThreads, kAvgSmemBytes, st>>>(
             feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
-            w.long_counter, w.long_sums, w.long_done, 0, n_out, out_feats, out_members, w.status);
-    }
-    METOK_LAUNCH_CHECK();
-    {
-        METOK_TIMED("merge_avg_long_kernel", st);
-        merge_avg_kernel<T><<<kAvgLongCap * (kAvgParts - 1), kAvgThreads, kAvgSmemBytes, st>>>(
-            feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
-            w.long_counter, w.long_sums, w.long_done, 1, n_out, out_feats, out_members, w.status);
+            w.long_counter, w.long_sums, w.long_done, kAvgLongCtas, n_out, out_feats, out_members, w.status);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;

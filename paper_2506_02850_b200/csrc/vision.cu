@@ -4,6 +4,7 @@
 
 #include "common.cuh"
 #include "select.cuh"
+#include "select_block.cuh"
 #include "sm100.cuh"
 #include "launchers.h"
 
@@ -394,6 +395,48 @@ event_topk_kernel(const float* __restrict__ token_score, const int32_t* __restri
     };
     for (int i = p_lo + threadIdx.x; i < p_hi; i += blockDim.x) is_key[lo + i] = flag(i) ? 1 : 0;
     cluster_compact(cx, p_lo, p_hi, flag, emit, sm);
+}
+
+// The same by one CTA per event, when the largest event a segmentation can produce fits a
+// CTA's shared memory (select_block.cuh): no cluster barriers.
+__global__ void __launch_bounds__(kBsThreads, 1)
+event_block_topk_kernel(const float* __restrict__ token_score, const int32_t* __restrict__ ev_lo, int N,
+                        const int32_t* __restrict__ ev_budget, const int32_t* __restrict__ ev_out_off,
+                        BlockSelLayout lay, uint8_t* __restrict__ is_key, int32_t* __restrict__ out_src,
+                        int32_t* __restrict__ out_event, int32_t* __restrict__ assign) {
+    __shared__ BlockSelSmem sm;
+    __shared__ int s_budget[1];
+    extern __shared__ __align__(16) unsigned char sel_dyn[];
+    const int e = blockIdx.x;
+    const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
+    const int n = hi - lo;
+    if (n <= 0) return;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_budget[0] = ev_budget[e];
+    __syncthreads();
+    const BlockSelView sel = block_sel_run(sm, sel_dyn, lay, token_score + lo, nullptr, n, 1, s_budget);
+    const int slot0 = ev_out_off[e];
+    const int n4 = (n + 3) >> 2;
+    for (int q = tid; q < n4; q += kBsThreads) {
+        const uint32_t m = sel.mask[q >> 3];
+        const int sh = (q & 7) * 4;
+        const uint32_t nib = (m >> sh) & 15u;
+        int slot = slot0 + sel.woff[q >> 3] + __popc(m & ((1u << sh) - 1u));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = q * 4 + u;
+            if (i < n) {
+                const bool key = (nib >> u) & 1u;
+                is_key[lo + i] = key ? 1 : 0;
+                if (key) {
+                    out_src[slot] = lo + i;
+                    out_event[slot] = e;
+                    assign[lo + i] = slot;
+                    ++slot;
+                }
+            }
+        }
+    }
 }
 
 // --------------------------------------------------------------------------- //
@@ -1141,12 +1184,21 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
 
     {
         // the cache is sized for the longest event there can be, the thread count for twice the mean
-        const SelectLayout lay = select_layout(1, select_items_per_cta((long long)(Tn - (k - 1)) * N));
-        const int nthreads = select_threads(select_items_per_cta(2LL * Nv / k));
-        if (lay.bytes > 32 * 1024)                        // static + dynamic beyond 48 KiB needs the opt-in
-            METOK_CUDA_TRY(cudaFuncSetAttribute(event_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                (int)lay.bytes));
-        {
+        // an event has at most Tn - (k - 1) frames
+        const BlockSelLayout bl = block_sel_layout(1, (long long)(Tn - (k - 1)) * N, 0);
+        if (bl.fits) {
+            if (bl.bytes > 32 * 1024)
+                METOK_CUDA_TRY(cudaFuncSetAttribute(event_block_topk_kernel,
+                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bl.bytes));
+            METOK_TIMED("event_topk_kernel", st);
+            event_block_topk_kernel<<<k, kBsThreads, bl.bytes, st>>>(token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off,
+                                                                     bl, w.is_key, out_src, out_event, assign);
+        } else {
+            const SelectLayout lay = select_layout(1, select_items_per_cta((long long)(Tn - (k - 1)) * N));
+            const int nthreads = select_threads(select_items_per_cta(2LL * Nv / k));
+            if (lay.bytes > 32 * 1024)                    // static + dynamic beyond 48 KiB needs the opt-in
+                METOK_CUDA_TRY(cudaFuncSetAttribute(event_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)lay.bytes));
             METOK_TIMED("event_topk_kernel", st);
             event_topk_kernel<<<k * kSelCluster, nthreads, lay.bytes, st>>>(
                 token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off, lay, w.is_key, out_src, out_event, assign);

@@ -156,7 +156,7 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
     float* s_sim = sm_f;                                   // [Tn]   (Tn-1 used)
     float* s_nrm = sm_f + Tn;                              // [Tn]
     int* s_flag = reinterpret_cast<int*>(sm_f + 2 * Tn);   // [Tn]  boundary after frame i
-    __shared__ int s_scan[1024];
+    __shared__ int s_scan[32];
     const int tid = threadIdx.x, nthr = blockDim.x;
 
     // eight lanes per frame: a lane takes the slabs 8 apart (all its loads are independent), then a
@@ -165,9 +165,20 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
         const int f = f0 + (tid >> 3), part = tid & 7;
         float a = 0.f, b = 0.f;
         if (f < Tn) {
-            for (int s = part; s < nslab; s += 8) {
-                a += part_nrm[(size_t)s * Tn + f];
-                if (f < Tn - 1) b += part_dot[(size_t)s * Tn + f];
+            const bool has_dot = f < Tn - 1;
+            constexpr int kB = 6;                           // loads in flight; the additions keep their order
+            for (int s0 = part; s0 < nslab; s0 += 8 * kB) {
+                float x[kB], y[kB];
+#pragma unroll
+                for (int u = 0; u < kB; ++u) {
+                    const int s = s0 + 8 * u;
+                    x[u] = s < nslab ? part_nrm[(size_t)s * Tn + f] : 0.f;
+                    y[u] = s < nslab && has_dot ? part_dot[(size_t)s * Tn + f] : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < kB; ++u) {
+                    if (s0 + 8 * u < nslab) { a += x[u]; b += y[u]; }
+                }
             }
         }
 #pragma unroll
@@ -202,20 +213,24 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
         s_flag[i] = flag;
     }
     __syncthreads();
-    // exclusive scan of the flags: contiguous ranges per thread, then a scan of the range totals
+    // exclusive scan of the flags: contiguous ranges per thread, a shuffle scan inside each warp,
+    // then the warps' totals
     const int per = (Tn + nthr - 1) / nthr;
     const int lo = min(Tn, tid * per), hi = min(Tn, lo + per);
     int local = 0;
     for (int i = lo; i < hi; ++i) local += s_flag[i];
-    s_scan[tid] = local;
-    __syncthreads();
-    for (int off = 1; off < nthr; off <<= 1) {
-        const int v = (tid >= off) ? s_scan[tid - off] : 0;
-        __syncthreads();
-        s_scan[tid] += v;
-        __syncthreads();
+    const int lane = tid & 31, warp = tid >> 5;
+    int incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
     }
-    int run = s_scan[tid] - local;                         // boundaries before frame lo
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    int before = 0;
+    for (int w = 0; w < warp; ++w) before += s_scan[w];
+    int run = before + incl - local;                       // boundaries before frame lo
     for (int i = lo; i < hi; ++i) {
         frame_event[i] = run;                              // event id = boundaries strictly before i
         if (s_flag[i] && run < nb) {                       // (NaN similarities could over-flag)

@@ -130,11 +130,24 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
     // frame_score[f] = mean of the frame's N token scores; eight lanes per frame (a lane's loads are
     // independent), fixed shuffle tree; the scores stay in shared memory for the event loops below
     float* s_frame = s_score + k;           // [Tn]
+    int* s_evlo = reinterpret_cast<int*>(s_frame + Tn);     // [k] first frame of the event, clamped
+    int* s_evhi = s_evlo + k;                                // [k] one past its last frame
+    int* s_bud = s_evhi + k;                                 // [k] budget of the event
+    unsigned char* s_key = reinterpret_cast<unsigned char*>(s_bud + k);   // [k]
     for (int f0 = 0; f0 < Tn; f0 += nthr >> 3) {
         const int f = f0 + (tid >> 3), part = tid & 7;
         float s = 0.f;
-        if (f < Tn)
-            for (int p = part; p < pp.N; p += 8) s += token_score[(size_t)f * pp.N + p];
+        if (f < Tn) {
+            constexpr int kB = 6;                           // loads in flight; the additions keep their order
+            for (int p0 = part; p0 < pp.N; p0 += 8 * kB) {
+                float x[kB];
+#pragma unroll
+                for (int u = 0; u < kB; ++u) x[u] = p0 + 8 * u < pp.N ? token_score[(size_t)f * pp.N + p0 + 8 * u] : 0.f;
+#pragma unroll
+                for (int u = 0; u < kB; ++u)
+                    if (p0 + 8 * u < pp.N) s += x[u];
+            }
+        }
 #pragma unroll
         for (int o = 4; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
         if (f < Tn && part == 0) {
@@ -148,6 +161,8 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
         int hi = min(max(event_offsets[e + 1], lo), Tn);
         ev_lo[e] = lo;
         if (e == k - 1) ev_lo[k] = hi;
+        s_evlo[e] = lo;
+        s_evhi[e] = hi;
         float s;
         if (hi <= lo) {
             s = -3.0e38f;
@@ -172,34 +187,32 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
             rank += (w > v) || (w == v && j < e);
         }
         event_is_key[e] = (uint8_t)(rank < pp.n_key_events);
+        s_key[e] = (unsigned char)(rank < pp.n_key_events);
     }
     __syncthreads();
     if (pp.mode == METOK_MODE_TOPK_MERGE) {
         for (int e = tid; e < k; e += nthr) {
-            const int lo = min(max(event_offsets[e], 0), Tn);
-            const int hi = min(max(event_offsets[e + 1], lo), Tn);
-            const int m = (hi - lo) * pp.N;
-            const double ratio = event_is_key[e] ? pp.keep_key : pp.keep_nonkey;
+            const int m = (s_evhi[e] - s_evlo[e]) * pp.N;
+            const double ratio = s_key[e] ? pp.keep_key : pp.keep_nonkey;
             const double c = ratio * (double)m - 1e-9;
             long long b = (long long)c;
             if ((double)b < c) b += 1;
             if (b < 1) b = 1;
             if (b > m) b = m;
             ev_budget[e] = (int)b;
+            s_bud[e] = (int)b;
         }
         __syncthreads();
-        if (tid == 0) {
+        if (tid == 0) {                                     // everything it reads is in shared memory
             int slots = 0, tiles = 0, units = 0;
             for (int e = 0; e < k; ++e) {
                 ev_out_off[e] = slots;
                 ev_tile_off[e] = tiles;
                 ev_unit_off[e] = units;
-                const int lo = min(max(event_offsets[e], 0), Tn);
-                const int hi = min(max(event_offsets[e + 1], lo), Tn);
-                slots += ev_budget[e];
-                const int t = ((hi - lo) * pp.N + pp.tile_rows - 1) / pp.tile_rows;
+                slots += s_bud[e];
+                const int t = ((s_evhi[e] - s_evlo[e]) * pp.N + pp.tile_rows - 1) / pp.tile_rows;
                 tiles += t;
-                units += t * ((ev_budget[e] + pp.chunk_cols - 1) / pp.chunk_cols);   // row tiles x key chunks
+                units += t * ((s_bud[e] + pp.chunk_cols - 1) / pp.chunk_cols);   // row tiles x key chunks
             }
             ev_out_off[k] = slots;
             ev_tile_off[k] = tiles;
@@ -1159,12 +1172,13 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     pp.grid = 1;
     while (pp.grid * pp.grid < N) ++pp.grid;
     pp.s1 = p->s1; pp.s2 = p->s2; pp.s1_nonkey = p->s1_nonkey; pp.s2_nonkey = p->s2_nonkey;
-    if ((size_t)(k + Tn) * sizeof(float) > 40 * 1024)
+    const size_t plan_smem = (size_t)(k + Tn) * sizeof(float) + (size_t)k * (3 * sizeof(int) + 1);
+    if (plan_smem > 40 * 1024)
         METOK_CUDA_TRY(cudaFuncSetAttribute(event_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)((size_t)(k + Tn) * sizeof(float))));
+                                            (int)plan_smem));
     {
         METOK_TIMED("event_plan_kernel", st);
-        event_plan_kernel<<<1, 1024, (size_t)(k + Tn) * sizeof(float), st>>>(token_score, frame_score, event_offsets, pp, event_score,
+        event_plan_kernel<<<1, 1024, plan_smem, st>>>(token_score, frame_score, event_offsets, pp, event_score,
                                                                   event_is_key, w.ev_lo, w.ev_budget, w.ev_out_off,
                                                                   w.ev_tile_off, w.ev_unit_off, w.frame_ev,
                                                                   w.frame_stride, w.frame_off, n_out);

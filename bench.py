@@ -42,11 +42,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # captures (profiles/), keyed by (kernel, workload); absent -> null in the JSON line.
 NCU_TRAFFIC_BYTES = {
     # profiles/kernel_sections_frames128.txt; averages over a step's launches of the kernel
-    ("class_topk_kernel", "frames128"): 0.17e6,
-    ("merge_assign_mma_kernel", "frames128"): 163.9e6,
-    ("seg_partial_kernel", "frames128"): 139.1e6,
-    ("tok_score_kernel", "frames128"): 135.7e6,
-    ("kv_copy_kernel", "frames128"): 100.3e6,
+    ("class_topk_kernel", "frames128"): 0.14e6,
+    ("merge_assign_mma_kernel", "frames128"): 163.1e6,
+    ("merge_avg_kernel", "frames128"): 149.2e6,
+    ("seg_score_kernel", "frames128"): 136.0e6,
+    ("tok_score_kernel", "frames128"): 136.4e6,
+    ("kv_copy_kernel", "frames128"): 101.4e6,
+    ("gather_rows_kernel", "frames128"): 23.2e6,
+    ("gather_key_rows_kernel", "frames128"): 26.6e6,
     ("attn_stats_mma_kernel", "frames128"): 9.9e6,
     ("attn_colsum_mma_kernel", "frames128"): 10.1e6,
 }
@@ -526,16 +529,34 @@ def main():
     ms_per_step = total_ms / args.steps
     value = replica_throughput(cfg.Nv * n_videos, world, ms_per_step)
 
-    # per-kernel times: the same K steps again with the library's event brackets on
+    # per-kernel times: one video's step with the library's event brackets on.  Captured in a CUDA
+    # graph the brackets are event-record nodes, so a replay times the kernels as they run in the
+    # timed region (no host launch gap inside a bracket); eager launches otherwise.
     barrier()
+    prof_steps = max(1, min(args.steps, 100))
     B.metok_profile_begin()
-    for _ in range(args.steps):
-        wl.step()
-    prof = B.metok_profile_end()
-    launches_per_step = sum(v["launches"] for v in prof.values()) // args.steps
+    if not args.no_graph:
+        graph_prof = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_prof):
+            wl.step()
+        prof = {}
+        for _ in range(prof_steps):
+            graph_prof.replay()
+            torch.cuda.synchronize()
+            for k_, v in B.metok_profile_read().items():
+                ent = prof.setdefault(k_, {"launches": 0, "ms": 0.0})
+                ent["launches"] += v["launches"]
+                ent["ms"] += v["ms"]
+        del graph_prof
+        B.metok_profile_end()
+    else:
+        for _ in range(prof_steps):
+            wl.step()
+        prof = B.metok_profile_end()
+    launches_per_step = sum(v["launches"] for v in prof.values()) // prof_steps
     work = wl.algorithmic_work()
     peaks = load_peaks()
-    kern_ms = {k_: v["ms"] / args.steps for k_, v in prof.items()}
+    kern_ms = {k_: v["ms"] / prof_steps for k_, v in prof.items()}
     top = max(kern_ms, key=kern_ms.get)
     bound, units = work.get(top, ("hbm", float("nan")))
     if bound == "tensor":
@@ -551,7 +572,7 @@ def main():
                 "per_kernel": {}}
     for k_, ms in sorted(kern_ms.items(), key=lambda kv: -kv[1]):
         bd, u = work.get(k_, (None, None))
-        ent = {"ms": round(ms, 5), "launches": prof[k_]["launches"] // args.steps}
+        ent = {"ms": round(ms, 5), "launches": prof[k_]["launches"] // prof_steps}
         if bd == "tensor":
             ent["TFLOP/s"] = round(u / (ms * 1e-3) / 1e12, 2)
             ent["frac"] = round(ent["TFLOP/s"] / float(peaks["bf16_tflops_sustained"]), 4)

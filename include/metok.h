@@ -314,8 +314,16 @@ METOK_API int metok_kv_compact(void* const* k_layers, void* const* v_layers, int
  * in first-launch order, into `out` (HOST, `cap` bytes, NUL-terminated; truncated
  * if too small).  Returns the number of kernel launches recorded, or a negative
  * status.  Not thread-safe against concurrent calls into the library; adds two
- * event records per launch, so never leave it on outside a measurement. */
+ * event records per launch, so never leave it on outside a measurement.
+ * Calls made while their stream is being captured into a CUDA graph put the
+ * brackets into the graph as event-record nodes: every replay of the graph then
+ * times its kernels without the host's launch gaps.  metok_profile_read stops
+ * bracketing further launches and reports like metok_profile_end but keeps the
+ * events, so that the graph can be replayed and read again; metok_profile_end
+ * releases them (destroy the graph first).  The paper has no counterpart of
+ * these three calls. */
 METOK_API int metok_profile_begin(void);
+METOK_API int metok_profile_read(char* out, size_t cap);
 METOK_API int metok_profile_end(char* out, size_t cap);
 
 METOK_API const char* metok_status_string(int status);

@@ -61,6 +61,7 @@ _SIGNATURES = {
     "metok_kv_compact": (_i, [_c.POINTER(_vp), _c.POINTER(_vp), _i, _i, _i, _i, _i, _i, _i, _i, _d, _i, _i,
                               _vp, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "metok_profile_begin": (_i, []),
+    "metok_profile_read": (_i, [_c.c_char_p, _sz]),
     "metok_profile_end": (_i, [_c.c_char_p, _sz]),
     "metok_status_string": (_c.c_char_p, [_i]),
     "metok_last_cuda_error": (_i, []),
@@ -348,14 +349,23 @@ def metok_profile_begin() -> None:
     _check("metok_profile_begin", lib().metok_profile_begin())
 
 
-def metok_profile_end() -> Dict[str, Dict[str, float]]:
-    """{kernel name: {"launches": n, "ms": total}} for the launches since metok_profile_begin."""
+def _profile(fn_name: str) -> Dict[str, Dict[str, float]]:
     buf = _c.create_string_buffer(1 << 16)
-    n = lib().metok_profile_end(buf, len(buf))
+    n = getattr(lib(), fn_name)(buf, len(buf))
     if n < 0:
-        _check("metok_profile_end", n)
+        _check(fn_name, n)
     out: Dict[str, Dict[str, float]] = {}
     for line in buf.value.decode().splitlines():
         name, cnt, ms = line.split()
         out[name] = {"launches": int(cnt), "ms": float(ms)}
     return out
+
+
+def metok_profile_read() -> Dict[str, Dict[str, float]]:
+    """Like metok_profile_end, but keeps the brackets: for replays of a graph that captured them."""
+    return _profile("metok_profile_read")
+
+
+def metok_profile_end() -> Dict[str, Dict[str, float]]:
+    """{kernel name: {"launches": n, "ms": total}} for the launches since metok_profile_begin."""
+    return _profile("metok_profile_end")

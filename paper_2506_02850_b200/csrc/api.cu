@@ -22,11 +22,20 @@ std::mutex g_mu;
 KernelTimer::KernelTimer(const char* n, cudaStream_t s) : name(n), st(s), a(nullptr), b(nullptr), active(g_profiling) {
     if (!active) return;
     if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { active = false; return; }
-    cudaEventRecord(a, st);
+    record(a);
+}
+// On a stream that is being captured the bracket becomes an event-record node of the graph, so that a
+// replay of the graph times its kernels without the host's launch gaps between them.
+void KernelTimer::record(cudaEvent_t e) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusActive)
+        cudaEventRecordWithFlags(e, st, cudaEventRecordExternal);
+    else
+        cudaEventRecord(e, st);
 }
 KernelTimer::~KernelTimer() {
     if (!active) return;
-    cudaEventRecord(b, st);
+    record(b);
     std::lock_guard<std::mutex> lk(g_mu);
     g_recs.push_back({name, a, b});
 }
@@ -68,7 +77,8 @@ extern "C" int metok_profile_begin(void) {
     return METOK_OK;
 }
 
-extern "C" int metok_profile_end(char* out, size_t cap) {
+// Elapsed times of all recorded brackets, one line per kernel name; `release` destroys the events.
+static int profile_collect(char* out, size_t cap, bool release) {
     metok::g_profiling = false;
     std::lock_guard<std::mutex> lk(metok::g_mu);
     struct Agg { const char* name; int n; double ms; };
@@ -85,10 +95,12 @@ extern "C" int metok_profile_end(char* out, size_t cap) {
         for (auto& g : agg)
             if (std::strcmp(g.name, r.name) == 0) { g.n += 1; g.ms += ms; found = true; break; }
         if (!found) agg.push_back({r.name, 1, (double)ms});
-        cudaEventDestroy(r.a);
-        cudaEventDestroy(r.b);
+        if (release) {
+            cudaEventDestroy(r.a);
+            cudaEventDestroy(r.b);
+        }
     }
-    metok::g_recs.clear();
+    if (release) metok::g_recs.clear();
     if (out && cap > 0) {
         std::string text;
         char line[256];
@@ -102,6 +114,9 @@ extern "C" int metok_profile_end(char* out, size_t cap) {
     }
     return launches;
 }
+
+extern "C" int metok_profile_read(char* out, size_t cap) { return profile_collect(out, cap, false); }
+extern "C" int metok_profile_end(char* out, size_t cap) { return profile_collect(out, cap, true); }
 
 extern "C" const char* metok_status_string(int status) {
     switch (status) {

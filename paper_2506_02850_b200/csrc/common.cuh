@@ -35,6 +35,7 @@ struct KernelTimer {
     bool active;
     KernelTimer(const char* n, cudaStream_t s);
     ~KernelTimer();
+    void record(cudaEvent_t e);
 };
 #define METOK_TIMED(name, st) ::metok::KernelTimer _metok_kt(name, st)
 

@@ -289,6 +289,7 @@ class_topk_kernel(const float* __restrict__ scores, size_t score_stride, const i
     }
 }
 
+template <bool kOne>                     // kOne: one class and no class array
 __global__ void __launch_bounds__(kBsThreads, 1)
 block_topk_kernel(const float* __restrict__ scores, size_t score_stride, const int32_t* __restrict__ token_group,
                   int n_vis, int G, BlockSelLayout lay, TopkBudgets budgets, int S, int vis_start,
@@ -300,7 +301,7 @@ block_topk_kernel(const float* __restrict__ scores, size_t score_stride, const i
     const float* sc = scores + (size_t)problem * score_stride;
     int32_t* keep = keep_idx + (size_t)problem * keep_stride;
     const int tid = threadIdx.x;
-    const BlockSelView sel = block_sel_run(sm, sel_dyn, lay, sc, token_group, n_vis, G, budgets.v);
+    const BlockSelView sel = block_sel_run<kOne>(sm, sel_dyn, lay, sc, kOne ? nullptr : token_group, n_vis, G, budgets.v);
     const uint32_t* mask = sel.mask;
     const int* woff = sel.woff;
     const int kept = sel.kept;
@@ -323,11 +324,9 @@ block_topk_kernel(const float* __restrict__ scores, size_t score_stride, const i
     }
     __syncthreads();
     const int total = vis_start + kept + (S - vis_end);
-    for (int r = 0; r < replicas; ++r) {
-        int32_t* out = keep + (size_t)r * keep_stride;
-        for (int i = tid; i < vis_start; i += kBsThreads) out[i] = i;
-        for (int i = tid; i < kept; i += kBsThreads) out[vis_start + i] = packed[i];
-        for (int i = tid; i < S - vis_end; i += kBsThreads) out[vis_start + kept + i] = vis_end + i;
+    for (int i = tid; i < total; i += kBsThreads) {
+        const int v = i < vis_start ? i : i < vis_start + kept ? packed[i - vis_start] : vis_end + (i - vis_start - kept);
+        for (int r = 0; r < replicas; ++r) keep[(size_t)r * keep_stride + i] = v;
     }
     for (int r = tid; r < replicas; r += kBsThreads) {
         if (count_a) count_a[problem + r] = total;
@@ -343,14 +342,13 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
     // problems whose keys fit one CTA's shared memory skip the cluster and its barriers
     const BlockSelLayout bl = block_sel_layout(G, n_vis, S);
     if (bl.fits) {
+        auto kernel = (G == 1 && !token_group) ? block_topk_kernel<true> : block_topk_kernel<false>;
         if (bl.bytes > 32 * 1024)
-            METOK_CUDA_TRY(cudaFuncSetAttribute(block_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                (int)bl.bytes));
+            METOK_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bl.bytes));
         {
             METOK_TIMED("class_topk_kernel", st);
-            block_topk_kernel<<<problems, kBsThreads, bl.bytes, st>>>(scores, score_stride, token_group, n_vis, G, bl,
-                                                                      b, S, vis_start, keep_idx, keep_stride, replicas,
-                                                                      count_a, count_b);
+            kernel<<<problems, kBsThreads, bl.bytes, st>>>(scores, score_stride, token_group, n_vis, G, bl, b, S,
+                                                           vis_start, keep_idx, keep_stride, replicas, count_a, count_b);
         }
         METOK_LAUNCH_CHECK();
         return METOK_OK;

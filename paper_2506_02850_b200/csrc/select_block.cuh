@@ -176,6 +176,9 @@ struct BlockSelView {
     int kept;
 };
 
+// kOne: a single class and no class array (token_group is null): the class bytes are neither
+// loaded, stored nor read back.
+template <bool kOne>
 __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned char* sel_dyn, const BlockSelLayout& lay,
                                                       const float* __restrict__ sc,
                                                       const int32_t* __restrict__ token_group, int n_vis, int G,
@@ -187,6 +190,13 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
     uint32_t* keys = reinterpret_cast<uint32_t*>(sel_dyn + lay.keys_off);
     unsigned char* cls = sel_dyn + lay.cls_off;
     const int n4 = (n_vis + 3) >> 2;                         // items are handled four at a time
+    // the class bytes of quad q (255 = takes no part) and the class of item j
+    auto cls4 = [&](int q) -> uint32_t {
+        if (!kOne) return reinterpret_cast<const uint32_t*>(cls)[q];
+        const int left = n_vis - q * 4;                      // items of the quad that exist
+        return left >= 4 ? 0u : 0xFFFFFFFFu << (8 * left);
+    };
+    auto cls1 = [&](int j) -> int { return kOne ? 0 : (int)cls[j]; };
 
     // sweep 1: the items, once: keys and classes into shared memory, and the key range
     for (int b = tid; b < G * NB; b += kBsThreads) hist[b] = 0u;
@@ -204,7 +214,7 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
                 if (vec && q * 4 + 3 < n_vis) {
                     const float4 f = *reinterpret_cast<const float4*>(sc + q * 4);
                     v[w][0] = f.x; v[w][1] = f.y; v[w][2] = f.z; v[w][3] = f.w;
-                    if (token_group) {
+                    if (!kOne && token_group) {
                         const int4 t = *reinterpret_cast<const int4*>(token_group + q * 4);
                         g[w][0] = t.x; g[w][1] = t.y; g[w][2] = t.z; g[w][3] = t.w;
                     } else {
@@ -215,7 +225,7 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
                     for (int u = 0; u < 4; ++u) {
                         const int j = q * 4 + u;
                         v[w][u] = j < n_vis ? sc[j] : 0.f;
-                        g[w][u] = j < n_vis ? (token_group ? token_group[j] : 0) : -1;
+                        g[w][u] = j < n_vis ? (!kOne && token_group ? token_group[j] : 0) : -1;
                     }
                 }
             }
@@ -236,7 +246,7 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
                     }
                 }
                 reinterpret_cast<uint4*>(keys)[q] = make_uint4(k4[0], k4[1], k4[2], k4[3]);
-                reinterpret_cast<uint32_t*>(cls)[q] = c4;
+                if (!kOne) reinterpret_cast<uint32_t*>(cls)[q] = c4;
             }
         }
     }
@@ -262,11 +272,16 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
         sm.state[g] = empty ? 0 : 1;
     }
     if (tid == 0) sm.busy = 0;
+    const int nwords = (n_vis + 31) >> 5;
+    uint32_t* mask = hist;                                   // the mask takes the histograms' place when they are done
+    int* woff = reinterpret_cast<int*>(hist) + nwords;
+    bool fast = false;
+    __syncthreads();
     if (!empty) {
         // first pass: every class has the range [mn, mx]; sweep 2 histograms bucket (key - mn) >> sh0
         for (int q = tid; q < n4; q += kBsThreads) {
             const uint4 k = reinterpret_cast<const uint4*>(keys)[q];
-            const uint32_t c4 = reinterpret_cast<const uint32_t*>(cls)[q];
+            const uint32_t c4 = cls4(q);
             const uint32_t k4[4] = {k.x, k.y, k.z, k.w};
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -277,29 +292,74 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
         __syncthreads();
         block_sel_walk(sm, hist, G, nb_log2, true, budgets);
         __syncthreads();
-        // sweep 3: the items of the buckets to collect
-        for (int q = tid; q < n4; q += kBsThreads) {
-            const uint4 k = reinterpret_cast<const uint4*>(keys)[q];
-            const uint32_t c4 = reinterpret_cast<const uint32_t*>(cls)[q];
-            const uint32_t k4[4] = {k.x, k.y, k.z, k.w};
+        if (!sm.busy) {
+            // Every class is decided or has its cut inside a small bucket: ONE more sweep marks the
+            // items above the bucket as kept and collects the items inside it; the few of those
+            // that make the cut get their bits afterwards.  A class that keeps everything has the
+            // bucket -1 (every item is above it), one that keeps nothing the largest int.
+            fast = true;
+            for (int g = tid; g < G; g += kBsThreads)
+                if (sm.state[g] != 2) sm.first_bucket[g] = sm.mode[g] == 1 ? -1 : 0x7FFFFFFF;
+            __syncthreads();
+            for (int q0 = 0; q0 < n4; q0 += kBsThreads) {
+                const int q = q0 + tid;
+                uint32_t nib = 0u;
+                if (q < n4) {
+                    const uint4 k = reinterpret_cast<const uint4*>(keys)[q];
+                    const uint32_t c4 = cls4(q);
+                    const uint32_t k4[4] = {k.x, k.y, k.z, k.w};
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t g = (c4 >> (8 * u)) & 255u;
-                if (g != 255u && (int)((k4[u] - mn) >> sh0) == sm.first_bucket[g])
-                    cand[g * kBsCand + atomicAdd(&sm.cand_n[g], 1)] = item_key64(k4[u], q * 4 + u);
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t g = (c4 >> (8 * u)) & 255u;
+                        if (g != 255u) {
+                            const int b = (int)((k4[u] - mn) >> sh0), fb = sm.first_bucket[g];
+                            nib |= (b > fb ? 1u : 0u) << u;
+                            if (b == fb) cand[g * kBsCand + atomicAdd(&sm.cand_n[g], 1)] = item_key64(k4[u], q * 4 + u);
+                        }
+                    }
+                }
+                uint32_t word = nib << (4 * (lane & 7));
+                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+                if ((lane & 7) == 0 && (q >> 3) < nwords) mask[q >> 3] = word;   // over the histograms: they are done
             }
+            __syncthreads();
+            block_sel_resolve(sm, cand, G);
+            __syncthreads();
+            for (int idx = tid; idx < G * kBsCand; idx += kBsThreads) {
+                const int g = idx / kBsCand, j = idx - g * kBsCand;
+                if (j < sm.cand_n[g] && sm.mode[g] == 2 && cand[idx] >= sm.thr[g]) {
+                    const uint32_t i = ~(uint32_t)(cand[idx] & 0xFFFFFFFFull);
+                    atomicOr(&mask[i >> 5], 1u << (i & 31u));
+                }
+            }
+        } else {
+            // sweep 3: the items of the buckets to collect
+            for (int q = tid; q < n4; q += kBsThreads) {
+                const uint4 k = reinterpret_cast<const uint4*>(keys)[q];
+                const uint32_t c4 = cls4(q);
+                const uint32_t k4[4] = {k.x, k.y, k.z, k.w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t g = (c4 >> (8 * u)) & 255u;
+                    if (g != 255u && (int)((k4[u] - mn) >> sh0) == sm.first_bucket[g])
+                        cand[g * kBsCand + atomicAdd(&sm.cand_n[g], 1)] = item_key64(k4[u], q * 4 + u);
+                }
+            }
+            __syncthreads();
+            block_sel_resolve(sm, cand, G);
+            __syncthreads();
         }
-        __syncthreads();
-        block_sel_resolve(sm, cand, G);
-        __syncthreads();
     }
+    if (!fast) {
     // classes whose first bucket held more than kBsCand items (many equal or near-equal scores)
     for (int pass = 1; pass < 16 && sm.busy; ++pass) {
         for (int b = tid; b < G * NB; b += kBsThreads) hist[b] = 0u;
         __syncthreads();
         if (tid == 0) sm.busy = 0;
         for (int j = tid; j < n_vis; j += kBsThreads) {
-            const int g = cls[j];
+            const int g = cls1(j);
             if (g != 255 && sm.state[g] == 1) {
                 const unsigned long long c = item_key64(keys[j], j);
                 const unsigned long long lo = sm.lo[g];
@@ -310,7 +370,7 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
         block_sel_walk(sm, hist, G, nb_log2, false, budgets);
         __syncthreads();
         for (int j = tid; j < n_vis; j += kBsThreads) {
-            const int g = cls[j];
+            const int g = cls1(j);
             if (g != 255 && sm.state[g] == 2) {
                 const unsigned long long c = item_key64(keys[j], j);
                 if (c >= sm.lo[g] && c <= sm.hi[g]) cand[g * kBsCand + atomicAdd(&sm.cand_n[g], 1)] = c;
@@ -328,16 +388,13 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
     }
     // sweep 4: one bit per item (kept or not), 32 items per word.  A thread decides its four
     // items; the eight lanes that share a word combine their bits with three shuffles.
-    const int nwords = (n_vis + 31) >> 5;
-    uint32_t* mask = hist;                                   // the histograms are no longer needed
-    int* woff = reinterpret_cast<int*>(hist) + nwords;
     __syncthreads();
     for (int q0 = 0; q0 < n4; q0 += kBsThreads) {
         const int q = q0 + tid;
         uint32_t nib = 0u;
         if (q < n4) {
             const uint4 k = reinterpret_cast<const uint4*>(keys)[q];
-            const uint32_t c4 = reinterpret_cast<const uint32_t*>(cls)[q];
+            const uint32_t c4 = cls4(q);
             const uint32_t k4[4] = {k.x, k.y, k.z, k.w};
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -354,6 +411,7 @@ __device__ __forceinline__ BlockSelView block_sel_run(BlockSelSmem& sm, unsigned
         word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
         word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
         if ((lane & 7) == 0 && (q >> 3) < nwords) mask[q >> 3] = word;
+    }
     }
     __syncthreads();
     // exclusive offsets of the words: a thread per word, the warps' totals scanned by warp 0

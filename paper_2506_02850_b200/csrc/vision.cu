@@ -427,7 +427,7 @@ event_block_topk_kernel(const float* __restrict__ token_score, const int32_t* __
     const int tid = threadIdx.x;
     if (tid == 0) s_budget[0] = ev_budget[e];
     __syncthreads();
-    const BlockSelView sel = block_sel_run(sm, sel_dyn, lay, token_score + lo, nullptr, n, 1, s_budget);
+    const BlockSelView sel = block_sel_run<true>(sm, sel_dyn, lay, token_score + lo, nullptr, n, 1, s_budget);
     const int slot0 = ev_out_off[e];
     const int n4 = (n + 3) >> 2;
     for (int q = tid; q < n4; q += kBsThreads) {

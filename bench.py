@@ -267,7 +267,11 @@ class Workload:
             "gather_rows_kernel": ("hbm", hidden_bytes),
             "gather_key_rows_kernel": ("hbm", 2.0 * n_out * d * b),
             "kv_copy_kernel": ("hbm", 2.0 * kv_rows * cfg.dh * b * 2 * cfg.Hkv * cfg.L),
-            "class_topk_kernel": ("hbm", 8.0 * (sum(s["n_vis"] for s in self.stages) + cfg.L * cfg.Nv)),
+            # scores and classes read once per level, scores once for the K/V lists; the lists written
+            "class_topk_kernel": ("hbm", 8.0 * sum(s["n_vis"] for s in self.stages) + 4.0 * Nv
+                                  + 4.0 * sum(cfg.Lt + sum(min(bg, int((s["groups"] == g).sum().item()))
+                                                           for g, bg in enumerate(s["budgets"])) for s in self.stages)
+                                  + 4.0 * cfg.L * kv_rows),
             "event_topk_kernel": ("hbm", 8.0 * Nv),
         }
         return work
@@ -570,6 +574,23 @@ def main():
                 "traffic": NCU_TRAFFIC_BYTES.get((top, cfg.name)),
                 "ms_per_step_in_kernel": kern_ms[top],
                 "per_kernel": {}}
+    # every bracket costs the same few microseconds on top of its kernel (two event nodes): what the
+    # brackets add up to beyond the step's own time, per launch
+    roofline["bracket_overhead_us_per_launch"] = (
+        max(0.0, sum(kern_ms.values()) - ms_one_video) * 1e3 / max(1, launches_per_step) if not partial else None)
+    if units < 1e6:
+        # the selection kernels touch a few hundred KB on one SM: their time is instruction issue and
+        # barriers, and an HBM fraction says nothing about them.  The largest kernel that streams data:
+        big = {k_: ms for k_, ms in kern_ms.items() if work.get(k_, (None, 0.0))[1] >= 1e6}
+        if big:
+            k2 = max(big, key=big.get)
+            b2, u2 = work[k2]
+            a2 = u2 / (kern_ms[k2] * 1e-3) / (1e12 if b2 == "tensor" else 1e9)
+            p2 = float(peaks["bf16_tflops_sustained"] if b2 == "tensor" else peaks["hbm_gbs"])
+            roofline["note"] = "top kernel by share is a one-SM selection; see largest_streaming_kernel"
+            roofline["largest_streaming_kernel"] = {
+                "kernel": k2, "bound": b2, "achieved": a2, "peak": p2, "unit": "TFLOP/s" if b2 == "tensor" else "GB/s",
+                "frac": a2 / p2, "traffic": NCU_TRAFFIC_BYTES.get((k2, cfg.name)), "ms_per_step_in_kernel": kern_ms[k2]}
     for k_, ms in sorted(kern_ms.items(), key=lambda kv: -kv[1]):
         bd, u = work.get(k_, (None, None))
         ent = {"ms": round(ms, 5), "launches": prof[k_]["launches"] // prof_steps}

@@ -293,24 +293,6 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tmem_alloc(smem_u32(&s_tmem_base), 512);
         tmem_relinquish();
     }
-    // log-sum-exp of every query row of the chunk from the key-split partials, fixed order
-    {
-        const int ns2 = dm.st_nsplit * 2;
-        for (int c = threadIdx.x; c < kCsMaxNQ; c += kAmThreads) {
-            const int r = chunk * NQ + c;
-            float nl = kNegInf;                                // rows past R contribute exp2(x - 3e38) = 0
-            if (c < NQ && r < dm.R) {
-                const float* pm = part_m + (size_t)g * ns2 * dm.R + r;
-                const float* pl = part_l + (size_t)g * ns2 * dm.R + r;
-                float M = kNegInf;
-                for (int s = 0; s < ns2; ++s) M = fmaxf(M, pm[(size_t)s * dm.R]);
-                float Z = 0.f;
-                for (int s = 0; s < ns2; ++s) Z += pl[(size_t)s * dm.R] * exp2f(pm[(size_t)s * dm.R] - M);
-                nl = -(M + log2f(Z));
-            }
-            s_nlse[c] = nl;
-        }
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -370,6 +352,38 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
         }
     } else {
+        // The epilogue warps first turn the key-split partials into the log-sum-exp of the chunk's
+        // query rows, one row per thread, while the producer's first copies and the first MMA are
+        // already under way; nobody else reads s_nlse, so a barrier among these 256 threads is enough.
+        {
+            const int c = threadIdx.x - 64;                    // 0 .. kCsMaxNQ - 1
+            const int r = chunk * NQ + c;
+            float nl = kNegInf;                                // rows past R contribute exp2(x - 3e38) = 0
+            if (c < NQ && r < dm.R) {
+                const int ns2 = dm.st_nsplit * 2;
+                const float* pm = part_m + (size_t)g * ns2 * dm.R + r;
+                const float* pl = part_l + (size_t)g * ns2 * dm.R + r;
+                float M = kNegInf, Z = 0.f;                    // running maximum and sum, partials in order
+                for (int s0 = 0; s0 < ns2; s0 += 8) {
+                    float m8[8], l8[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const bool in = s0 + u < ns2;
+                        m8[u] = in ? pm[(size_t)(s0 + u) * dm.R] : kNegInf;
+                        l8[u] = in ? pl[(size_t)(s0 + u) * dm.R] : 0.f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const float Mn = fmaxf(M, m8[u]);
+                        Z = Z * exp2f(M - Mn) + l8[u] * exp2f(m8[u] - Mn);
+                        M = Mn;
+                    }
+                }
+                nl = -(M + log2f(Z));
+            }
+            s_nlse[c] = nl;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+        }
         const int quad = warp & 3;
         const int half = (warp - 2) >> 2;
         const int h0 = ((NQ / 16 + 1) / 2) * 16;               // first column of the second half

@@ -96,6 +96,10 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     __shared__ int s_abort;
 
     const int split = blockIdx.x, rt = blockIdx.y, g = blockIdx.z;
+    // The call's status word starts cleared: written by the first CTA of the call's first kernel
+    // instead of by a memset node.  A CTA that gives up writes it only after its waits have run
+    // out, seconds later.
+    if (split == 0 && rt == 0 && g == 0 && threadIdx.x == 0) *status = 0;
     const int t_lo = split * dm.st_per;
     const int nt = min(dm.st_tiles, t_lo + dm.st_per) - t_lo;          // >= 1 by construction
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

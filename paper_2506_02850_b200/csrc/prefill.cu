@@ -611,7 +611,7 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
     const bool mma = use_mma_attn(dtype, dh);
     Carver cv(ws);
     PrefillWs w = carve_prefill(cv, dm, mma);
-    METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
+    if (!mma) METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));   // else attn_stats_mma_kernel clears it
     int rc;
     if (mma) {
         rc = launch_attn_scores_mma(q_text, k_all, Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale, w.part_m,

@@ -115,6 +115,27 @@ struct PlanParams {
     double keep_key, keep_nonkey, beta;
 };
 
+// The workspace regions that later kernels of the call expect cleared: written here, at the start of
+// the call's first kernel, instead of by separate memset nodes (each costs the chain a launch).
+struct PlanClears {
+    void* zero_a; size_t zero_a_bytes;      // packed argmax per token (tensor-core path), may be null
+    void* zero_b; size_t zero_b_bytes;      // member bits, member counts, long-list counters
+    void* ones;   size_t ones_bytes;        // output -> long-list index, all bits set = none
+    int32_t* status;                        // device status word
+};
+// part `part` of `parts` of the fill; p 16-byte aligned, bytes % 4 == 0
+__device__ __forceinline__ void block_fill(void* p, size_t bytes, uint32_t word, int part, int parts) {
+    if (!p) return;
+    uint4* q = reinterpret_cast<uint4*>(p);
+    const size_t n16 = bytes / 16;
+    for (size_t i = (size_t)part * blockDim.x + threadIdx.x; i < n16; i += (size_t)parts * blockDim.x)
+        q[i] = make_uint4(word, word, word, word);
+    uint32_t* t = reinterpret_cast<uint32_t*>(q + n16);
+    if (part == 0)
+        for (size_t i = threadIdx.x; i < (bytes - n16 * 16) / 4; i += blockDim.x) t[i] = word;
+}
+constexpr int kPlanFillCtas = 8;
+
 __global__ void __launch_bounds__(1024)
 event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ frame_score,
                   const int32_t* __restrict__ event_offsets, PlanParams pp,
@@ -122,8 +143,15 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
                   int32_t* __restrict__ ev_lo, int32_t* __restrict__ ev_budget, int32_t* __restrict__ ev_out_off,
                   int32_t* __restrict__ ev_tile_off, int32_t* __restrict__ ev_unit_off,
                   int32_t* __restrict__ frame_ev, int32_t* __restrict__ frame_stride,
-                  int32_t* __restrict__ frame_off, int32_t* __restrict__ n_out) {
+                  int32_t* __restrict__ frame_off, int32_t* __restrict__ n_out, PlanClears clr) {
     extern __shared__ float s_score[];      // [k]
+    if (blockIdx.x > 0) {                   // CTAs 1 .. kPlanFillCtas only clear; CTA 0 plans
+        block_fill(clr.zero_a, clr.zero_a_bytes, 0u, (int)blockIdx.x - 1, kPlanFillCtas);
+        block_fill(clr.zero_b, clr.zero_b_bytes, 0u, (int)blockIdx.x - 1, kPlanFillCtas);
+        block_fill(clr.ones, clr.ones_bytes, 0xFFFFFFFFu, (int)blockIdx.x - 1, kPlanFillCtas);
+        return;
+    }
+    if (threadIdx.x == 0) *clr.status = 0;
     __shared__ int s_scan[1024];
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int k = pp.k, Tn = pp.Tn;
@@ -1147,7 +1175,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     const bool mma = kBf16 && use_mma_path(d) && p->mode == METOK_MODE_TOPK_MERGE;
     Carver cv(ws);
     VisionWs w = carve_vision(cv, Tn, N, k, d, cap, mma);
-    METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
+    // (the status word and the scratch that must start cleared are written by event_plan_kernel)
 
     // Eq. 5 per token, unless the caller brings the scores and norms from metok_segment_score_events
     const float* inv_norm = p->token_inv_norm ? p->token_inv_norm : w.inv_norm;
@@ -1176,12 +1204,21 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     if (plan_smem > 40 * 1024)
         METOK_CUDA_TRY(cudaFuncSetAttribute(event_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)plan_smem));
+    PlanClears clr;
+    const bool merging = p->mode == METOK_MODE_TOPK_MERGE;
+    clr.zero_a = mma ? w.best64 : nullptr;
+    clr.zero_a_bytes = (size_t)Nv * sizeof(unsigned long long);
+    clr.zero_b = merging ? w.slot_blocks : nullptr;
+    clr.zero_b_bytes = w.zero_bytes;
+    clr.ones = merging ? w.long_index : nullptr;
+    clr.ones_bytes = ((size_t)cap + 64) * sizeof(int32_t);
+    clr.status = w.status;
     {
         METOK_TIMED("event_plan_kernel", st);
-        event_plan_kernel<<<1, 1024, plan_smem, st>>>(token_score, frame_score, event_offsets, pp, event_score,
+        event_plan_kernel<<<1 + kPlanFillCtas, 1024, plan_smem, st>>>(token_score, frame_score, event_offsets, pp, event_score,
                                                                   event_is_key, w.ev_lo, w.ev_budget, w.ev_out_off,
                                                                   w.ev_tile_off, w.ev_unit_off, w.frame_ev,
-                                                                  w.frame_stride, w.frame_off, n_out);
+                                                                  w.frame_stride, w.frame_off, n_out, clr);
     }
     METOK_LAUNCH_CHECK();
 
@@ -1235,7 +1272,6 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         if (r2 != METOK_OK) return r2;
         METOK_CUDA_TRY(cudaFuncSetAttribute(merge_assign_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)kMmaSmemBytes));
-        METOK_CUDA_TRY(cudaMemsetAsync(w.best64, 0, (size_t)Nv * sizeof(unsigned long long), st));
         {
             METOK_TIMED("merge_assign_mma_kernel", st);
             merge_assign_mma_kernel<<<kNumSMs, kMmaThreads, kMmaSmemBytes, st>>>(
@@ -1254,8 +1290,6 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         METOK_LAUNCH_CHECK();
     }
 
-    METOK_CUDA_TRY(cudaMemsetAsync(w.slot_blocks, 0, w.zero_bytes, st));
-    METOK_CUDA_TRY(cudaMemsetAsync(w.long_index, 0xFF, ((size_t)cap + 64) * sizeof(int32_t), st));
     {
         METOK_TIMED("merge_decode_kernel", st);
         merge_decode_kernel<<<ceil_div(Nv, 256), 256, 0, st>>>(mma ? w.best64 : nullptr, w.is_key, Nv, N, w.ev_lo, k,

@@ -892,16 +892,18 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
 #pragma unroll
         for (int u = 0; u < kAvgChunks; ++u) Vec16<T>::zero(acc[u]);
         int seen = 0;                                          // members met in earlier passes
-        for (int qs = 0; qs < total_q && seen < r_hi; qs += kAvgThreads * kAvgQuads) {
-            // this thread's run: kAvgQuads consecutive groups of the searched blocks
+        // a thread's run is qpt consecutive groups: as few as cover the search in one pass (most
+        // outputs have a handful of groups: one each for the first threads, nothing for the rest)
+        const int qpt = min(kAvgQuads, (total_q + kAvgThreads - 1) / kAvgThreads);
+        for (int qs = 0; qs < total_q && seen < r_hi; qs += kAvgThreads * qpt) {
             int4 a[kAvgQuads];
             int qidx[kAvgQuads], j_lo[kAvgQuads], j_hi[kAvgQuads];   // group index; the block's token range
 #pragma unroll
             for (int u = 0; u < kAvgQuads; ++u) {
-                const int qf = qs + tid * kAvgQuads + u;
+                const int qf = qs + tid * qpt + u;
                 a[u] = make_int4(-1, -1, -1, -1);
                 qidx[u] = 0; j_lo[u] = 0; j_hi[u] = 0;
-                if (qf < total_q) {
+                if (u < qpt && qf < total_q) {
                     const int bi = qf / qpb, wq = qf - bi * qpb;
                     const int st = lo + s_blocks[bi] * bt;
                     const int q = (st >> 2) + wq;
@@ -918,6 +920,7 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
             unsigned match = 0;                                // bit 4u+i: token 4*qidx[u]+i belongs to output c
 #pragma unroll
             for (int u = 0; u < kAvgQuads; ++u) {
+                if (u >= qpt) break;
                 const int j = qidx[u] * 4;
                 match |= (unsigned)(a[u].x == c && j + 0 >= j_lo[u] && j + 0 < j_hi[u]) << (4 * u + 0);
                 match |= (unsigned)(a[u].y == c && j + 1 >= j_lo[u] && j + 1 < j_hi[u]) << (4 * u + 1);

@@ -803,7 +803,8 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
                     int N, const int32_t* __restrict__ ev_lo, int k, int32_t* __restrict__ assign,
                     unsigned long long* __restrict__ slot_blocks, int32_t* __restrict__ slot_cnt,
                     int32_t* __restrict__ long_index, int32_t* __restrict__ long_slot,
-                    int32_t* __restrict__ long_counter, int long_threshold, int long_cap) {
+                    int32_t* __restrict__ long_counter, int long_threshold, int long_cap,
+                    int32_t* __restrict__ few_members, int few_cap) {
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= Nv) return;
     int slot;
@@ -818,7 +819,9 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
     atomicOr(&slot_blocks[slot], 1ull << ((row - lo) / avg_block_tokens(m)));
     // member count; the token that takes an output past the threshold books scratch for it (which
     // scratch an output gets depends on arrival order, what is computed in it does not)
-    if (atomicAdd(&slot_cnt[slot], 1) == long_threshold) {
+    const int pos = atomicAdd(&slot_cnt[slot], 1);
+    if (pos < few_cap) few_members[(size_t)slot * few_cap + pos] = row;   // the first few_cap arrivals are listed
+    if (pos == long_threshold) {
         const int l = atomicAdd(long_counter, 1);
         long_index[slot] = l;
         if (l < long_cap) long_slot[l] = slot;
@@ -842,10 +845,16 @@ constexpr int kAvgStages = 4;      // member rows in flight
 constexpr int kAvgList = 512;      // members listed at a time
 constexpr int kAvgStageBytes = kAvgThreads * kAvgChunks * 16;
 constexpr size_t kAvgSmemBytes = (size_t)kAvgStages * kAvgStageBytes + 128;
-constexpr int kAvgLong = 128;      // outputs with more members than this are split ...
-constexpr int kAvgParts = 8;       // ... over this many CTAs (fp32 partial sums, added in part order)
+constexpr int kAvgFew = 16;        // outputs with at most this many members get them listed by merge_decode
+constexpr int kAvgLong = 32;       // outputs with more members than this are split ...
+constexpr int kAvgParts = 8;       // ... over up to this many CTAs (fp32 partial sums, added in part order)
 constexpr int kAvgLongCap = 256;   // long outputs that get scratch for their partial sums
-constexpr int kAvgLongCtas = kNumSMs;   // CTAs that take the extra parts of the long outputs
+constexpr int kAvgLongCtas = kAvgLongCap * (kAvgParts - 1);   // CTAs for the parts after the first
+// parts of an output with `count` > kAvgLong members: about eight members each
+__host__ __device__ inline int avg_parts(int count) {
+    const int p = (count + 7) / 8;
+    return p < kAvgParts ? p : kAvgParts;
+}
 
 // One (output, part): the members of output c with ranks in this part's range, added in token order.
 template <typename T>
@@ -855,18 +864,22 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
                const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
                const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
                const unsigned long long* __restrict__ slot_blocks, const int32_t* __restrict__ slot_cnt,
-               const int32_t* __restrict__ long_index, float* __restrict__ long_sums,
-               int32_t* __restrict__ long_done, T* __restrict__ out_feats, int32_t* __restrict__ out_members,
+               const int32_t* __restrict__ long_index, const int32_t* __restrict__ few_members,
+               float* __restrict__ long_sums, int32_t* __restrict__ long_done, T* __restrict__ out_feats, int32_t* __restrict__ out_members,
                int32_t* __restrict__ status) {
     using namespace sm100;
     constexpr int VN = Vec16<T>::N;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int& s_abort = *s_abort_p;
     int& s_last = *s_last_p;
+    // an output with at most kAvgFew members has them listed by merge_decode (in arrival order):
+    // fetched together with the output's other data, no search of `assign`
+    const int few_tok = lane < kAvgFew ? few_members[(size_t)c * kAvgFew + lane] : 0;
     const int count = slot_cnt[c];
+    const bool few = count <= kAvgFew;
     int li = long_index[c];
     if (li >= kAvgLongCap) li = -1;                            // no scratch left: one CTA does it all
-    const int nparts = li >= 0 ? kAvgParts : 1;
+    const int nparts = li >= 0 ? avg_parts(count) : 1;
     const int per = (count + nparts - 1) / nparts;
     const int r_lo = part * per, r_hi = min(count, r_lo + per);
     const int e = out_event[c];
@@ -880,7 +893,14 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
     const int nblk = __popcll(blocks);
     const int bt = avg_block_tokens(hi - lo), qpb = bt / 4 + 1;
     const int total_q = nblk * qpb;
-    if (tid == 0) {
+    if (few) {
+        if (warp == 0) {                                       // into token order: rank = members before it
+            const int mine = lane < count ? few_tok : 0x7FFFFFFF;
+            int rank = 0;
+            for (int j = 0; j < count; ++j) rank += __shfl_sync(0xFFFFFFFFu, mine, j) < mine;
+            if (lane < count) s_list[rank] = mine;
+        }
+    } else if (tid == 0) {
         unsigned long long mm = blocks;
         for (int i = 0; mm; ++i, mm &= mm - 1) s_blocks[i] = __ffsll((long long)mm) - 1;
     }
@@ -891,6 +911,54 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
         float acc[kAvgChunks][VN];
 #pragma unroll
         for (int u = 0; u < kAvgChunks; ++u) Vec16<T>::zero(acc[u]);
+        // the listed members' rows, kAvgStages in flight, added in list order
+        auto consume = [&](int nlist) {
+        // a ring: row m goes to stage m % kAvgStages; the stage is refilled with row m + kAvgStages as
+        // soon as every thread has added row m, so kAvgStages rows stay in flight until the list ends
+        auto issue = [&](int m) {
+            const int j = m % kAvgStages;
+            const uint32_t bar = smem_u32(&s_bar[j]);
+            mbar_arrive_expect_tx(bar, seg_bytes);
+            bulk_load(stage0 + (uint32_t)j * kAvgStageBytes, feats + (size_t)s_list[m] * d + (size_t)cb * VN,
+                      seg_bytes, bar);
+        };
+        if (tid == 0)
+            for (int m = 0; m < nlist && m < kAvgStages; ++m) issue(m);
+        for (int m = 0; m < nlist; ++m) {
+            const int j = m % kAvgStages;
+            const bool ok = mbar_wait(smem_u32(&s_bar[j]), (phase >> j) & 1u, abort_flag);
+            phase ^= 1u << j;
+            if (ok) {
+                const uint8_t* row = avg_dyn + (stage0 - smem_u32(avg_dyn)) + (size_t)j * kAvgStageBytes;
+#pragma unroll
+                for (int u = 0; u < kAvgChunks; ++u) {
+                    const int ch = cb + u * kAvgThreads + tid;
+                    if (ch < nchunk) {
+                        const uint4 raw = *reinterpret_cast<const uint4*>(row + (size_t)(u * kAvgThreads + tid) * 16);
+                        float v[VN];
+                        if constexpr (sizeof(T) == 4) {
+                            v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
+                            v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+                        } else {
+                            const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                v[2 * i]     = __uint_as_float(w4[i] << 16);
+                                v[2 * i + 1] = __uint_as_float(w4[i] & 0xFFFF0000u);
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < VN; ++q) acc[u][q] += v[q];
+                    }
+                }
+            }
+            __syncthreads();                                   // every thread is done with stage j
+            if (tid == 0 && m + kAvgStages < nlist && !*abort_flag) issue(m + kAvgStages);
+        }
+        };
+        if (few) {
+            consume(count);                                    // s_list holds them already
+        } else {
         int seen = 0;                                          // members met in earlier passes
         // a thread's run is qpt consecutive groups: as few as cover the search in one pass (most
         // outputs have a handful of groups: one each for the first threads, nothing for the rest)
@@ -958,48 +1026,11 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
                     }
                 }
                 __syncthreads();
-                for (int m0 = 0; m0 < nlist; m0 += kAvgStages) {
-                    const int nr = min(kAvgStages, nlist - m0);
-                    if (tid == 0) {
-                        for (int j = 0; j < nr; ++j) {
-                            const uint32_t bar = smem_u32(&s_bar[j]);
-                            mbar_arrive_expect_tx(bar, seg_bytes);
-                            bulk_load(stage0 + (uint32_t)j * kAvgStageBytes,
-                                      feats + (size_t)s_list[m0 + j] * d + (size_t)cb * VN, seg_bytes, bar);
-                        }
-                    }
-                    for (int j = 0; j < nr; ++j) {
-                        const bool ok = mbar_wait(smem_u32(&s_bar[j]), (phase >> j) & 1u, abort_flag);
-                        phase ^= 1u << j;
-                        if (!ok) continue;
-                        const uint8_t* row = avg_dyn + (stage0 - smem_u32(avg_dyn)) + (size_t)j * kAvgStageBytes;
-#pragma unroll
-                        for (int u = 0; u < kAvgChunks; ++u) {
-                            const int ch = cb + u * kAvgThreads + tid;
-                            if (ch < nchunk) {
-                                const uint4 raw = *reinterpret_cast<const uint4*>(row + (size_t)(u * kAvgThreads + tid) * 16);
-                                float v[VN];
-                                if constexpr (sizeof(T) == 4) {
-                                    v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
-                                    v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
-                                } else {
-                                    const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                                    for (int i = 0; i < 4; ++i) {
-                                        v[2 * i]     = __uint_as_float(w4[i] << 16);
-                                        v[2 * i + 1] = __uint_as_float(w4[i] & 0xFFFF0000u);
-                                    }
-                                }
-#pragma unroll
-                                for (int q = 0; q < VN; ++q) acc[u][q] += v[q];
-                            }
-                        }
-                    }
-                    __syncthreads();                           // every thread is done with the stages
-                }
+                consume(nlist);
             }
             seen += total;
             __syncthreads();                                   // s_wtot and s_list are reused by the next pass
+        }
         }
         if (nparts == 1) {
             const float inv = 1.0f / (float)count;
@@ -1038,10 +1069,22 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
             __threadfence();
             const float inv = 1.0f / (float)count;
             const float* ps = long_sums + (size_t)li * kAvgParts * d;
-            for (int i = tid; i < d; i += kAvgThreads) {
-                float a = 0.f;
-                for (int q = 0; q < kAvgParts; ++q) a += __ldcg(ps + (size_t)q * d + i);
-                from_float(out_feats[(size_t)c * d + i], a * inv);
+            // four elements per thread and trip, the parts' loads all in flight, added in part order
+            // (d is a multiple of 4: rows are whole 16-byte chunks)
+            for (int i = tid * 4; i < d; i += kAvgThreads * 4) {
+                float4 v[kAvgParts];
+#pragma unroll
+                for (int q = 0; q < kAvgParts; ++q)
+                    v[q] = q < nparts ? __ldcg(reinterpret_cast<const float4*>(ps + (size_t)q * d + i))
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int q = 0; q < kAvgParts; ++q) {
+                    if (q < nparts) { a.x += v[q].x; a.y += v[q].y; a.z += v[q].z; a.w += v[q].w; }
+                }
+                T* o = out_feats + (size_t)c * d + i;
+                from_float(o[0], a.x * inv); from_float(o[1], a.y * inv);
+                from_float(o[2], a.z * inv); from_float(o[3], a.w * inv);
             }
         }
     }
@@ -1053,8 +1096,8 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
                  const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
                  const unsigned long long* __restrict__ slot_blocks, const int32_t* __restrict__ slot_cnt,
                  const int32_t* __restrict__ long_index, const int32_t* __restrict__ long_slot,
-                 const int32_t* __restrict__ long_counter, float* __restrict__ long_sums,
-                 int32_t* __restrict__ long_done, int long_ctas, const int32_t* __restrict__ n_out,
+                 const int32_t* __restrict__ long_counter, const int32_t* __restrict__ few_members,
+                 float* __restrict__ long_sums, int32_t* __restrict__ long_done, int long_ctas, const int32_t* __restrict__ n_out,
                  T* __restrict__ out_feats, int32_t* __restrict__ out_members, int32_t* __restrict__ status) {
     using namespace sm100;
     extern __shared__ uint8_t avg_dyn[];
@@ -1063,45 +1106,36 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
     __shared__ int s_wtot[kAvgThreads / 32];
     __shared__ int s_blocks[64];
     __shared__ int s_abort, s_last;
-    // The first long_ctas CTAs take the extra parts of the outputs with many members: such an
-    // output is shared by kAvgParts CTAs, each taking a range of member ranks; part 0 comes from
-    // the output's own CTA, the other parts are dealt round-robin to the long CTAs (booked by
-    // merge_decode, so the work is known when this kernel starts).  They come first in the grid
-    // so that they do not end up in its tail.
-    // The other CTAs start in index order and take the outputs from the last one down, so that
-    // this pass begins with the rows of V that the preceding (ascending) pass left in L2.
+    // An output with more than kAvgLong members is shared by up to kAvgParts CTAs, each taking a range
+    // of member ranks: one CTA would add its rows four at a time and hold up the end of the kernel
+    // (the longest list sets the kernel's time otherwise).  Part 0 comes from the output's own CTA;
+    // the other parts have CTAs of their own, the first long_ctas of the grid, so that they start at
+    // once (booked by merge_decode, so the work is known when this kernel starts; a CTA without work
+    // leaves right away).  The other CTAs start in index order and take the outputs from the last
+    // one down, so that this pass begins with the rows of V that the preceding (ascending) pass left
+    // in L2.
     const int tid = threadIdx.x;
-    const int first_long = (int)gridDim.x - long_ctas;       // the long CTAs are the last of the grid
-    const bool long_cta = (int)blockIdx.x >= first_long;
-    int w_first, w_step, w_limit;
-    if (long_cta) {
-        w_first = (int)blockIdx.x - first_long;
-        w_step = long_ctas;
-        w_limit = min(*long_counter, kAvgLongCap) * (kAvgParts - 1);
+    int c, part;
+    if ((int)blockIdx.x < long_ctas) {
+        const int l = (int)blockIdx.x / (kAvgParts - 1);
+        if (l >= min(*long_counter, kAvgLongCap)) return;
+        c = long_slot[l];
+        part = 1 + (int)blockIdx.x % (kAvgParts - 1);
+        if (part >= avg_parts(slot_cnt[c])) return;
     } else {
-        w_first = 0; w_step = 1;
-        w_limit = (*n_out - 1 - (int)blockIdx.x) >= 0 ? 1 : 0;
+        c = *n_out - 1 - ((int)blockIdx.x - long_ctas);
+        part = 0;
+        if (c < 0) return;
     }
-    if (w_first >= w_limit) return;
     if (tid == 32) {                                           // not thread 0: it is busy with the block list below
         for (int j = 0; j < kAvgStages; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
         s_abort = 0;
         mbar_fence_init();
     }
     uint32_t phase = 0;                                        // bit j: parity of the next completion of barrier j
-#define METOK_AVG_ITEM(C, PART)                                                                                     \
-    merge_avg_item<T>(C, PART, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,  \
-                      ev_lo, out_event, assign, slot_blocks, slot_cnt, long_index, long_sums, long_done, out_feats,  \
-                      out_members, status)
-    if (!long_cta) {
-        METOK_AVG_ITEM(*n_out - 1 - (int)blockIdx.x, 0);
-        return;
-    }
-    for (int wi = w_first; wi < w_limit; wi += w_step) {
-        METOK_AVG_ITEM(long_slot[wi / (kAvgParts - 1)], 1 + wi % (kAvgParts - 1));
-        __syncthreads();                                       // s_blocks and s_last are reused by the next item
-    }
-#undef METOK_AVG_ITEM
+    merge_avg_item<T>(c, part, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,
+                      ev_lo, out_event, assign, slot_blocks, slot_cnt, long_index, few_members, long_sums, long_done,
+                      out_feats, out_members, status);
 }
 
 // --------------------------------------------------------------------------- //
@@ -1121,6 +1155,7 @@ struct VisionWs {
     int32_t* long_done;                // ... parts of each that have finished
     int32_t* long_index;               // output -> index among the long ones, -1 otherwise
     int32_t* long_slot;                // and back
+    int32_t* few_members;              // per output token: its first kAvgFew members, in arrival order
     float* long_sums;                  // partial sums of their parts
     size_t zero_bytes;                 // slot_blocks .. long_done are cleared together
 };
@@ -1150,6 +1185,7 @@ static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, b
         w.long_done = w.long_counter + 64;
         w.long_index = cv.take<int32_t>(n);
         w.long_slot = cv.take<int32_t>(kAvgLongCap);
+        w.few_members = cv.take<int32_t>(n * kAvgFew);
         w.long_sums = cv.take<float>((size_t)kAvgLongCap * kAvgParts * d);
     }
     return w;
@@ -1297,7 +1333,8 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         METOK_TIMED("merge_decode_kernel", st);
         merge_decode_kernel<<<ceil_div(Nv, 256), 256, 0, st>>>(mma ? w.best64 : nullptr, w.is_key, Nv, N, w.ev_lo, k,
                                                                assign, w.slot_blocks, w.slot_cnt, w.long_index,
-                                                               w.long_slot, w.long_counter, kAvgLong, kAvgLongCap);
+                                                               w.long_slot, w.long_counter, kAvgLong, kAvgLongCap,
+                                                               w.few_members, kAvgFew);
     }
     METOK_LAUNCH_CHECK();
     METOK_CUDA_TRY(cudaFuncSetAttribute(merge_avg_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1306,7 +1343,8 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         METOK_TIMED("merge_avg_kernel", st);
         merge_avg_kernel<T><<<kAvgLongCtas + cap, kAvgThreads, kAvgSmemBytes, st>>>(
             feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
-            w.long_counter, w.long_sums, w.long_done, kAvgLongCtas, n_out, out_feats, out_members, w.status);
+            w.long_counter, w.few_members, w.long_sums, w.long_done, kAvgLongCtas, n_out, out_feats, out_members,
+            w.status);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;

@@ -841,7 +841,7 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
 constexpr int kAvgThreads = 128;
 constexpr int kAvgChunks = 4;      // 16-byte chunks per thread per pass over d
 constexpr int kAvgQuads = 5;       // 16-byte groups of `assign` per thread and pass
-constexpr int kAvgStages = 4;      // member rows in flight
+constexpr int kAvgStages = 3;      // member rows in flight
 constexpr int kAvgList = 512;      // members listed at a time
 constexpr int kAvgStageBytes = kAvgThreads * kAvgChunks * 16;
 constexpr size_t kAvgSmemBytes = (size_t)kAvgStages * kAvgStageBytes + 128;
@@ -1091,7 +1091,7 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kAvgThreads, 6)
+__global__ void __launch_bounds__(kAvgThreads, 8)
 merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
                  const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
                  const unsigned long long* __restrict__ slot_blocks, const int32_t* __restrict__ slot_cnt,

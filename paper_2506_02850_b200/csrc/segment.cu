@@ -159,10 +159,14 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
     __shared__ int s_scan[32];
     const int tid = threadIdx.x, nthr = blockDim.x;
 
-    // eight lanes per frame: a lane takes the slabs 8 apart (all its loads are independent), then a
-    // fixed shuffle tree over the eight; 128 frames per sweep of the CTA
-    for (int f0 = 0; f0 < Tn; f0 += nthr >> 3) {
-        const int f = f0 + (tid >> 3), part = tid & 7;
+    // The partial sums: 128 consecutive frames per sweep, eight groups of 128 threads; a group takes the
+    // slabs 8 apart, so a warp's load is 128 contiguous bytes of one slab (one CTA's L1 handles a sector
+    // per cycle: whole sectors matter), six loads in flight; the eight groups' sums are then added in
+    // group order.
+    __shared__ float s_pn[8][128], s_pd[8][128];
+    for (int f0 = 0; f0 < Tn; f0 += 128) {
+        const int fl = tid & 127, part = tid >> 7;            // nthr == 1024
+        const int f = f0 + fl;
         float a = 0.f, b = 0.f;
         if (f < Tn) {
             const bool has_dot = f < Tn - 1;
@@ -181,15 +185,17 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
                 }
             }
         }
+        s_pn[part][fl] = a;
+        s_pd[part][fl] = b;
+        __syncthreads();
+        if (tid < 128 && f < Tn) {
+            float an = 0.f, ad = 0.f;
 #pragma unroll
-        for (int o = 4; o > 0; o >>= 1) {
-            a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
-            b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
+            for (int g = 0; g < 8; ++g) { an += s_pn[g][tid]; ad += s_pd[g][tid]; }
+            s_nrm[f] = fmaxf(sqrtf(an), kEps);
+            s_sim[f] = ad;                                  // dot product for now
         }
-        if (f < Tn && part == 0) {
-            s_nrm[f] = fmaxf(sqrtf(a), kEps);
-            s_sim[f] = b;                                   // dot product for now
-        }
+        __syncthreads();
     }
     __syncthreads();
     for (int i = tid; i < Tn - 1; i += nthr) {
@@ -523,10 +529,14 @@ seg_score_mma_kernel(const __nv_bfloat16* __restrict__ feats, const __nv_bfloat1
     }
     __syncthreads();
     const float tn = s_tn;
-    const int nruns = (Tn + kFsFrames - 1) / kFsFrames;
-    const int gw = blockIdx.x * (kFsThreads / 32) + warp;   // the warp owns position p and eight frames
-    if (gw >= N * nruns) return;
-    const int p = gw % N, run = gw / N;
+    // the CTA owns eight frames and four consecutive positions, one per warp: their norms and dots are
+    // added here (in warp order), so that seg_finish has a quarter of the partial sums to read
+    constexpr int kFsWarps = kFsThreads / 32;
+    const int pgroups = (N + kFsWarps - 1) / kFsWarps;
+    const int run = blockIdx.x / pgroups, pg = blockIdx.x - run * pgroups;
+    const int p_raw = pg * kFsWarps + warp;
+    const bool has_p = p_raw < N;
+    const int p = has_p ? p_raw : N - 1;                    // an idle warp repeats the last position and writes nothing
     const int f0 = run * kFsFrames;
     const int g = lane >> 2, q = lane & 3;
     const int f = f0 + g;                                   // this lane's frame
@@ -581,17 +591,29 @@ seg_score_mma_kernel(const __nv_bfloat16* __restrict__ feats, const __nv_bfloat1
     }
     cp_async_wait<0>();
     // the diagonal element of group g sits in the lane with q == g / 2, at column g % 2
-    if (q == (g >> 1) && has_f) {
+    __shared__ float s_nn[kFsWarps][kFsFrames], s_dp[kFsWarps][kFsFrames];
+    if (q == (g >> 1)) {
         const bool odd = g & 1;
         const float nn = odd ? cn[0][1] + cn[1][3] : cn[0][0] + cn[1][2];
         const float dp = odd ? cp[0][1] + cp[1][3] : cp[0][0] + cp[1][2];
         const float dt = odd ? ct[0][1] + ct[1][3] : ct[0][0] + ct[1][2];
-        const size_t r = (size_t)f * N + p;
-        const float n = fmaxf(sqrtf(nn), kEps);
-        part_nrm[(size_t)p * Tn + f] = nn;
-        token_score[r] = dt / (n * tn);
-        inv_norm[r] = 1.0f / n;
-        if (f > 0) part_dot[(size_t)p * Tn + (f - 1)] = dp;       // dot of frames f-1 and f at position p
+        s_nn[warp][g] = has_p && has_f ? nn : 0.f;
+        s_dp[warp][g] = has_p && has_f ? dp : 0.f;
+        if (has_p && has_f) {
+            const size_t r = (size_t)f * N + p;
+            const float n = fmaxf(sqrtf(nn), kEps);
+            token_score[r] = dt / (n * tn);
+            inv_norm[r] = 1.0f / n;
+        }
+    }
+    __syncthreads();
+    if (tid < kFsFrames && f0 + tid < Tn) {
+        float nn = 0.f, dp = 0.f;
+#pragma unroll
+        for (int w = 0; w < kFsWarps; ++w) { nn += s_nn[w][tid]; dp += s_dp[w][tid]; }
+        const int ff = f0 + tid;
+        part_nrm[(size_t)pg * Tn + ff] = nn;
+        if (ff > 0) part_dot[(size_t)pg * Tn + (ff - 1)] = dp;    // dots of frames ff-1 and ff, four positions
     }
 }
 
@@ -618,15 +640,16 @@ static int launch_seg_score(const void* feats, const void* text, int Tn, int N, 
     float* part_dot = cv.take<float>((size_t)N * Tn);
     float* part_nrm = cv.take<float>((size_t)N * Tn);
     int fpw = 1;
+    int nslab = N;                                         // partial sums per frame that seg_finish adds up
     if constexpr (sizeof(T) == 2) {
         const int nslice = (d / 8 + 3) / 4;
         const size_t smem_t = (size_t)nslice * 4 * sizeof(uint4) + (size_t)(kFsThreads / 32) * kFsDepth * kFsStageBytes;
         auto kernel = (d / 8) % 4 == 0 ? seg_score_mma_kernel<true> : seg_score_mma_kernel<false>;
         if (smem_t > 40 * 1024)
             METOK_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_t));
-        const int warps = N * ceil_div(Tn, kFsFrames);
+        nslab = ceil_div(N, kFsThreads / 32);              // the kernel adds the four positions of a CTA
         METOK_TIMED("seg_score_kernel", st);
-        kernel<<<ceil_div(warps, kFsThreads / 32), kFsThreads, smem_t, st>>>(
+        kernel<<<nslab * ceil_div(Tn, kFsFrames), kFsThreads, smem_t, st>>>(
             reinterpret_cast<const __nv_bfloat16*>(feats), reinterpret_cast<const __nv_bfloat16*>(text), Tn, N, d,
             part_dot, part_nrm, token_score, inv_norm);
     } else {
@@ -645,7 +668,7 @@ static int launch_seg_score(const void* feats, const void* text, int Tn, int N, 
         METOK_CUDA_TRY(cudaFuncSetAttribute(seg_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     {
         METOK_TIMED("seg_finish_kernel", st);
-        seg_finish_kernel<<<1, 1024, smem, st>>>(part_dot, part_nrm, N, Tn, k, sims, boundaries, event_offsets,
+        seg_finish_kernel<<<1, 1024, smem, st>>>(part_dot, part_nrm, nslab, Tn, k, sims, boundaries, event_offsets,
                                              frame_event);
     }
     METOK_LAUNCH_CHECK();

@@ -67,7 +67,7 @@ def test_segment_events_ties_go_to_lower_index_and_repeatable():
         assert torch.equal(a, B.metok_segment_events(x, 4)["sims"])
 
 
-@pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128"])
+@pytest.mark.parametrize("name", ["tiny", "frames32", "frames64", "frames128", "frames128d1024", "stress"])
 def test_segment_score_events_one_pass(name):
     """Segmentation and Eq. 5 token scores from one pass over V: both against the oracle, and the
     compressor fed with them against the compressor that scores by itself."""

@@ -224,9 +224,15 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 } else {
                     // the scale is positive: the maximum of the raw logits, scaled, is the maximum of the
                     // scaled ones, and scaling folds into the exponent's multiply-add
-                    float cm = v[0];
+                    float t16[16];                             // a tree: the maximum is five steps deep, not 31
 #pragma unroll
-                    for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
+                    for (int j = 0; j < 16; ++j) t16[j] = fmaxf(v[2 * j], v[2 * j + 1]);
+#pragma unroll
+                    for (int w = 8; w >= 1; w >>= 1) {
+#pragma unroll
+                        for (int j = 0; j < w; ++j) t16[j] = fmaxf(t16[j], t16[j + w]);
+                    }
+                    const float cm = t16[0];
                     m_new = fmaxf(m_run, cm * sc);
                     const float neg_m = -m_new;
 #pragma unroll

@@ -29,6 +29,8 @@ namespace {
 
 constexpr int kAmThreads = 320;
 constexpr int kAmEpiWarps = 8;
+constexpr int kStEpiWarps = 16;           // stats: four warps per TMEM lane quadrant, 64 columns of a tile each
+constexpr int kStThreads = 64 + kStEpiWarps * 32;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegInf = -3.0e38f;       // finite stand-in: keeps (m_old - m_new) free of inf - inf
 
@@ -81,7 +83,7 @@ __host__ AttnMmaDims make_mma_dims(int Hq, int Hkv, int Lt, int S, int vis_start
 // stats
 // --------------------------------------------------------------------------- //
 template <int DH>
-__global__ void __launch_bounds__(kAmThreads, 1)
+__global__ void __launch_bounds__(kStThreads, 1)
 attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       AttnMmaDims dm, float* __restrict__ part_m, float* __restrict__ part_l,
                       int32_t* __restrict__ status) {
@@ -94,6 +96,7 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         tempty_bar[2];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ float s_pm[4][kStBM], s_pl[4][kStBM];          // the column quarters' (max, sum) per query row
 
     const int split = blockIdx.x, rt = blockIdx.y, g = blockIdx.z;
     // The call's status word starts cleared: written by the first CTA of the call's first kernel
@@ -113,7 +116,7 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         mbar_init(smem_u32(&q_bar), 1);
         mbar_init(smem_u32(&drain_bar), 1);
         for (int s = 0; s < kStStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tfull_bar[b]), 1); mbar_init(smem_u32(&tempty_bar[b]), kAmEpiWarps); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tfull_bar[b]), 1); mbar_init(smem_u32(&tempty_bar[b]), kStEpiWarps); }
         s_abort = 0;
         mbar_fence_init();
     }
@@ -182,7 +185,7 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
     } else {
         const int quad = warp & 3;                             // TMEM lanes 32*quad .. 32*quad+31
-        const int half = (warp - 2) >> 2;                      // column half of every tile
+        const int part = (warp - 2) >> 2;                      // column quarter of every tile
         const int r = rt * kStBM + quad * 32 + lane;
         const bool valid = r < dm.R;
         const int limit = valid ? text_start + (r % dm.Lt) : -1;     // last key this query may see
@@ -196,17 +199,17 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             if (!ok) break;
             tc_fence_after();
             const int u_tile = (t_lo + it) * kStBN;
-            const int u0 = u_tile + half * (kStBN / 2);
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * kStBN + half * (kStBN / 2));
+            const int u0 = u_tile + part * (kStBN / 4);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * kStBN + part * (kStBN / 4));
             const bool masked = u_tile + kStBN - 1 > text_start;       // some query cannot see some key of the tile
             uint32_t raw[2][32];
             tmem_ld32_issue(taddr, raw[0]);
 #pragma unroll
-            for (int ci = 0; ci < kStBN / 64; ++ci) {
+            for (int ci = 0; ci < kStBN / 128; ++ci) {
                 // the next 32 columns are fetched while these are reduced
                 const int c0 = ci * 32;
                 tmem_ld32_wait(raw[ci & 1]);
-                if (ci + 1 < kStBN / 64) tmem_ld32_issue(taddr + (uint32_t)(c0 + 32), raw[(ci + 1) & 1]);
+                if (ci + 1 < kStBN / 128) tmem_ld32_issue(taddr + (uint32_t)(c0 + 32), raw[(ci + 1) & 1]);
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[ci & 1][j]);
@@ -248,10 +251,21 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[b]));
         }
-        if (ok && valid) {
-            const size_t o = ((size_t)g * (dm.st_nsplit * 2) + (size_t)(split * 2 + half)) * dm.R + r;
-            part_m[o] = m_run;
-            part_l[o] = l_run;
+        // the four column quarters of a row are merged here, in quarter order: one pair per row and split
+        const int rl = quad * 32 + lane;
+        s_pm[part][rl] = m_run;
+        s_pl[part][rl] = l_run;
+        asm volatile("bar.sync 1, %0;" ::"n"(kStEpiWarps * 32) : "memory");
+        if (part == 0 && ok && valid) {
+            float M = s_pm[0][rl];
+#pragma unroll
+            for (int p2 = 1; p2 < 4; ++p2) M = fmaxf(M, s_pm[p2][rl]);
+            float Z = 0.f;
+#pragma unroll
+            for (int p2 = 0; p2 < 4; ++p2) Z += s_pl[p2][rl] * fast_exp2(s_pm[p2][rl] - M);
+            const size_t o = ((size_t)g * dm.st_nsplit + (size_t)split) * dm.R + r;
+            part_m[o] = M;
+            part_l[o] = Z;
         }
     }
     tc_fence_before();
@@ -370,7 +384,7 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             const int r = chunk * NQ + c;
             float nl = kNegInf;                                // rows past R contribute exp2(x - 3e38) = 0
             if (c < NQ && r < dm.R) {
-                const int ns2 = dm.st_nsplit * 2;
+                const int ns2 = dm.st_nsplit;                  // one (max, sum) pair per key split
                 const float* pm = part_m + (size_t)g * ns2 * dm.R + r;
                 const float* pl = part_l + (size_t)g * ns2 * dm.R + r;
                 float M = kNegInf, Z = 0.f;                    // running maximum and sum, partials in order
@@ -468,7 +482,7 @@ int launch_dh(const void* q_text, const void* k_all, const AttnMmaDims& dm, floa
                                         (int)((size_t)KB * (kCsMaxNQ + kCsStages * kCsBM) * 128 + 1024)));
     {
         METOK_TIMED("attn_stats_mma_kernel", st);
-        attn_stats_mma_kernel<DH><<<dim3(dm.st_nsplit, dm.st_nrt, dm.Hkv), kAmThreads, smem_st, st>>>(
+        attn_stats_mma_kernel<DH><<<dim3(dm.st_nsplit, dm.st_nrt, dm.Hkv), kStThreads, smem_st, st>>>(
             tmQs, tmKs, dm, part_m, part_l, status);
     }
     METOK_LAUNCH_CHECK();

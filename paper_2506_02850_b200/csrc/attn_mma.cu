@@ -8,7 +8,7 @@
 //   stats  : D = Q_tile (128 query rows = TMEM lanes) x K_tile^T (256 keys = columns).
 //            A thread owns one query row, so the running (max, sum) of the softmax is
 //            thread-local.  The keys are split over CTAs; each CTA leaves one (max,
-//            sum) pair per row and column half.
+//            sum) pair per row (the column quarters are merged in the CTA).
 //   colsum : D = K_tile (128 keys = TMEM lanes) x Q_chunk^T (up to 256 query rows =
 //            columns).  The row normalisers are known now (log-sum-exp per query row,
 //            kept in shared memory), a thread owns one key and adds up
@@ -16,9 +16,9 @@
 //            too.  Only key tiles that touch the visual span are visited.
 //
 // Warp roles in both: warp 0 = TMA producer, warp 1 = MMA issuer (one elected lane),
-// warps 2..9 = epilogue, two warps per TMEM lane quadrant, each taking half of the
-// columns.  Two accumulators in TMEM (2 x 256 columns) so that the epilogue of tile i
-// overlaps the MMA of tile i+1.  Every wait is bounded.
+// the others = epilogue: four (stats) or two (colsum) warps per TMEM lane quadrant, each
+// taking a quarter or half of the columns.  Two accumulators in TMEM (2 x 256 columns) so
+// that the epilogue of tile i overlaps the MMA of tile i+1.  Every wait is bounded.
 #include "common.cuh"
 #include "launchers.h"
 #include "sm100.cuh"

@@ -239,9 +239,11 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     m_new = fmaxf(m_run, cm * sc);
                     const float neg_m = -m_new;
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
+                    for (int j = 0; j < 32; j += 4) {           // every fourth exponential on the FMA pipe
                         a0 += fast_exp2(fmaf(v[j], sc, neg_m));
                         a1 += fast_exp2(fmaf(v[j + 1], sc, neg_m));
+                        a0 += fast_exp2(fmaf(v[j + 2], sc, neg_m));
+                        a1 += exp2_fma(fmaf(v[j + 3], sc, neg_m));
                     }
                 }
                 l_run = l_run * fast_exp2(m_run - m_new) + (a0 + a1);
@@ -435,7 +437,7 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     a0 += fast_exp2(fmaf(v[j], sc, nl.x));
                     a1 += fast_exp2(fmaf(v[j + 1], sc, nl.y));
                     a0 += fast_exp2(fmaf(v[j + 2], sc, nl.z));
-                    a1 += fast_exp2(fmaf(v[j + 3], sc, nl.w));
+                    a1 += exp2_fma(fmaf(v[j + 3], sc, nl.w));     // every fourth exponential on the FMA pipe
                 }
             }
             if (c < c_hi) {                                    // halves are multiples of 16 columns
@@ -447,7 +449,7 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     a0 += fast_exp2(fmaf(v[j], sc, nl.x));
                     a1 += fast_exp2(fmaf(v[j + 1], sc, nl.y));
                     a0 += fast_exp2(fmaf(v[j + 2], sc, nl.z));
-                    a1 += fast_exp2(fmaf(v[j + 3], sc, nl.w));
+                    a1 += exp2_fma(fmaf(v[j + 3], sc, nl.w));     // every fourth exponential on the FMA pipe
                 }
             }
             tc_fence_before();

@@ -186,6 +186,22 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// 2^x for x <= 0 on the FMA pipe instead of the special-function unit: round x to an integer with
+// the 1.5 * 2^23 trick, a degree-5 polynomial for 2^f on f in [-0.5, 0.5] (relative error 2e-7, that
+// of ex2.approx), and the integer added to the exponent.  Used for a share of an epilogue's
+// exponentials so that both pipes work.
+__device__ __forceinline__ float exp2_fma(float x) {
+    x = fmaxf(x, -125.0f);
+    const float t = x + 12582912.0f;
+    const float f = x - (t - 12582912.0f);
+    float p = 0.001326472731307149f;
+    p = fmaf(p, f, 0.009671512991189957f);
+    p = fmaf(p, f, 0.05550733581185341f);
+    p = fmaf(p, f, 0.24022242426872253f);
+    p = fmaf(p, f, 0.6931470036506653f);
+    p = fmaf(p, f, 1.0f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
 
 // Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes
 // (64 bf16) in the 128-byte swizzle, 8-row groups 1024 bytes apart; the tile base is

@@ -804,7 +804,8 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
                     unsigned long long* __restrict__ slot_blocks, int32_t* __restrict__ slot_cnt,
                     int32_t* __restrict__ long_index, int32_t* __restrict__ long_slot,
                     int32_t* __restrict__ long_counter, int long_threshold, int long_cap,
-                    int32_t* __restrict__ few_members, int few_cap) {
+                    int32_t* __restrict__ few_members, int few_cap, int32_t* __restrict__ heavy_index,
+                    int32_t* __restrict__ heavy_slot, int32_t* __restrict__ heavy_counter, int heavy_cap) {
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= Nv) return;
     int slot;
@@ -821,6 +822,11 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
     // scratch an output gets depends on arrival order, what is computed in it does not)
     const int pos = atomicAdd(&slot_cnt[slot], 1);
     if (pos < few_cap) few_members[(size_t)slot * few_cap + pos] = row;   // the first few_cap arrivals are listed
+    if (pos == few_cap) {                                     // more than that: an output to be started early
+        const int hh = atomicAdd(heavy_counter, 1);
+        heavy_index[slot] = hh;
+        if (hh < heavy_cap) heavy_slot[hh] = slot;
+    }
     if (pos == long_threshold) {
         const int l = atomicAdd(long_counter, 1);
         long_index[slot] = l;
@@ -849,7 +855,8 @@ constexpr int kAvgFew = 16;        // outputs with at most this many members get
 constexpr int kAvgLong = 32;       // outputs with more members than this are split ...
 constexpr int kAvgParts = 8;       // ... over up to this many CTAs (fp32 partial sums, added in part order)
 constexpr int kAvgLongCap = 256;   // long outputs that get scratch for their partial sums
-constexpr int kAvgLongCtas = kAvgLongCap * (kAvgParts - 1);   // CTAs for the parts after the first
+constexpr int kAvgHeavyCap = 2048;  // outputs with more than kAvgFew members that are listed to be started first
+constexpr int kAvgFrontCtas = 8 * kNumSMs;   // CTAs at the front of the grid that take the listed outputs and parts
 // parts of an output with `count` > kAvgLong members: about eight members each
 __host__ __device__ inline int avg_parts(int count) {
     const int p = (count + 7) / 8;
@@ -1097,7 +1104,9 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
                  const unsigned long long* __restrict__ slot_blocks, const int32_t* __restrict__ slot_cnt,
                  const int32_t* __restrict__ long_index, const int32_t* __restrict__ long_slot,
                  const int32_t* __restrict__ long_counter, const int32_t* __restrict__ few_members,
-                 float* __restrict__ long_sums, int32_t* __restrict__ long_done, int long_ctas, const int32_t* __restrict__ n_out,
+                 const int32_t* __restrict__ heavy_index, const int32_t* __restrict__ heavy_slot,
+                 const int32_t* __restrict__ heavy_counter,
+                 float* __restrict__ long_sums, int32_t* __restrict__ long_done, int front_ctas, const int32_t* __restrict__ n_out,
                  T* __restrict__ out_feats, int32_t* __restrict__ out_members, int32_t* __restrict__ status) {
     using namespace sm100;
     extern __shared__ uint8_t avg_dyn[];
@@ -1106,36 +1115,52 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
     __shared__ int s_wtot[kAvgThreads / 32];
     __shared__ int s_blocks[64];
     __shared__ int s_abort, s_last;
-    // An output with more than kAvgLong members is shared by up to kAvgParts CTAs, each taking a range
-    // of member ranks: one CTA would add its rows four at a time and hold up the end of the kernel
-    // (the longest list sets the kernel's time otherwise).  Part 0 comes from the output's own CTA;
-    // the other parts have CTAs of their own, the first long_ctas of the grid, so that they start at
-    // once (booked by merge_decode, so the work is known when this kernel starts; a CTA without work
-    // leaves right away).  The other CTAs start in index order and take the outputs from the last
-    // one down, so that this pass begins with the rows of V that the preceding (ascending) pass left
-    // in L2.
+    // A CTA adds the rows of its output about three at a time, one memory latency per three rows:
+    // an output with many members lasts many times longer than the usual one, and would set the
+    // kernel's time if it started late.  So merge_decode lists every output with more than kAvgFew
+    // members, and the first front_ctas CTAs of the grid take the listed work round-robin, before the
+    // other outputs' CTAs start: the outputs with more than kAvgLong members part by part (up to
+    // kAvgParts parts of about eight members, partial sums combined in part order by the last part
+    // to finish), the others whole.  A listed output's own CTA leaves at once.  The other CTAs start
+    // in index order and take the outputs from the last one down, so that this pass begins with the
+    // rows of V that the preceding (ascending) pass left in L2.
     const int tid = threadIdx.x;
-    int c, part;
-    if ((int)blockIdx.x < long_ctas) {
-        const int l = (int)blockIdx.x / (kAvgParts - 1);
-        if (l >= min(*long_counter, kAvgLongCap)) return;
-        c = long_slot[l];
-        part = 1 + (int)blockIdx.x % (kAvgParts - 1);
-        if (part >= avg_parts(slot_cnt[c])) return;
-    } else {
-        c = *n_out - 1 - ((int)blockIdx.x - long_ctas);
-        part = 0;
-        if (c < 0) return;
-    }
     if (tid == 32) {                                           // not thread 0: it is busy with the block list below
         for (int j = 0; j < kAvgStages; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
         s_abort = 0;
         mbar_fence_init();
     }
     uint32_t phase = 0;                                        // bit j: parity of the next completion of barrier j
-    merge_avg_item<T>(c, part, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,
-                      ev_lo, out_event, assign, slot_blocks, slot_cnt, long_index, few_members, long_sums, long_done,
-                      out_feats, out_members, status);
+#define METOK_AVG_ITEM(C, PART)                                                                                     \
+    merge_avg_item<T>(C, PART, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,  \
+                      ev_lo, out_event, assign, slot_blocks, slot_cnt, long_index, few_members, long_sums, long_done,  \
+                      out_feats, out_members, status)
+    if ((int)blockIdx.x >= front_ctas) {
+        const int c = *n_out - 1 - ((int)blockIdx.x - front_ctas);
+        if (c < 0) return;
+        const int hh = heavy_index[c], ll = long_index[c];
+        if ((hh >= 0 && hh < kAvgHeavyCap) || (ll >= 0 && ll < kAvgLongCap)) return;   // listed: the front CTAs have it
+        METOK_AVG_ITEM(c, 0);
+        return;
+    }
+    const int n_long = min(*long_counter, kAvgLongCap), n_heavy = min(*heavy_counter, kAvgHeavyCap);
+    const int n_items = n_long * kAvgParts + n_heavy;
+    for (int it = (int)blockIdx.x; it < n_items; it += front_ctas) {
+        int c, part;
+        if (it < n_long * kAvgParts) {
+            c = long_slot[it / kAvgParts];
+            part = it % kAvgParts;
+            if (part >= avg_parts(slot_cnt[c])) continue;
+        } else {
+            c = heavy_slot[it - n_long * kAvgParts];
+            part = 0;
+            const int li = long_index[c];
+            if (li >= 0 && li < kAvgLongCap) continue;         // split into parts: taken above
+        }
+        METOK_AVG_ITEM(c, part);
+        __syncthreads();                                       // the shared lists are reused by the next item
+    }
+#undef METOK_AVG_ITEM
 }
 
 // --------------------------------------------------------------------------- //
@@ -1155,6 +1180,9 @@ struct VisionWs {
     int32_t* long_done;                // ... parts of each that have finished
     int32_t* long_index;               // output -> index among the long ones, -1 otherwise
     int32_t* long_slot;                // and back
+    int32_t* heavy_counter;            // outputs with more than kAvgFew members ...
+    int32_t* heavy_index;              // ... output -> index among them, -1 otherwise (directly after long_index)
+    int32_t* heavy_slot;               // ... and back
     int32_t* few_members;              // per output token: its first kAvgFew members, in arrival order
     float* long_sums;                  // partial sums of their parts
     size_t zero_bytes;                 // slot_blocks .. long_done are cleared together
@@ -1177,13 +1205,16 @@ static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, b
     w.best64 = mma ? cv.take<unsigned long long>((size_t)Tn * N) : nullptr;
     {
         const size_t n = (size_t)cap + 64;
-        w.zero_bytes = n * 8 + n * 4 + (size_t)(64 + kAvgLongCap) * 4;
+        w.zero_bytes = n * 8 + n * 4 + (size_t)(64 + kAvgLongCap + 64) * 4;
         unsigned char* z = cv.take<unsigned char>(w.zero_bytes);
         w.slot_blocks = reinterpret_cast<unsigned long long*>(z);
         w.slot_cnt = reinterpret_cast<int32_t*>(z + n * 8);
         w.long_counter = w.slot_cnt + n;
         w.long_done = w.long_counter + 64;
-        w.long_index = cv.take<int32_t>(n);
+        w.heavy_counter = w.long_done + kAvgLongCap;
+        w.long_index = cv.take<int32_t>(2 * n);         // long_index, then heavy_index: filled with -1 together
+        w.heavy_index = w.long_index + n;
+        w.heavy_slot = cv.take<int32_t>(kAvgHeavyCap);
         w.long_slot = cv.take<int32_t>(kAvgLongCap);
         w.few_members = cv.take<int32_t>(n * kAvgFew);
         w.long_sums = cv.take<float>((size_t)kAvgLongCap * kAvgParts * d);
@@ -1250,7 +1281,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     clr.zero_b = merging ? w.slot_blocks : nullptr;
     clr.zero_b_bytes = w.zero_bytes;
     clr.ones = merging ? w.long_index : nullptr;
-    clr.ones_bytes = ((size_t)cap + 64) * sizeof(int32_t);
+    clr.ones_bytes = 2 * ((size_t)cap + 64) * sizeof(int32_t);
     clr.status = w.status;
     {
         METOK_TIMED("event_plan_kernel", st);
@@ -1334,16 +1365,18 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         merge_decode_kernel<<<ceil_div(Nv, 256), 256, 0, st>>>(mma ? w.best64 : nullptr, w.is_key, Nv, N, w.ev_lo, k,
                                                                assign, w.slot_blocks, w.slot_cnt, w.long_index,
                                                                w.long_slot, w.long_counter, kAvgLong, kAvgLongCap,
-                                                               w.few_members, kAvgFew);
+                                                               w.few_members, kAvgFew, w.heavy_index, w.heavy_slot,
+                                                               w.heavy_counter, kAvgHeavyCap);
     }
     METOK_LAUNCH_CHECK();
     METOK_CUDA_TRY(cudaFuncSetAttribute(merge_avg_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)kAvgSmemBytes));
     {
         METOK_TIMED("merge_avg_kernel", st);
-        merge_avg_kernel<T><<<kAvgLongCtas + cap, kAvgThreads, kAvgSmemBytes, st>>>(
+        merge_avg_kernel<T><<<kAvgFrontCtas + cap, kAvgThreads, kAvgSmemBytes, st>>>(
             feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
-            w.long_counter, w.few_members, w.long_sums, w.long_done, kAvgLongCtas, n_out, out_feats, out_members,
+            w.long_counter, w.few_members, w.heavy_index, w.heavy_slot, w.heavy_counter, w.long_sums, w.long_done,
+            kAvgFrontCtas, n_out, out_feats, out_members,
             w.status);
     }
     METOK_LAUNCH_CHECK();

@@ -91,6 +91,16 @@ CONFIGS: Dict[str, Config] = {
 # the 128-frame workload with the vision tower's own feature width
 CONFIGS["frames128d1024"] = dataclasses.replace(CONFIGS["frames128"], name="frames128d1024", d=1024)
 
+# The paper's two other model sizes (Implementation Details): 32 frames of 196 tokens into a 24-layer
+# decoder with 14 query / 2 key-value heads of 64, k = 5, r = 0.76; and 16 frames of 196 tokens into a
+# 40-layer decoder with 40 heads of 128 and no head sharing, k = 3, r = 0.65, L_H = [13, 24, 34].
+CONFIGS["small24"] = Config("small24", 5, T=32, N=196, d=1152, dtype="bf16", k=5, sigma=0.1, Lt=24,
+                            Hq=14, Hkv=2, dh=64, D=896, L=24, alpha=0.5, keep_enc=0.25,
+                            keep_prefill=0.76, keep_kv=0.1, n_stages=3, kv_text=24, events="compose")
+CONFIGS["large40"] = Config("large40", 6, T=16, N=196, d=1152, dtype="bf16", k=3, sigma=0.1, Lt=40,
+                            Hq=40, Hkv=40, dh=128, D=5120, L=40, alpha=0.5, keep_enc=0.25,
+                            keep_prefill=0.65, keep_kv=0.1, n_stages=3, kv_text=40, events="compose")
+
 CONFIG_ORDER = ["tiny", "frames32", "frames64", "frames128", "stress"]
 
 

@@ -350,3 +350,51 @@ def test_chained_pipeline_tiny_and_frames32():
         assert np.array_equal(out["event_is_key"].cpu().numpy(), want["event_is_key"])
         same = np.mean(out["out_src"][:n].cpu().numpy() == want["out_src"])
         assert same > 0.99
+
+
+# ---------------------------------------- other model sizes, ablation settings ----- #
+
+@pytest.mark.parametrize("name,l1", [("small24", 3), ("large40", 13)])
+def test_other_model_sizes_all_four_calls(name, l1):
+    """The paper's smallest and largest decoders (24 layers, 14/2 heads of 64; 40 layers, 40 heads of
+    128 without head sharing): every call at those shapes, three pruning levels, both K/V policies."""
+    cfg = W.CONFIGS[name]
+    vis = vis_of(name)
+    Vd, td = P.to_torch(vis["V"], cfg.dtype), P.to_torch(vis["t"], cfg.dtype)
+    got = B.metok_segment_score_events(Vd, cfg.k, td)
+    want = O.segment_events(vis["V"], cfg.k)
+    P.check_scores(got["sims"].cpu().numpy(), want["sims"], cfg.dtype, "sims")
+    assert np.array_equal(got["event_offsets"].cpu().numpy(), want["event_offsets"])
+    assert np.array_equal(want["event_offsets"], vis["event_offsets"])
+    rep = R.compress_case(vis["V"], vis["t"], vis["event_offsets"], cfg.dtype, cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+    assert "event_class_flip" not in rep
+    assert rep["key_mismatches"] <= rep["key_near_ties"] and rep["assign_mismatches"] <= rep["assign_near_ties"]
+    for stage in (1, 2, 3):
+        groups, budgets = _prefill_stage_inputs(cfg, stage, vis)
+        pf = W.prefill_inputs(cfg, stage, groups.size, groups)
+        hidden = W.payload_torch(W.hidden_salt(cfg, stage), pf["S"], cfg.D, cfg.dtype, "cuda")
+        r = R.prefill_case(pf["Q"], pf["K"], cfg.dtype, 0, groups.size, groups, budgets, cfg.dh ** -0.5, hidden)
+        assert r["S_out"] == cfg.Lt + sum(min(b, int((groups == g).sum())) for g, b in enumerate(budgets))
+    del hidden
+    torch.cuda.empty_cache()
+    R.kv_case(cfg, O.KV_TOPK)
+    R.kv_case(cfg, O.KV_PAPER, l1=l1)
+
+
+def test_ablation_uniform_segmentation_max_events_last_token_scores():
+    """Settings of the paper's ablations that are arguments of the calls: events of equal length
+    instead of Eq. 4's (the caller's offsets), the event score as the maximum over frames
+    (Algorithm 1), and attention scores from the last text token alone (one query row)."""
+    cfg = W.CONFIGS["frames32"]
+    vis = vis_of("frames32")
+    uniform = np.linspace(0, cfg.T, cfg.k + 1).round().astype(np.int32)
+    assert not np.array_equal(uniform, vis["event_offsets"])
+    for agg in (O.AGG_MEAN, O.AGG_MAX):
+        rep = R.compress_case(vis["V"], vis["t"], uniform, cfg.dtype, cfg.alpha, cfg.keep_enc, cfg.keep_enc, agg)
+        assert "event_class_flip" not in rep
+        assert rep["key_mismatches"] <= rep["key_near_ties"] and rep["assign_mismatches"] <= rep["assign_near_ties"]
+    groups, budgets = _prefill_stage_inputs(cfg, 1, vis)
+    pf = W.prefill_inputs(cfg, 1, cfg.Nv, groups)
+    # the keys of the earlier text tokens stay in the sequence; only the last one asks
+    r = R.prefill_case(pf["Q"][:, -1:, :], pf["K"], cfg.dtype, 0, cfg.Nv, groups, budgets, cfg.dh ** -0.5)
+    assert r["S_out"] == cfg.Lt + sum(min(b, int((groups == g).sum())) for g, b in enumerate(budgets))

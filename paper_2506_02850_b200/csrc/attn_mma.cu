@@ -87,6 +87,7 @@ __global__ void __launch_bounds__(kStThreads, 1)
 attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       AttnMmaDims dm, float* __restrict__ part_m, float* __restrict__ part_l,
                       int32_t* __restrict__ status) {
+    grid_dep_wait();
     using namespace sm100;
     constexpr int KB = DH / 64;                               // 64-element (128-byte) K blocks
     constexpr uint32_t kQBlk = kStBM * 128, kKBlk = kStBN * 128;
@@ -284,6 +285,7 @@ __global__ void __launch_bounds__(kAmThreads, 1)
 attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        AttnMmaDims dm, const float* __restrict__ part_m, const float* __restrict__ part_l,
                        float* __restrict__ part_col, int32_t* __restrict__ status) {
+    grid_dep_wait();
     using namespace sm100;
     constexpr int KB = DH / 64;
     constexpr uint32_t kKBlk = kCsBM * 128;
@@ -484,13 +486,13 @@ int launch_dh(const void* q_text, const void* k_all, const AttnMmaDims& dm, floa
                                         (int)((size_t)KB * (kCsMaxNQ + kCsStages * kCsBM) * 128 + 1024)));
     {
         METOK_TIMED("attn_stats_mma_kernel", st);
-        attn_stats_mma_kernel<DH><<<dim3(dm.st_nsplit, dm.st_nrt, dm.Hkv), kStThreads, smem_st, st>>>(
+        launch_chained(attn_stats_mma_kernel<DH>, dim3(dim3(dm.st_nsplit, dm.st_nrt, dm.Hkv)), dim3(kStThreads), smem_st, st, 
             tmQs, tmKs, dm, part_m, part_l, status);
     }
     METOK_LAUNCH_CHECK();
     {
         METOK_TIMED("attn_colsum_mma_kernel", st);
-        attn_colsum_mma_kernel<DH><<<dim3(dm.cs_nsplit, dm.cs_nchunk, dm.Hkv), kAmThreads, smem_cs, st>>>(
+        launch_chained(attn_colsum_mma_kernel<DH>, dim3(dim3(dm.cs_nsplit, dm.cs_nchunk, dm.Hkv)), dim3(kAmThreads), smem_cs, st, 
             tmQc, tmKc, dm, part_m, part_l, part_col, status);
     }
     METOK_LAUNCH_CHECK();

@@ -39,6 +39,35 @@ struct KernelTimer {
 };
 #define METOK_TIMED(name, st) ::metok::KernelTimer _metok_kt(name, st)
 
+// Launch with programmatic stream serialisation: the grid may be scheduled while the kernel before it
+// on the stream is still draining, and every one of its CTAs calls grid_dep_wait() before it touches
+// memory, which returns once that kernel has completed and its writes are visible.  Because every CTA
+// of every kernel launched this way waits first, completion of a kernel implies completion of all
+// kernels before it on the stream.  The launch error is picked up by METOK_LAUNCH_CHECK().
+template <typename... P, typename... A>
+inline void launch_chained(void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    (void)cudaLaunchKernelEx(&cfg, kern, static_cast<P>(args)...);
+}
+
+#ifdef __CUDACC__
+// First statements of a kernel launched by launch_chained(): wait for the kernel before it, then let
+// the kernel after it be scheduled as soon as all CTAs of this one have started.
+__device__ __forceinline__ void grid_dep_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

@@ -101,6 +101,7 @@ __global__ void __launch_bounds__(kKvFastThreads)
 kv_stage_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row_chunks,
                 const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ keep_len, int stage_rows,
                 int32_t* __restrict__ haz, uint4* __restrict__ stage) {
+    grid_dep_wait();
     __shared__ int s_h;
     const SlabId id = slab_of(blockIdx.y, Hkv);
     const int layer = layer0 + id.ll;
@@ -132,6 +133,7 @@ __global__ void __launch_bounds__(kKvFastThreads)
 kv_copy_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row_chunks,
                const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ keep_len, int stage_rows,
                const int32_t* __restrict__ haz, const uint4* __restrict__ stage) {
+    grid_dep_wait();
     const SlabId id = slab_of(blockIdx.y, Hkv);
     const int layer = layer0 + id.ll;
     const int h = haz[layer];
@@ -321,13 +323,13 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
         const int slabs = nl * 2 * Hkv;
         {
             METOK_TIMED("kv_stage_kernel", st);
-            kv_stage_kernel<<<dim3(kKvStageSplit, slabs), kKvFastThreads, 0, st>>>(
+            launch_chained(kv_stage_kernel, dim3(dim3(kKvStageSplit, slabs)), dim3(kKvFastThreads), 0, st, 
                 ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len, w.stage_rows, w.haz, w.stage);
         }
         METOK_LAUNCH_CHECK();
         {
             METOK_TIMED("kv_copy_kernel", st);
-            kv_copy_kernel<<<dim3(kKvCopySplit, slabs), kKvFastThreads, 0, st>>>(
+            launch_chained(kv_copy_kernel, dim3(dim3(kKvCopySplit, slabs)), dim3(kKvFastThreads), 0, st, 
                 ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len, w.stage_rows, w.haz, w.stage);
         }
         METOK_LAUNCH_CHECK();

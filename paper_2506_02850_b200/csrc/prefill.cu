@@ -214,6 +214,7 @@ attn_colsum_kernel(const T* __restrict__ q_text, const T* __restrict__ k_all, At
 __global__ void __launch_bounds__(256)
 attn_score_reduce_kernel(const float* __restrict__ part_col, int nparts, int n_vis, float inv_rows,
                          float* __restrict__ scores) {
+    grid_dep_wait();
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n_vis) return;
     float a = 0.f;
@@ -295,6 +296,7 @@ block_topk_kernel(const float* __restrict__ scores, size_t score_stride, const i
                   int n_vis, int G, BlockSelLayout lay, TopkBudgets budgets, int S, int vis_start,
                   int32_t* __restrict__ keep_idx, size_t keep_stride, int replicas,
                   int32_t* __restrict__ count_a, int32_t* __restrict__ count_b) {
+    grid_dep_wait();
     __shared__ BlockSelSmem sm;
     extern __shared__ __align__(16) unsigned char sel_dyn[];
     const int problem = blockIdx.x;
@@ -347,7 +349,7 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
             METOK_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bl.bytes));
         {
             METOK_TIMED("class_topk_kernel", st);
-            kernel<<<problems, kBsThreads, bl.bytes, st>>>(scores, score_stride, token_group, n_vis, G, bl, b, S,
+            launch_chained(kernel, dim3(problems), dim3(kBsThreads), bl.bytes, st, scores, score_stride, token_group, n_vis, G, bl, b, S,
                                                            vis_start, keep_idx, keep_stride, replicas, count_a, count_b);
         }
         METOK_LAUNCH_CHECK();
@@ -386,6 +388,7 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 __global__ void __launch_bounds__(kGatherThreads)
 gather_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const int32_t* __restrict__ keep_idx,
                    const int32_t* __restrict__ n_rows, int row_chunks) {
+    grid_dep_wait();
     const int n = *n_rows;
     const int lane = threadIdx.x & 31;
     const int warps = gridDim.x * (kGatherThreads / 32);
@@ -415,6 +418,7 @@ __global__ void __launch_bounds__(32)
 gather_rows_bulk_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
                         const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ n_rows,
                         uint32_t row_bytes, int32_t* __restrict__ status) {
+    grid_dep_wait();
     using namespace sm100;
     extern __shared__ uint8_t gb_dyn[];
     __shared__ __align__(8) uint64_t s_bar[kGbStages];
@@ -471,7 +475,7 @@ int launch_gather_rows_bulk(const void* src, void* dst, const int32_t* idx, cons
                                         (int)kGbSmemBytes));
     {
         METOK_TIMED(timer_name, st);
-        gather_rows_bulk_kernel<<<kNumSMs * 6, 32, kGbSmemBytes, st>>>(
+        launch_chained(gather_rows_bulk_kernel, dim3(kNumSMs * 6), dim3(32), kGbSmemBytes, st, 
             reinterpret_cast<const uint8_t*>(src), reinterpret_cast<uint8_t*>(dst), idx, n_rows, (uint32_t)row_bytes,
             status);
     }
@@ -483,7 +487,7 @@ int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int
                        const char* timer_name, cudaStream_t st) {
     {
         METOK_TIMED(timer_name, st);
-        gather_rows_kernel<<<kNumSMs * 8, kGatherThreads, 0, st>>>(reinterpret_cast<const uint4*>(src),
+        launch_chained(gather_rows_kernel, dim3(kNumSMs * 8), dim3(kGatherThreads), 0, st, reinterpret_cast<const uint4*>(src),
                                                         reinterpret_cast<uint4*>(dst), idx, n_rows, row_chunks);
     }
     METOK_LAUNCH_CHECK();
@@ -539,7 +543,7 @@ static PrefillWs carve_prefill(Carver& cv, const AttnDims& dm, bool mma) {
 static int launch_score_reduce(const PrefillWs& w, const AttnDims& dm, float* scores, cudaStream_t st) {
     {
         METOK_TIMED("attn_score_reduce_kernel", st);
-        attn_score_reduce_kernel<<<ceil_div(dm.n_vis, 256), 256, 0, st>>>(w.part_col, w.n_planes, dm.n_vis,
+        launch_chained(attn_score_reduce_kernel, dim3(ceil_div(dm.n_vis, 256)), dim3(256), 0, st, w.part_col, w.n_planes, dm.n_vis,
                                                                       1.0f / (float)(dm.Hq * dm.Lt), scores);
     }
     METOK_LAUNCH_CHECK();

@@ -152,6 +152,7 @@ __global__ void __launch_bounds__(1024)
 seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ part_nrm, int nslab,
                   int Tn, int k, float* __restrict__ sims, int32_t* __restrict__ boundaries,
                   int32_t* __restrict__ event_offsets, int32_t* __restrict__ frame_event) {
+    grid_dep_wait();
     extern __shared__ float sm_f[];
     float* s_sim = sm_f;                                   // [Tn]   (Tn-1 used)
     float* s_nrm = sm_f + Tn;                              // [Tn]
@@ -297,7 +298,7 @@ static int launch_segment(const void* feats, int Tn, int N, int d, int k, int si
     }
     {
         METOK_TIMED("seg_finish_kernel", st);
-        seg_finish_kernel<<<1, 1024, smem, st>>>(part_dot, part_nrm, nslab, Tn, k, sims, boundaries, event_offsets,
+        launch_chained(seg_finish_kernel, dim3(1), dim3(1024), smem, st, part_dot, part_nrm, nslab, Tn, k, sims, boundaries, event_offsets,
                                              frame_event);
     }
     METOK_LAUNCH_CHECK();
@@ -500,6 +501,7 @@ __global__ void __launch_bounds__(kFsThreads)
 seg_score_mma_kernel(const __nv_bfloat16* __restrict__ feats, const __nv_bfloat16* __restrict__ text, int Tn, int N,
                      int d, float* __restrict__ part_dot, float* __restrict__ part_nrm,
                      float* __restrict__ token_score, float* __restrict__ inv_norm) {
+    grid_dep_wait();
     extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ float s_red[kFsThreads / 32];
     __shared__ float s_tn;
@@ -649,7 +651,7 @@ static int launch_seg_score(const void* feats, const void* text, int Tn, int N, 
             METOK_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_t));
         nslab = ceil_div(N, kFsThreads / 32);              // the kernel adds the four positions of a CTA
         METOK_TIMED("seg_score_kernel", st);
-        kernel<<<nslab * ceil_div(Tn, kFsFrames), kFsThreads, smem_t, st>>>(
+        launch_chained(kernel, dim3(nslab * ceil_div(Tn, kFsFrames)), dim3(kFsThreads), smem_t, st, 
             reinterpret_cast<const __nv_bfloat16*>(feats), reinterpret_cast<const __nv_bfloat16*>(text), Tn, N, d,
             part_dot, part_nrm, token_score, inv_norm);
     } else {
@@ -668,7 +670,7 @@ static int launch_seg_score(const void* feats, const void* text, int Tn, int N, 
         METOK_CUDA_TRY(cudaFuncSetAttribute(seg_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     {
         METOK_TIMED("seg_finish_kernel", st);
-        seg_finish_kernel<<<1, 1024, smem, st>>>(part_dot, part_nrm, nslab, Tn, k, sims, boundaries, event_offsets,
+        launch_chained(seg_finish_kernel, dim3(1), dim3(1024), smem, st, part_dot, part_nrm, nslab, Tn, k, sims, boundaries, event_offsets,
                                              frame_event);
     }
     METOK_LAUNCH_CHECK();

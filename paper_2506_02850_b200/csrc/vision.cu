@@ -144,6 +144,7 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
                   int32_t* __restrict__ ev_tile_off, int32_t* __restrict__ ev_unit_off,
                   int32_t* __restrict__ frame_ev, int32_t* __restrict__ frame_stride,
                   int32_t* __restrict__ frame_off, int32_t* __restrict__ n_out, PlanClears clr) {
+    grid_dep_wait();
     extern __shared__ float s_score[];      // [k]
     if (blockIdx.x > 0) {                   // CTAs 1 .. kPlanFillCtas only clear; CTA 0 plans
         block_fill(clr.zero_a, clr.zero_a_bytes, 0u, (int)blockIdx.x - 1, kPlanFillCtas);
@@ -445,6 +446,7 @@ event_block_topk_kernel(const float* __restrict__ token_score, const int32_t* __
                         const int32_t* __restrict__ ev_budget, const int32_t* __restrict__ ev_out_off,
                         BlockSelLayout lay, uint8_t* __restrict__ is_key, int32_t* __restrict__ out_src,
                         int32_t* __restrict__ out_event, int32_t* __restrict__ assign) {
+    grid_dep_wait();
     __shared__ BlockSelSmem sm;
     __shared__ int s_budget[1];
     extern __shared__ __align__(16) unsigned char sel_dyn[];
@@ -646,6 +648,7 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         const int32_t* __restrict__ ev_unit_off, const int32_t* __restrict__ out_src,
                         const float* __restrict__ inv_norm, const uint8_t* __restrict__ is_key,
                         unsigned long long* __restrict__ best64, int32_t* __restrict__ status) {
+    grid_dep_wait();
     using namespace sm100;
     extern __shared__ uint8_t smem_dyn[];
     __shared__ __align__(8) uint64_t full_bar[kMmaStages], empty_bar[kMmaStages], tfull_bar, tempty_bar, drain_bar;
@@ -806,6 +809,7 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
                     int32_t* __restrict__ long_counter, int long_threshold, int long_cap,
                     int32_t* __restrict__ few_members, int few_cap, int32_t* __restrict__ heavy_index,
                     int32_t* __restrict__ heavy_slot, int32_t* __restrict__ heavy_counter, int heavy_cap) {
+    grid_dep_wait();
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= Nv) return;
     int slot;
@@ -1108,6 +1112,7 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
                  const int32_t* __restrict__ heavy_counter,
                  float* __restrict__ long_sums, int32_t* __restrict__ long_done, int front_ctas, const int32_t* __restrict__ n_out,
                  T* __restrict__ out_feats, int32_t* __restrict__ out_members, int32_t* __restrict__ status) {
+    grid_dep_wait();
     using namespace sm100;
     extern __shared__ uint8_t avg_dyn[];
     __shared__ __align__(8) uint64_t s_bar[kAvgStages];
@@ -1285,7 +1290,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     clr.status = w.status;
     {
         METOK_TIMED("event_plan_kernel", st);
-        event_plan_kernel<<<1 + kPlanFillCtas, 1024, plan_smem, st>>>(token_score, frame_score, event_offsets, pp, event_score,
+        launch_chained(event_plan_kernel, dim3(1 + kPlanFillCtas), dim3(1024), plan_smem, st, token_score, frame_score, event_offsets, pp, event_score,
                                                                   event_is_key, w.ev_lo, w.ev_budget, w.ev_out_off,
                                                                   w.ev_tile_off, w.ev_unit_off, w.frame_ev,
                                                                   w.frame_stride, w.frame_off, n_out, clr);
@@ -1312,7 +1317,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
                 METOK_CUDA_TRY(cudaFuncSetAttribute(event_block_topk_kernel,
                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bl.bytes));
             METOK_TIMED("event_topk_kernel", st);
-            event_block_topk_kernel<<<k, kBsThreads, bl.bytes, st>>>(token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off,
+            launch_chained(event_block_topk_kernel, dim3(k), dim3(kBsThreads), bl.bytes, st, token_score, w.ev_lo, N, w.ev_budget, w.ev_out_off,
                                                                      bl, w.is_key, out_src, out_event, assign);
         } else {
             const SelectLayout lay = select_layout(1, select_items_per_cta((long long)(Tn - (k - 1)) * N));
@@ -1344,7 +1349,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
                                             (int)kMmaSmemBytes));
         {
             METOK_TIMED("merge_assign_mma_kernel", st);
-            merge_assign_mma_kernel<<<kNumSMs, kMmaThreads, kMmaSmemBytes, st>>>(
+            launch_chained(merge_assign_mma_kernel, dim3(kNumSMs), dim3(kMmaThreads), kMmaSmemBytes, st, 
                 tmA, tmA_half, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, inv_norm, w.is_key, w.best64,
                 w.status);
         }
@@ -1362,7 +1367,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
 
     {
         METOK_TIMED("merge_decode_kernel", st);
-        merge_decode_kernel<<<ceil_div(Nv, 256), 256, 0, st>>>(mma ? w.best64 : nullptr, w.is_key, Nv, N, w.ev_lo, k,
+        launch_chained(merge_decode_kernel, dim3(ceil_div(Nv, 256)), dim3(256), 0, st, mma ? w.best64 : nullptr, w.is_key, Nv, N, w.ev_lo, k,
                                                                assign, w.slot_blocks, w.slot_cnt, w.long_index,
                                                                w.long_slot, w.long_counter, kAvgLong, kAvgLongCap,
                                                                w.few_members, kAvgFew, w.heavy_index, w.heavy_slot,
@@ -1373,7 +1378,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
                                         (int)kAvgSmemBytes));
     {
         METOK_TIMED("merge_avg_kernel", st);
-        merge_avg_kernel<T><<<kAvgFrontCtas + cap, kAvgThreads, kAvgSmemBytes, st>>>(
+        launch_chained(merge_avg_kernel<T>, dim3(kAvgFrontCtas + cap), dim3(kAvgThreads), kAvgSmemBytes, st, 
             feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
             w.long_counter, w.few_members, w.heavy_index, w.heavy_slot, w.heavy_counter, w.long_sums, w.long_done,
             kAvgFrontCtas, n_out, out_feats, out_members,

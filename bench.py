@@ -43,12 +43,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES = {
     # profiles/kernel_sections_frames128.txt; averages over a step's launches of the kernel
     ("class_topk_kernel", "frames128"): 0.14e6,
-    ("merge_assign_mma_kernel", "frames128"): 163.1e6,
-    ("merge_avg_kernel", "frames128"): 149.1e6,
+    ("merge_assign_mma_kernel", "frames128"): 163.7e6,
+    ("merge_avg_kernel", "frames128"): 151.6e6,
     ("seg_score_kernel", "frames128"): 136.0e6,
-    ("tok_score_kernel", "frames128"): 136.5e6,
-    ("kv_copy_kernel", "frames128"): 101.0e6,
-    ("gather_rows_kernel", "frames128"): 23.1e6,
+    ("tok_score_kernel", "frames128"): 135.9e6,
+    ("kv_copy_kernel", "frames128"): 100.7e6,
+    ("gather_rows_kernel", "frames128"): 23.3e6,
     ("gather_key_rows_kernel", "frames128"): 26.6e6,
     ("attn_stats_mma_kernel", "frames128"): 9.9e6,
     ("attn_colsum_mma_kernel", "frames128"): 10.1e6,

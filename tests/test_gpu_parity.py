@@ -398,3 +398,75 @@ def test_ablation_uniform_segmentation_max_events_last_token_scores():
     # the keys of the earlier text tokens stay in the sequence; only the last one asks
     r = R.prefill_case(pf["Q"][:, -1:, :], pf["K"], cfg.dtype, 0, cfg.Nv, groups, budgets, cfg.dh ** -0.5)
     assert r["S_out"] == cfg.Lt + sum(min(b, int((groups == g).sum())) for g, b in enumerate(budgets))
+
+
+def test_cuda_graph_replay_equals_eager_calls():
+    """The four calls enqueue on a stream and never synchronise: captured once in a CUDA graph
+    (kernel-to-kernel edges become programmatic ones) and replayed, they must leave exactly what
+    the eager calls leave."""
+    cfg = W.CONFIGS["frames32"]
+    vis = vis_of("frames32")
+    Vd, td = P.to_torch(vis["V"], cfg.dtype), P.to_torch(vis["t"], cfg.dtype)
+    p = B.vision_params(cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+    groups, budgets = _prefill_stage_inputs(cfg, 1, vis)
+    pf = W.prefill_inputs(cfg, 1, cfg.Nv, groups)
+    Q, K = P.to_torch(pf["Q"], cfg.dtype), P.to_torch(pf["K"], cfg.dtype)
+    hidden = W.payload_torch(W.hidden_salt(cfg, 1), pf["S"], cfg.D, cfg.dtype, "cuda")
+    grp = torch.from_numpy(groups.astype(np.int32)).cuda()
+    S_cur = cfg.Nv + cfg.kv_text
+    layers = 4
+
+    def step(o, ks, vs):
+        o["seg"] = B.metok_segment_score_events(Vd, cfg.k, td, out=o.get("seg"))
+        o["cv"] = B.metok_compress_vision(Vd, o["seg"]["event_offsets"], td, p, out=o.get("cv"), scored=o["seg"])
+        o["pf"] = B.metok_prefill_prune(Q, K, hidden, 0, cfg.Nv, grp, budgets, cfg.dh ** -0.5, out=o.get("pf"))
+        kv = o.get("kv") or {"keep_idx": None, "keep_len": None, "new_len": None}
+        o["kv"] = B.metok_kv_compact(ks, vs, S_cur, B.KV_TOPK, 0, cfg.Nv, keep_ratio=cfg.keep_kv,
+                                     scores=o["pf"]["scores"], keep_idx=kv["keep_idx"], keep_len=kv["keep_len"],
+                                     new_len=kv["new_len"])
+
+    def caches():
+        return W.kv_cache_torch(cfg, torch.device("cuda"), layers)
+
+    side = torch.cuda.Stream()
+    eager, replay = {}, {}
+    ks_e, vs_e = caches()
+    ks_g, vs_g = caches()
+    with torch.cuda.stream(side):
+        step(eager, ks_e, vs_e)
+        scratch_k, scratch_v = caches()
+        step(replay, scratch_k, scratch_v)                     # allocates the outputs the graph will write
+    side.synchronize()
+    for d in replay.values():                                   # nothing of the warm-up may survive by accident
+        for t in d.values():
+            if isinstance(t, torch.Tensor) and t.numel() and not t.dtype.is_floating_point:
+                t.fill_(-1) if t.dtype != torch.uint8 else t.fill_(255)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step(replay, ks_g, vs_g)
+    graph.replay()
+    torch.cuda.synchronize()
+
+    def same(a, b):
+        return torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a,
+                           b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+
+    for name in ("sims", "boundaries", "event_offsets", "frame_event", "token_score", "token_inv_norm"):
+        assert same(eager["seg"][name], replay["seg"][name]), name
+    n = int(eager["cv"]["n_out"].item())
+    assert n == int(replay["cv"]["n_out"].item()) and n > 0
+    for name in ("out_feats", "out_src", "out_event", "out_members"):
+        assert same(eager["cv"][name][:n], replay["cv"][name][:n]), name
+    for name in ("assign", "frame_score", "event_score", "event_is_key"):
+        assert same(eager["cv"][name], replay["cv"][name]), name
+    s_out = int(eager["pf"]["S_out"].item())
+    assert s_out == int(replay["pf"]["S_out"].item())
+    assert same(eager["pf"]["scores"], replay["pf"]["scores"])
+    assert same(eager["pf"]["keep_idx"][:s_out], replay["pf"]["keep_idx"][:s_out])
+    assert same(eager["pf"]["hidden_out"][:s_out], replay["pf"]["hidden_out"][:s_out])
+    new_len = eager["kv"]["new_len"].cpu().tolist()
+    assert new_len == replay["kv"]["new_len"].cpu().tolist()
+    for layer in range(layers):
+        m = new_len[layer]
+        assert same(eager["kv"]["keep_idx"][layer, :m], replay["kv"]["keep_idx"][layer, :m])
+        assert same(ks_e[layer][:, :m], ks_g[layer][:, :m]) and same(vs_e[layer][:, :m], vs_g[layer][:, :m])

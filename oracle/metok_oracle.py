@@ -413,6 +413,31 @@ def weighted_topk(scores: np.ndarray, token_group: np.ndarray, group_budget: Seq
     return {"keep_idx": keep_idx, "S_out": keep_idx.size, "near_tie": near}
 
 
+def prune_schedule(Qs: Sequence[np.ndarray], Ks: Sequence[np.ndarray], token_group: np.ndarray, alpha: float,
+                   r: float, vis_start: int, softmax_scale: float) -> List[Dict[str, np.ndarray]]:
+    """The pruning levels l1, l2, l3 one after the other (section 3.2.2): level s scores the visual
+    tokens that survived level s-1 with that layer's text queries and keys (Qs[s], Ks[s]: rows of
+    the survivors, in order), and keeps per class the budget of Eq. 6/7 for stage s, which is
+    relative to the class counts N0 at the first level.  A survivor keeps its class.  Per level:
+    the level's result plus `token_group` (its input classes) and `origin` (for each of its visual
+    tokens the index among the first level's)."""
+    group = np.asarray(token_group, dtype=np.int32)
+    N0 = [int((group == 0).sum()), int((group == 1).sum())]
+    origin = np.arange(group.size, dtype=np.int32)
+    levels = []
+    for s, (Q, K) in enumerate(zip(Qs, Ks), start=1):
+        n_vis = group.size
+        S = K.shape[1]
+        a = attention_scores(Q, K, vis_start, n_vis, softmax_scale)
+        budget = retention_budgets(alpha, r, s, N0)
+        sel = weighted_topk(a, group, budget, S, vis_start)
+        sel.update({"scores": a, "token_group": group, "origin": origin, "budget": budget})
+        levels.append(sel)
+        kept_vis = sel["keep_idx"][(sel["keep_idx"] >= vis_start) & (sel["keep_idx"] < vis_start + n_vis)] - vis_start
+        group, origin = group[kept_vis], origin[kept_vis]
+    return levels
+
+
 # --------------------------------------------------------------------------- #
 # a7 / a9: order-preserving row gathers
 # --------------------------------------------------------------------------- #

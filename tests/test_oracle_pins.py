@@ -551,3 +551,44 @@ def test_pool2d_and_adaptive_pool():
     assert np.all(np.diff(out["out_frame"]) >= 0)
     ek = np.repeat(out["event_is_key"], np.diff(vis["event_offsets"]))
     assert set(out["frame_stride"][ek == 1]) <= {2, 3} and set(out["frame_stride"][ek == 0]) <= {4, 6}
+
+
+def test_prune_schedule_planted_order_and_printed_ratios():
+    """Three levels on logits planted per level (one head, one text query, K[j] = c_j u, Q = u, so
+    the score is monotone in c_j): the survivors must be the per-class top budgets of a plain sort
+    of c, with the paper's r = 0.55, alpha = 0.5 (stage ratios .55/.275, .3025/0, 0/0)."""
+    rng = np.random.default_rng(11)
+    dh, n_vis, vis_start, tail = 8, 300, 3, 2                  # 2 non-visual positions after the visual span, 1 text query last
+    group = (rng.random(n_vis) < 0.33).astype(np.int32)       # 1 = non-key
+    N0 = [int((group == 0).sum()), int((group == 1).sum())]
+    u = np.zeros(dh); u[2] = 1.0
+    alive = np.arange(n_vis)
+    Qs, Ks, want_alive, cs = [], [], [], []
+    for stage, ratios in zip((1, 2, 3), ((0.55, 0.275), (0.3025, 0.0), (0.0, 0.0))):
+        c = rng.permutation(alive.size).astype(np.float64) * 0.01      # distinct, reshuffled at every level
+        S = vis_start + alive.size + tail + 1
+        K = rng.standard_normal((1, S, dh)) * 0.01
+        K[0, :, 2] = 0.0
+        K[0, vis_start:vis_start + alive.size] += c[:, None] * u[None, :]
+        Qs.append(u[None, None, :].copy()); Ks.append(K); cs.append(c)
+        keep = []
+        for g in (0, 1):
+            members = [i for i in range(alive.size) if group[alive[i]] == g]
+            n = min(len(members), math.ceil(ratios[g] * N0[g] - 1e-9))
+            keep += sorted(members, key=lambda i: -c[i])[:n]
+        alive = alive[sorted(keep)]
+        want_alive.append(alive)
+    lv = O.prune_schedule(Qs, Ks, group, 0.5, 0.55, vis_start, 1.0)
+    assert len(lv) == 3
+    assert lv[0]["budget"].tolist() == [math.ceil(0.55 * N0[0] - 1e-9), math.ceil(0.275 * N0[1] - 1e-9)]
+    for s in range(3):
+        S = Ks[s].shape[1]
+        n_in = lv[s]["token_group"].size
+        k = lv[s]["keep_idx"]
+        vis = k[(k >= vis_start) & (k < vis_start + n_in)] - vis_start
+        assert np.array_equal(lv[s]["origin"][vis], want_alive[s]), s
+        assert np.array_equal(lv[s]["token_group"], group[lv[s]["origin"]])
+        non_vis = [p for p in range(S) if not (vis_start <= p < vis_start + n_in)]
+        assert set(non_vis) <= set(k.tolist())                 # every non-visual position survives
+    assert want_alive[1].size == math.ceil(0.3025 * N0[0] - 1e-9) and want_alive[2].size == 0
+    assert np.all(group[want_alive[1]] == 0)                   # no non-key token passes the second level

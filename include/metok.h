@@ -273,6 +273,51 @@ METOK_API int metok_prefill_prune(const void* q_text, const void* k_all, const v
 METOK_API int metok_retention_budgets(double alpha, double r, int stage, const int32_t* N0, int32_t* budget);
 
 /* ------------------------------------------------------------------------- *
+ * (3b) The pruning levels l1, l2, l3 in one call -- section 3.2.2, Eq. 6 and 7.
+ *
+ *   Level s (1-based) is metok_prefill_prune on the tokens that survived level
+ *   s-1, with the budgets of metok_retention_budgets(alpha, r, s, N0); a
+ *   survivor keeps its class.  Everything is enqueued on `stream`; nothing is
+ *   read back between levels.  N0 = {key-event, non-key-event} counts of the
+ *   first level's token_group (classes 0 and 1; HOST): they fix the sizes of all
+ *   levels, n_vis_s = budget_0(s-1) + budget_1(s-1) (n_vis_1 = N0[0] + N0[1]),
+ *   S_s = S - n_vis + n_vis_s, which metok_prune_schedule_sizes returns.
+ *
+ *   Per level s, all DEVICE: q_text [Hq][Lt][dh] and k_all [Hkv][S_s][dh] of that
+ *   layer (rows of the survivors, in order), hidden [S_s][D] / hidden_out
+ *   (both or neither), scores [n_vis_s], keep_idx [S_s], S_out scalar,
+ *   token_group [n_vis_s] (level 1: input; later levels: written), origin
+ *   [n_vis_s] (written: index among the first level's visual tokens).
+ *   `status` DEVICE int32: written 0, or METOK_ERR_INVALID_ARG when N0 does not
+ *   match the first level's classes (later levels are then meaningless).
+ *
+ *   Errors: those of metok_prefill_prune per level; INVALID_ARG also for
+ *   n_levels outside [1, 3], N0 not summing to n_vis, or a level without visual
+ *   tokens.  Workspace: the largest of the levels' (..._schedule_workspace_bytes; 0 = invalid).
+ * ------------------------------------------------------------------------- */
+typedef struct {
+    const void* q_text;
+    const void* k_all;
+    const void* hidden;
+    void* hidden_out;
+    float* scores;
+    int32_t* keep_idx;
+    int32_t* S_out;
+    int32_t* token_group;
+    int32_t* origin;
+} metok_prune_level;
+
+/* HOST: n_vis_of_level[s] for s = 0..n_levels (entry n_levels = survivors of the last level). */
+METOK_API int metok_prune_schedule_sizes(int n_levels, double alpha, double r, const int32_t* N0,
+                        int32_t* n_vis_of_level);
+METOK_API size_t metok_prefill_prune_schedule_workspace_bytes(int n_levels, int dtype, int Hq, int Hkv, int Lt,
+                        int S, int dh, int n_vis, double alpha, double r, const int32_t* N0);
+METOK_API int metok_prefill_prune_schedule(const metok_prune_level* levels, int n_levels, int dtype,
+                        int Hq, int Hkv, int Lt, int S, int dh, int D, int vis_start, int n_vis,
+                        double alpha, double r, const int32_t* N0, float softmax_scale,
+                        int32_t* status, void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
  * (4) KV-cache selection and in-place compaction -- section 3.3.
  *
  *   For every layer l a keep list (ascending positions < S_cur) is chosen:

@@ -34,6 +34,11 @@ class VisionParams(_c.Structure):
                 ("token_inv_norm", _vp)]
 
 
+class PruneLevel(_c.Structure):
+    _fields_ = [("q_text", _vp), ("k_all", _vp), ("hidden", _vp), ("hidden_out", _vp), ("scores", _vp),
+                ("keep_idx", _vp), ("S_out", _vp), ("token_group", _vp), ("origin", _vp)]
+
+
 class MetokError(RuntimeError):
     def __init__(self, fn: str, status: int, text: str, cuda_error: int = 0):
         self.status = status
@@ -57,6 +62,11 @@ _SIGNATURES = {
     "metok_prefill_prune": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i,
                                  _c.POINTER(_c.c_int32), _f, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "metok_retention_budgets": (_i, [_d, _d, _i, _c.POINTER(_c.c_int32), _c.POINTER(_c.c_int32)]),
+    "metok_prune_schedule_sizes": (_i, [_i, _d, _d, _c.POINTER(_c.c_int32), _c.POINTER(_c.c_int32)]),
+    "metok_prefill_prune_schedule_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i, _i, _d, _d,
+                                                          _c.POINTER(_c.c_int32)]),
+    "metok_prefill_prune_schedule": (_i, [_c.POINTER(PruneLevel), _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _d, _d,
+                                          _c.POINTER(_c.c_int32), _f, _vp, _vp, _sz, _vp]),
     "metok_kv_compact_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "metok_kv_compact": (_i, [_c.POINTER(_vp), _c.POINTER(_vp), _i, _i, _i, _i, _i, _i, _i, _i, _d, _i, _i,
                               _vp, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -308,6 +318,64 @@ def metok_prefill_prune(q_text: torch.Tensor, k_all: torch.Tensor, hidden: Optio
     _check("metok_prefill_prune", st)
     out["status"] = ws[:4].view(torch.int32)      # device status word (0, or -5 after a device-side timeout)
     return out
+
+
+def metok_prune_schedule_sizes(n_levels: int, alpha: float, r: float, N0: Sequence[int]) -> List[int]:
+    n0 = (_c.c_int32 * 2)(int(N0[0]), int(N0[1]))
+    out = (_c.c_int32 * (n_levels + 1))()
+    _check("metok_prune_schedule_sizes", lib().metok_prune_schedule_sizes(n_levels, alpha, r, n0, out))
+    return [int(v) for v in out]
+
+
+def metok_prefill_prune_schedule(q_texts: Sequence[torch.Tensor], k_alls: Sequence[torch.Tensor],
+                                 hiddens: Optional[Sequence[torch.Tensor]], vis_start: int, token_group: torch.Tensor,
+                                 alpha: float, r: float, N0: Sequence[int],
+                                 softmax_scale: float) -> List[Dict[str, torch.Tensor]]:
+    """The pruning levels chained in one call: per level the tensors of that layer (rows of the
+    survivors of the level before, in order).  Returns one dict per level."""
+    n_levels = len(q_texts)
+    token_group = _cuda_contig(token_group, "token_group")
+    n_vis = token_group.numel()
+    sizes = metok_prune_schedule_sizes(n_levels, alpha, r, N0)
+    Hq, Lt, dh = q_texts[0].shape
+    Hkv, S, _ = k_alls[0].shape
+    dev = token_group.device
+    D = 0 if hiddens is None else hiddens[0].shape[1]
+    i32 = dict(dtype=torch.int32, device=dev)
+    outs: List[Dict[str, torch.Tensor]] = []
+    arr = (PruneLevel * n_levels)()
+    for s in range(n_levels):
+        q, k_ = _cuda_contig(q_texts[s], "q_text"), _cuda_contig(k_alls[s], "k_all")
+        S_s = S - n_vis + sizes[s]
+        if tuple(k_.shape) != (Hkv, S_s, dh):
+            raise ValueError(f"level {s + 1}: k_all must be {(Hkv, S_s, dh)}, got {tuple(k_.shape)}")
+        h = None if hiddens is None else _cuda_contig(hiddens[s], "hidden")
+        o = {
+            "scores": torch.empty(max(sizes[s], 1), dtype=torch.float32, device=dev),
+            "keep_idx": torch.empty(S_s, **i32), "S_out": torch.zeros(1, **i32),
+            "hidden_out": None if h is None else torch.empty_like(h),
+            "token_group": token_group if s == 0 else torch.empty(max(sizes[s], 1), **i32),
+            "origin": torch.empty(max(sizes[s], 1), **i32), "n_vis": sizes[s], "S": S_s,
+        }
+        arr[s] = PruneLevel(q.data_ptr(), k_.data_ptr(), None if h is None else h.data_ptr(),
+                            None if h is None else o["hidden_out"].data_ptr(), o["scores"].data_ptr(),
+                            o["keep_idx"].data_ptr(), o["S_out"].data_ptr(), o["token_group"].data_ptr(),
+                            o["origin"].data_ptr())
+        o["_inputs"] = (q, k_, h)                               # keep the tensors alive until the caller is done
+        outs.append(o)
+    n0 = (_c.c_int32 * 2)(int(N0[0]), int(N0[1]))
+    L = lib()
+    need = L.metok_prefill_prune_schedule_workspace_bytes(n_levels, _dt(q_texts[0]), Hq, Hkv, Lt, S, dh, n_vis, alpha, r, n0)
+    if need == 0:
+        _check("metok_prefill_prune_schedule", -1)
+    ws = workspace(need, dev)
+    status = torch.zeros(1, **i32)
+    st = L.metok_prefill_prune_schedule(arr, n_levels, _dt(q_texts[0]), Hq, Hkv, Lt, S, dh, D, vis_start, n_vis, alpha, r,
+                                        n0, softmax_scale, _ptr(status), _ptr(ws), ws.numel(), _stream())
+    _check("metok_prefill_prune_schedule", st)
+    for o in outs:
+        o["status"] = status
+    return outs
 
 
 def metok_kv_compact(k_layers: Sequence[torch.Tensor], v_layers: Sequence[torch.Tensor], S_cur: int, policy: int,

@@ -653,3 +653,109 @@ extern "C" int metok_retention_budgets(double alpha, double r, int stage, const 
     budget[1] = bn < N0[1] ? bn : N0[1];
     return METOK_OK;
 }
+
+// --------------------------------------------------------------------------- //
+// The pruning levels chained on the device.
+// --------------------------------------------------------------------------- //
+namespace metok {
+
+// One CTA: origin[i] = i, and the class counts of the first level against the caller's N0.
+__global__ void __launch_bounds__(1024)
+schedule_init_kernel(const int32_t* __restrict__ token_group, int n_vis, int n0_key, int n0_nonkey,
+                     int32_t* __restrict__ origin, int32_t* __restrict__ status) {
+    __shared__ int s_cnt[2];
+    if (threadIdx.x < 2) s_cnt[threadIdx.x] = 0;
+    __syncthreads();
+    int c0 = 0, c1 = 0;
+    for (int i = threadIdx.x; i < n_vis; i += blockDim.x) {
+        origin[i] = i;
+        const int g = token_group[i];
+        c0 += g == 0;
+        c1 += g == 1;
+    }
+    c0 = warp_sum_int(c0);
+    c1 = warp_sum_int(c1);
+    if ((threadIdx.x & 31) == 0) { atomicAdd(&s_cnt[0], c0); atomicAdd(&s_cnt[1], c1); }
+    __syncthreads();
+    if (threadIdx.x == 0)
+        *status = (s_cnt[0] == n0_key && s_cnt[1] == n0_nonkey && s_cnt[0] + s_cnt[1] == n_vis) ? METOK_OK
+                                                                                                 : METOK_ERR_INVALID_ARG;
+}
+
+// Class and origin of the i-th surviving visual token: the keep list holds every position before
+// the visual span, so its entry vis_start + i is that token's position at the level before.
+__global__ void __launch_bounds__(256)
+schedule_propagate_kernel(const int32_t* __restrict__ keep_idx, int vis_start, int n_cur, int n_next,
+                          const int32_t* __restrict__ group, const int32_t* __restrict__ origin,
+                          int32_t* __restrict__ group_next, int32_t* __restrict__ origin_next) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_next) return;
+    int j = keep_idx[vis_start + i] - vis_start;
+    j = j < 0 ? 0 : (j >= n_cur ? n_cur - 1 : j);            // only reached with a wrong N0 (status says so)
+    group_next[i] = group[j];
+    origin_next[i] = origin[j];
+}
+
+}  // namespace metok
+
+extern "C" int metok_prune_schedule_sizes(int n_levels, double alpha, double r, const int32_t* N0,
+                                          int32_t* n_vis_of_level) {
+    if (!N0 || !n_vis_of_level || n_levels < 1 || n_levels > 3) return METOK_ERR_INVALID_ARG;
+    for (int s = 0; s <= n_levels; ++s) {
+        int32_t b[2];
+        const int rc = metok_retention_budgets(alpha, r, s, N0, b);
+        if (rc != METOK_OK) return rc;
+        n_vis_of_level[s] = b[0] + b[1];
+    }
+    return METOK_OK;
+}
+
+extern "C" size_t metok_prefill_prune_schedule_workspace_bytes(int n_levels, int dtype, int Hq, int Hkv, int Lt, int S,
+                                                               int dh, int n_vis, double alpha, double r,
+                                                               const int32_t* N0) {
+    int32_t sizes[4];
+    if (metok_prune_schedule_sizes(n_levels, alpha, r, N0, sizes) != METOK_OK || sizes[0] != n_vis) return 0;
+    size_t need = 0;
+    for (int s = 0; s < n_levels; ++s) {
+        const size_t b = metok_prefill_prune_workspace_bytes(dtype, Hq, Hkv, Lt, S - n_vis + sizes[s], dh, sizes[s]);
+        if (b == 0) return 0;
+        need = b > need ? b : need;
+    }
+    return need;
+}
+
+extern "C" int metok_prefill_prune_schedule(const metok_prune_level* levels, int n_levels, int dtype, int Hq, int Hkv,
+                                            int Lt, int S, int dh, int D, int vis_start, int n_vis, double alpha,
+                                            double r, const int32_t* N0, float softmax_scale, int32_t* status,
+                                            void* ws, size_t ws_bytes, void* stream) {
+    if (!levels || !N0 || !status) return METOK_ERR_INVALID_ARG;
+    int32_t sizes[4];
+    int rc = metok_prune_schedule_sizes(n_levels, alpha, r, N0, sizes);
+    if (rc != METOK_OK) return rc;
+    if (sizes[0] != n_vis || n_vis < 1) return METOK_ERR_INVALID_ARG;
+    for (int s = 0; s < n_levels; ++s) {
+        if (sizes[s] < 1) return METOK_ERR_INVALID_ARG;
+        if (!levels[s].token_group || !levels[s].origin) return METOK_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    schedule_init_kernel<<<1, 1024, 0, st>>>(levels[0].token_group, n_vis, N0[0], N0[1], levels[0].origin, status);
+    METOK_LAUNCH_CHECK();
+    for (int s = 0; s < n_levels; ++s) {
+        const metok_prune_level& lv = levels[s];
+        int32_t budget[2];
+        rc = metok_retention_budgets(alpha, r, s + 1, N0, budget);
+        if (rc != METOK_OK) return rc;
+        const int S_s = S - n_vis + sizes[s];
+        rc = metok_prefill_prune(lv.q_text, lv.k_all, lv.hidden, dtype, Hq, Hkv, Lt, S_s, dh, D, vis_start, sizes[s],
+                                 lv.token_group, 2, budget, softmax_scale, lv.scores, lv.keep_idx, lv.S_out,
+                                 lv.hidden_out, ws, ws_bytes, stream);
+        if (rc != METOK_OK) return rc;
+        if (s + 1 < n_levels) {
+            const metok_prune_level& nx = levels[s + 1];
+            schedule_propagate_kernel<<<ceil_div(sizes[s + 1], 256), 256, 0, st>>>(
+                lv.keep_idx, vis_start, sizes[s], sizes[s + 1], lv.token_group, lv.origin, nx.token_group, nx.origin);
+            METOK_LAUNCH_CHECK();
+        }
+    }
+    return METOK_OK;
+}

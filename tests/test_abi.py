@@ -160,3 +160,33 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         B.lib()
+
+
+def test_prune_schedule_sizes_and_validation(lib):
+    """Sizes of the levels follow Eq. 6/7 on the host; bad schedules are rejected before any launch."""
+    assert B.metok_prune_schedule_sizes(3, 0.5, 0.55, (200, 100)) == [300, 110 + 28, 61, 0]
+    from oracle import metok_oracle as O
+    for alpha, r, N0 in [(0.5, 0.76, (3000, 3272)), (0.5, 0.65, (1, 1)), (0.3, 0.9, (7, 0))]:
+        want = [int(O.retention_budgets(alpha, r, s, N0).sum()) for s in range(4)]
+        assert B.metok_prune_schedule_sizes(3, alpha, r, N0) == want
+    with pytest.raises(B.MetokError):
+        B.metok_prune_schedule_sizes(4, 0.5, 0.5, (1, 1))
+    fake, null = ctypes.c_void_p(0x10000), ctypes.c_void_p(0)
+    lv = (B.PruneLevel * 3)()
+    for s in range(3):
+        lv[s] = B.PruneLevel(*([0x10000] * 9))
+    n0 = (ctypes.c_int32 * 2)(200, 100)
+    fn = lib.metok_prefill_prune_schedule
+    args = [lv, 3, B.BF16, 28, 4, 16, 316, 128, 3584, 0, 300, 0.5, 0.55, n0, 0.088, fake, fake, 1 << 26, null]
+
+    def call(idx, val):
+        a = list(args); a[idx] = val
+        return fn(*a)
+    assert call(1, 0) == -1 and call(1, 4) == -1              # number of levels
+    assert call(10, 299) == -1                                # N0 does not sum to n_vis
+    assert call(12, 1.5) == -1                                # r
+    assert call(15, null) == -1                               # status pointer
+    n0_empty = (ctypes.c_int32 * 2)(0, 300)                   # no key-event tokens: level 3 would get no visual token
+    assert call(13, n0_empty) == -1
+    assert lib.metok_prefill_prune_schedule_workspace_bytes(3, B.BF16, 28, 4, 16, 316, 128, 300, 0.5, 0.55, n0) > 0
+    assert lib.metok_prefill_prune_schedule_workspace_bytes(3, B.BF16, 28, 4, 16, 316, 128, 299, 0.5, 0.55, n0) == 0

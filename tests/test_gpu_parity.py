@@ -470,3 +470,61 @@ def test_cuda_graph_replay_equals_eager_calls():
         m = new_len[layer]
         assert same(eager["kv"]["keep_idx"][layer, :m], replay["kv"]["keep_idx"][layer, :m])
         assert same(ks_e[layer][:, :m], ks_g[layer][:, :m]) and same(vs_e[layer][:, :m], vs_g[layer][:, :m])
+
+
+@pytest.mark.parametrize("name", ["frames32", "small24", "tiny"])
+def test_prefill_prune_schedule_three_levels_in_one_call(name):
+    """The pruning levels chained on the device (classes and origins of the survivors handed from
+    level to level without a read-back) against the oracle's chain."""
+    cfg = W.CONFIGS[name]
+    vis = vis_of(name)
+    groups = W.token_groups(cfg, cfg.Nv, vis=vis)
+    N0 = [int((groups == 0).sum()), int((groups == 1).sum())]
+    n_levels = 3 if N0[0] > 3 else 2
+    r = cfg.keep_prefill
+    sizes = B.metok_prune_schedule_sizes(n_levels, cfg.alpha, r, N0)
+    # inputs of level s depend on who survived level s-1: generated along the oracle's chain
+    Qs, Ks, hid = [], [], []
+    g_s = groups
+    for s in range(1, n_levels + 1):
+        assert g_s.size == sizes[s - 1]
+        pf = W.prefill_inputs(cfg, s, g_s.size, g_s)
+        Qs.append(pf["Q"]); Ks.append(pf["K"])
+        hid.append(W.payload_torch(W.hidden_salt(cfg, s), pf["S"], cfg.D, cfg.dtype, "cuda"))
+        want_s = O.prune_schedule(Qs, Ks, groups, cfg.alpha, r, 0, O.f32(cfg.dh ** -0.5))
+        k_ = want_s[-1]["keep_idx"]
+        g_s = g_s[k_[k_ < g_s.size]]
+    want = want_s
+    got = B.metok_prefill_prune_schedule([P.to_torch(q, cfg.dtype) for q in Qs], [P.to_torch(k_, cfg.dtype) for k_ in Ks],
+                                         hid, 0, torch.from_numpy(groups.astype(np.int32)).cuda(), cfg.alpha, r, N0,
+                                         cfg.dh ** -0.5)
+    torch.cuda.synchronize()
+    assert int(got[0]["status"].item()) == 0
+    for s in range(n_levels):
+        w, g = want[s], got[s]
+        n_in = sizes[s]
+        assert g["n_vis"] == n_in == w["token_group"].size
+        assert np.array_equal(g["token_group"][:n_in].cpu().numpy(), w["token_group"]), s
+        assert np.array_equal(g["origin"][:n_in].cpu().numpy(), w["origin"]), s
+        P.check_scores(g["scores"][:n_in].cpu().numpy(), w["scores"], cfg.dtype, f"scores of level {s + 1}")
+        S_out = int(g["S_out"].item())
+        assert S_out == w["S_out"] == g["S"] - n_in + sizes[s + 1]
+        keep = g["keep_idx"][:S_out].cpu().numpy()
+        mism = P.check_index_set(keep, w["keep_idx"], lambda u: u < n_in and bool(w["near_tie"][u]), "keep_idx")
+        ho = g["hidden_out"][:S_out]
+        ref = hid[s][torch.from_numpy(keep.astype(np.int64)).cuda()]
+        assert torch.equal(ho.view(torch.int16) if ho.dtype == torch.bfloat16 else ho,
+                           ref.view(torch.int16) if ref.dtype == torch.bfloat16 else ref)
+        if mism:                                               # a near-tie went the other way: later levels see other tokens
+            break
+    # wrong class counts are reported by the device status word
+    bad = [N0[0] + 1, N0[1] - 1]
+    if bad[1] >= 0 and min(B.metok_prune_schedule_sizes(n_levels, cfg.alpha, r, bad)[:n_levels]) > 0:
+        sz = B.metok_prune_schedule_sizes(n_levels, cfg.alpha, r, bad)
+        Ks_bad = [torch.zeros((cfg.Hkv, Ks[0].shape[1] - cfg.Nv + sz[s], cfg.dh), dtype=P.to_torch(Ks[0], cfg.dtype).dtype,
+                              device="cuda") for s in range(n_levels)]
+        out = B.metok_prefill_prune_schedule([P.to_torch(q, cfg.dtype) for q in Qs], Ks_bad, None, 0,
+                                             torch.from_numpy(groups.astype(np.int32)).cuda(), cfg.alpha, r, bad,
+                                             cfg.dh ** -0.5)
+        torch.cuda.synchronize()
+        assert int(out[0]["status"].item()) == -1

@@ -528,3 +528,42 @@ def test_prefill_prune_schedule_three_levels_in_one_call(name):
                                              cfg.dh ** -0.5)
         torch.cuda.synchronize()
         assert int(out[0]["status"].item()) == -1
+
+
+def test_two_videos_on_two_streams_do_not_share_scratch():
+    """Independent videos in flight on streams of their own (the benchmark's batch): each call takes
+    its scratch per stream, so the results equal those of the same calls made one after the other."""
+    cfg = W.CONFIGS["frames32"]
+    vis = vis_of("frames32")
+    p = B.vision_params(cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+    rng = np.random.default_rng(5)
+    Va = vis["V"]
+    Vb = W.quantize((Va[::-1] + 0.05 * rng.standard_normal(Va.shape)).astype(np.float32), cfg.dtype)
+    td = P.to_torch(vis["t"], cfg.dtype)
+    vids = [P.to_torch(Va, cfg.dtype), P.to_torch(Vb, cfg.dtype)]
+
+    def one(V):
+        seg = B.metok_segment_score_events(V, cfg.k, td)
+        cv = B.metok_compress_vision(V, seg["event_offsets"], td, p, scored=seg)
+        return seg, cv
+
+    alone = []
+    for V in vids:
+        alone.append(one(V))
+        torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for _ in range(3):
+        both = []
+        for V, st in zip(vids, streams):
+            with torch.cuda.stream(st):
+                both.append(one(V))
+        torch.cuda.synchronize()
+        for (seg_a, cv_a), (seg_b, cv_b) in zip(alone, both):
+            assert torch.equal(seg_a["event_offsets"], seg_b["event_offsets"])
+            assert torch.equal(seg_a["token_score"], seg_b["token_score"])
+            n = int(cv_a["n_out"].item())
+            assert n == int(cv_b["n_out"].item())
+            assert torch.equal(cv_a["out_src"][:n], cv_b["out_src"][:n])
+            assert torch.equal(cv_a["assign"], cv_b["assign"])
+            assert torch.equal(cv_a["out_feats"][:n].view(torch.int16), cv_b["out_feats"][:n].view(torch.int16))
+    assert not torch.equal(alone[0][1]["assign"], alone[1][1]["assign"])      # the two videos do differ

@@ -265,6 +265,25 @@ METOK_API int metok_prefill_prune(const void* q_text, const void* k_all, const v
                         float softmax_scale, float* scores, int32_t* keep_idx, int32_t* S_out,
                         void* hidden_out, void* ws, size_t ws_bytes, void* stream);
 
+/* The two halves of metok_prefill_prune as calls of their own, for a caller that shards the
+ * attention heads over several GPUs (each rank: its own query heads and the KV heads they use,
+ * whole groups) and adds the ranks' scores before selecting:
+ *   metok_attention_scores: scores[j] = (sum over THIS call's heads h and the Lt text queries q of
+ *     softmax(...)[vis_start + j]) / rows_total, rows_total = all ranks' Hq * Lt (0: this call's),
+ *     so that the sum of the ranks' scores is metok_prefill_prune's score.  Arguments, layouts,
+ *     errors and workspace size as metok_prefill_prune; rows_total < Hq*Lt (and != 0) is INVALID_ARG.
+ *   metok_prune_by_scores: the class-wise top-k and the hidden-state gather of
+ *     metok_prefill_prune on the caller's DEVICE scores[n_vis]; the visual span may lie anywhere
+ *     in [0, S].  Workspace: metok_prune_by_scores_workspace_bytes(). */
+METOK_API int metok_attention_scores(const void* q_text, const void* k_all, int dtype, int Hq, int Hkv, int Lt,
+                        int S, int dh, int vis_start, int n_vis, float softmax_scale, int rows_total,
+                        float* scores, void* ws, size_t ws_bytes, void* stream);
+METOK_API size_t metok_prune_by_scores_workspace_bytes(void);
+METOK_API int metok_prune_by_scores(const float* scores, const void* hidden, int dtype, int S, int D,
+                        int vis_start, int n_vis, const int32_t* token_group, int G,
+                        const int32_t* group_budget, int32_t* keep_idx, int32_t* S_out, void* hidden_out,
+                        void* ws, size_t ws_bytes, void* stream);
+
 /* Eq. 6 and 7: token budgets after pruning level `stage` (1, 2, 3 = layers l1,
  * l2, l3; 0 = before l1) for N0 = {key-event tokens, non-key-event tokens}
  * first passed into the LLM:  R_key = 1, r, r^2, 0 ;  R_nonkey = 1, alpha*r, 0, 0.

@@ -61,6 +61,10 @@ _SIGNATURES = {
     "metok_prefill_prune_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "metok_prefill_prune": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i,
                                  _c.POINTER(_c.c_int32), _f, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "metok_attention_scores": (_i, [_vp, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _sz, _vp]),
+    "metok_prune_by_scores_workspace_bytes": (_sz, []),
+    "metok_prune_by_scores": (_i, [_vp, _vp, _i, _i, _i, _i, _i, _vp, _i, _c.POINTER(_c.c_int32), _vp, _vp, _vp,
+                                   _vp, _sz, _vp]),
     "metok_retention_budgets": (_i, [_d, _d, _i, _c.POINTER(_c.c_int32), _c.POINTER(_c.c_int32)]),
     "metok_prune_schedule_sizes": (_i, [_i, _d, _d, _c.POINTER(_c.c_int32), _c.POINTER(_c.c_int32)]),
     "metok_prefill_prune_schedule_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i, _i, _d, _d,
@@ -318,6 +322,80 @@ def metok_prefill_prune(q_text: torch.Tensor, k_all: torch.Tensor, hidden: Optio
     _check("metok_prefill_prune", st)
     out["status"] = ws[:4].view(torch.int32)      # device status word (0, or -5 after a device-side timeout)
     return out
+
+
+def metok_attention_scores(q_text: torch.Tensor, k_all: torch.Tensor, vis_start: int, n_vis: int,
+                           softmax_scale: float, rows_total: int = 0,
+                           scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The scoring half of metok_prefill_prune for the heads given; `rows_total` = Hq * Lt over all
+    ranks when the heads are sharded (the ranks' results then add up to the full score)."""
+    q_text = _cuda_contig(q_text, "q_text")
+    k_all = _cuda_contig(k_all, "k_all")
+    Hq, Lt, dh = q_text.shape
+    Hkv, S, _ = k_all.shape
+    dev = q_text.device
+    if scores is None:
+        scores = torch.empty(n_vis, dtype=torch.float32, device=dev)
+    L = lib()
+    ws = workspace(L.metok_prefill_prune_workspace_bytes(_dt(q_text), Hq, Hkv, Lt, S, dh, n_vis), dev)
+    st = L.metok_attention_scores(_ptr(q_text), _ptr(k_all), _dt(q_text), Hq, Hkv, Lt, S, dh, vis_start, n_vis,
+                                  softmax_scale, rows_total, _ptr(scores), _ptr(ws), ws.numel(), _stream())
+    _check("metok_attention_scores", st)
+    return scores
+
+
+def metok_prune_by_scores(scores: torch.Tensor, hidden: Optional[torch.Tensor], S: int, vis_start: int,
+                          token_group: torch.Tensor, group_budget: Sequence[int],
+                          dtype: Optional[torch.dtype] = None) -> Dict[str, torch.Tensor]:
+    """The selection half of metok_prefill_prune on scores the caller holds."""
+    scores = _cuda_contig(scores, "scores")
+    token_group = _cuda_contig(token_group, "token_group")
+    n_vis = scores.numel()
+    dev = scores.device
+    D = 0
+    if hidden is not None:
+        hidden = _cuda_contig(hidden, "hidden")
+        D = hidden.shape[1]
+        dtype = hidden.dtype
+    code = F32 if dtype in (None, torch.float32) else BF16
+    G = len(group_budget)
+    budgets = (_c.c_int32 * G)(*[int(b) for b in group_budget])
+    out = {"scores": scores, "keep_idx": torch.empty(S, dtype=torch.int32, device=dev),
+           "S_out": torch.zeros(1, dtype=torch.int32, device=dev),
+           "hidden_out": None if hidden is None else torch.empty_like(hidden)}
+    L = lib()
+    ws = workspace(L.metok_prune_by_scores_workspace_bytes(), dev)
+    st = L.metok_prune_by_scores(_ptr(scores), _ptr(hidden), code, S, D, vis_start, n_vis, _ptr(token_group), G,
+                                 budgets, _ptr(out["keep_idx"]), _ptr(out["S_out"]), _ptr(out["hidden_out"]), _ptr(ws),
+                                 ws.numel(), _stream())
+    _check("metok_prune_by_scores", st)
+    out["status"] = ws[:4].view(torch.int32)
+    return out
+
+
+def head_shard(Hq: int, Hkv: int, rank: int, world: int):
+    """Query heads [h0, h1) and KV heads [g0, g1) of `rank` when whole KV-head groups are dealt out."""
+    if Hq % Hkv or Hkv % world:
+        raise ValueError(f"{Hkv} KV heads (of {Hq} query heads) do not split over {world} ranks")
+    per, rep = Hkv // world, Hq // Hkv
+    return (rank * per * rep, (rank + 1) * per * rep), (rank * per, (rank + 1) * per)
+
+
+def metok_prefill_prune_sharded(q_text_local: torch.Tensor, k_all_local: torch.Tensor, hidden: Optional[torch.Tensor],
+                                vis_start: int, n_vis: int, token_group: torch.Tensor, group_budget: Sequence[int],
+                                softmax_scale: float, group=None) -> Dict[str, torch.Tensor]:
+    """One pruning level with the attention heads sharded over the ranks of `group` (head_shard): every
+    rank scores with its own heads, one all-reduce (sum) of the n_vis scores, then every rank runs the
+    same selection on the same scores."""
+    import torch.distributed as dist
+    world = dist.get_world_size(group) if dist.is_available() and dist.is_initialized() else 1
+    Hq_local, Lt, _ = q_text_local.shape
+    scores = metok_attention_scores(q_text_local, k_all_local, vis_start, n_vis, softmax_scale,
+                                    rows_total=Hq_local * world * Lt)
+    if world > 1:
+        dist.all_reduce(scores, op=dist.ReduceOp.SUM, group=group)
+    return metok_prune_by_scores(scores, hidden, k_all_local.shape[1], vis_start, token_group, group_budget,
+                                 dtype=q_text_local.dtype)
 
 
 def metok_prune_schedule_sizes(n_levels: int, alpha: float, r: float, N0: Sequence[int]) -> List[int]:

@@ -540,11 +540,11 @@ static PrefillWs carve_prefill(Carver& cv, const AttnDims& dm, bool mma) {
     return w;
 }
 
-static int launch_score_reduce(const PrefillWs& w, const AttnDims& dm, float* scores, cudaStream_t st) {
+static int launch_score_reduce(const PrefillWs& w, const AttnDims& dm, float inv_rows, float* scores, cudaStream_t st) {
     {
         METOK_TIMED("attn_score_reduce_kernel", st);
-        launch_chained(attn_score_reduce_kernel, dim3(ceil_div(dm.n_vis, 256)), dim3(256), 0, st, w.part_col, w.n_planes, dm.n_vis,
-                                                                      1.0f / (float)(dm.Hq * dm.Lt), scores);
+        launch_chained(attn_score_reduce_kernel, dim3(ceil_div(dm.n_vis, 256)), dim3(256), 0, st, w.part_col, w.n_planes,
+                       dm.n_vis, inv_rows, scores);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;
@@ -552,7 +552,7 @@ static int launch_score_reduce(const PrefillWs& w, const AttnDims& dm, float* sc
 
 template <typename T>
 static int launch_attn_scores(const void* q_text, const void* k_all, const AttnDims& dm, const PrefillWs& w,
-                              float* scores, cudaStream_t st) {
+                              float inv_rows, float* scores, cudaStream_t st) {
     const size_t smem = (size_t)2 * dm.dh * kAtLD * sizeof(float);
     METOK_CUDA_TRY(cudaFuncSetAttribute(attn_stats_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     METOK_CUDA_TRY(cudaFuncSetAttribute(attn_colsum_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -570,12 +570,28 @@ static int launch_attn_scores(const void* q_text, const void* k_all, const AttnD
                                                    w.part_col);
     }
     METOK_LAUNCH_CHECK();
-    return launch_score_reduce(w, dm, scores, st);
+    return launch_score_reduce(w, dm, inv_rows, scores, st);
 }
 
 }  // namespace metok
 
 using namespace metok;
+
+// a5 as the calls run it: the status word cleared, then the two passes and the plane sum;
+// scores[j] = inv_rows * (sum over this call's heads and text queries of the probabilities).
+static int run_attention_scores(const void* q_text, const void* k_all, int dtype, const AttnDims& dm,
+                                const PrefillWs& w, float softmax_scale, float inv_rows, float* scores,
+                                cudaStream_t st) {
+    const bool mma = use_mma_attn(dtype, dm.dh);
+    if (!mma) METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));   // else attn_stats_mma_kernel clears it
+    if (mma) {
+        const int rc = launch_attn_scores_mma(q_text, k_all, dm.Hq, dm.Hkv, dm.Lt, dm.S, dm.dh, dm.vis_start, dm.n_vis,
+                                              softmax_scale, w.part_m, w.part_l, w.part_col, w.status, st);
+        return rc == METOK_OK ? launch_score_reduce(w, dm, inv_rows, scores, st) : rc;
+    }
+    return dtype == METOK_F32 ? launch_attn_scores<float>(q_text, k_all, dm, w, inv_rows, scores, st)
+                              : launch_attn_scores<__nv_bfloat16>(q_text, k_all, dm, w, inv_rows, scores, st);
+}
 
 extern "C" size_t metok_prefill_prune_workspace_bytes(int dtype, int Hq, int Hkv, int Lt, int S, int dh, int n_vis) {
     if (Hq < 1 || Hkv < 1 || Lt < 1 || S < 1 || dh < 1 || n_vis < 1 || Hq % Hkv) return 0;
@@ -612,19 +628,9 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
     AttnDims dm = make_dims(Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale);
-    const bool mma = use_mma_attn(dtype, dh);
     Carver cv(ws);
-    PrefillWs w = carve_prefill(cv, dm, mma);
-    if (!mma) METOK_CUDA_TRY(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));   // else attn_stats_mma_kernel clears it
-    int rc;
-    if (mma) {
-        rc = launch_attn_scores_mma(q_text, k_all, Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale, w.part_m,
-                                    w.part_l, w.part_col, w.status, st);
-        if (rc == METOK_OK) rc = launch_score_reduce(w, dm, scores, st);
-    } else {
-        rc = dtype == METOK_F32 ? launch_attn_scores<float>(q_text, k_all, dm, w, scores, st)
-                                : launch_attn_scores<__nv_bfloat16>(q_text, k_all, dm, w, scores, st);
-    }
+    PrefillWs w = carve_prefill(cv, dm, use_mma_attn(dtype, dh));
+    int rc = run_attention_scores(q_text, k_all, dtype, dm, w, softmax_scale, 1.0f / (float)(Hq * Lt), scores, st);
     if (rc != METOK_OK) return rc;
     rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, 1, S_out,
                            nullptr, 1, st);
@@ -635,6 +641,57 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
         if (rc != METOK_OK) return rc;
     }
     return METOK_OK;
+}
+
+extern "C" int metok_attention_scores(const void* q_text, const void* k_all, int dtype, int Hq, int Hkv, int Lt, int S,
+                                      int dh, int vis_start, int n_vis, float softmax_scale, int rows_total,
+                                      float* scores, void* ws, size_t ws_bytes, void* stream) {
+    if (!q_text || !k_all || !scores) return METOK_ERR_INVALID_ARG;
+    if (dtype != METOK_F32 && dtype != METOK_BF16) return METOK_ERR_INVALID_ARG;
+    if (Hq < 1 || Hkv < 1 || Lt < 1 || S < 1 || dh < 1 || n_vis < 1) return METOK_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0 || Lt > S) return METOK_ERR_INVALID_ARG;
+    if (vis_start < 0 || (long long)vis_start + n_vis > (long long)S - Lt) return METOK_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || !aligned16(q_text) || !aligned16(k_all)) return METOK_ERR_INVALID_ARG;
+    if (rows_total != 0 && (long long)rows_total < (long long)Hq * Lt) return METOK_ERR_INVALID_ARG;
+    if (dtype == METOK_BF16 && dh != 64 && dh != 128) return METOK_ERR_UNSUPPORTED;
+    if (dtype == METOK_F32 && (dh > 128 || dh % 4 != 0)) return METOK_ERR_UNSUPPORTED;
+    const size_t need = metok_prefill_prune_workspace_bytes(dtype, Hq, Hkv, Lt, S, dh, n_vis);
+    if (!ws || ws_bytes < need || !aligned16(ws)) return METOK_ERR_WORKSPACE;
+    AttnDims dm = make_dims(Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale);
+    Carver cv(ws);
+    PrefillWs w = carve_prefill(cv, dm, use_mma_attn(dtype, dh));
+    const float inv_rows = 1.0f / (float)(rows_total ? rows_total : Hq * Lt);
+    return run_attention_scores(q_text, k_all, dtype, dm, w, softmax_scale, inv_rows, scores,
+                                reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t metok_prune_by_scores_workspace_bytes(void) { return 1024; }
+
+extern "C" int metok_prune_by_scores(const float* scores, const void* hidden, int dtype, int S, int D, int vis_start,
+                                     int n_vis, const int32_t* token_group, int G, const int32_t* group_budget,
+                                     int32_t* keep_idx, int32_t* S_out, void* hidden_out, void* ws, size_t ws_bytes,
+                                     void* stream) {
+    if (!scores || !token_group || !group_budget || !keep_idx || !S_out) return METOK_ERR_INVALID_ARG;
+    if ((hidden == nullptr) != (hidden_out == nullptr)) return METOK_ERR_INVALID_ARG;
+    if (dtype != METOK_F32 && dtype != METOK_BF16) return METOK_ERR_INVALID_ARG;
+    if (S < 1 || n_vis < 1 || (hidden && D < 1)) return METOK_ERR_INVALID_ARG;
+    if (vis_start < 0 || (long long)vis_start + n_vis > (long long)S) return METOK_ERR_INVALID_ARG;
+    if (G < 1 || G > METOK_MAX_GROUPS) return METOK_ERR_INVALID_ARG;
+    for (int g = 0; g < G; ++g)
+        if (group_budget[g] < 0) return METOK_ERR_INVALID_ARG;
+    if (hidden && (!aligned16(hidden) || !aligned16(hidden_out))) return METOK_ERR_INVALID_ARG;
+    const int eb = dtype == METOK_F32 ? 4 : 2;
+    if (hidden && ((long long)D * eb) % 16 != 0) return METOK_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < metok_prune_by_scores_workspace_bytes() || !aligned16(ws)) return METOK_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int32_t* status = reinterpret_cast<int32_t*>(ws);
+    METOK_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    int rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, 1, S_out,
+                               nullptr, 1, st);
+    if (rc != METOK_OK) return rc;
+    if (hidden)
+        rc = launch_gather_rows_bulk(hidden, hidden_out, keep_idx, S_out, (size_t)D * eb, status, "gather_rows_kernel", st);
+    return rc;
 }
 
 extern "C" int metok_retention_budgets(double alpha, double r, int stage, const int32_t* N0, int32_t* budget) {

@@ -567,3 +567,46 @@ def test_two_videos_on_two_streams_do_not_share_scratch():
             assert torch.equal(cv_a["assign"], cv_b["assign"])
             assert torch.equal(cv_a["out_feats"][:n].view(torch.int16), cv_b["out_feats"][:n].view(torch.int16))
     assert not torch.equal(alone[0][1]["assign"], alone[1][1]["assign"])      # the two videos do differ
+
+
+@pytest.mark.parametrize("name,world", [("frames32", 2), ("frames32", 4), ("tiny", 1), ("small24", 2)])
+def test_head_sharded_scores_then_selection(name, world):
+    """The two halves of the pruning call on their own: the scores of each shard of KV-head groups
+    (normalised by all heads' rows) add up to the unsharded scores, and the selection on the sum is
+    the fused call's.  The shards run one after the other on this GPU; a sum on the device stands in
+    for the all-reduce between ranks."""
+    cfg = W.CONFIGS[name]
+    vis = vis_of(name)
+    groups, budgets = _prefill_stage_inputs(cfg, 1, vis)
+    pf = W.prefill_inputs(cfg, 1, cfg.Nv, groups)
+    Q, K = P.to_torch(pf["Q"], cfg.dtype), P.to_torch(pf["K"], cfg.dtype)
+    hidden = W.payload_torch(W.hidden_salt(cfg, 1), pf["S"], cfg.D, cfg.dtype, "cuda")
+    grp = torch.from_numpy(groups.astype(np.int32)).cuda()
+    scale = cfg.dh ** -0.5
+    fused = B.metok_prefill_prune(Q, K, hidden, 0, cfg.Nv, grp, budgets, scale)
+    total = torch.zeros(cfg.Nv, dtype=torch.float32, device="cuda")
+    for rank in range(world):
+        (h0, h1), (g0, g1) = B.head_shard(cfg.Hq, cfg.Hkv, rank, world)
+        part = B.metok_attention_scores(Q[h0:h1].contiguous(), K[g0:g1].contiguous(), 0, cfg.Nv, scale,
+                                        rows_total=cfg.Hq * cfg.Lt)
+        total += part
+    torch.cuda.synchronize()
+    want_scores = O.attention_scores(pf["Q"], pf["K"], 0, cfg.Nv, O.f32(scale))
+    P.check_scores(total.cpu().numpy(), want_scores, cfg.dtype, "sum of the shards' scores")
+    assert torch.allclose(total, fused["scores"], rtol=2e-5, atol=1e-9)
+    if world == 1:
+        assert torch.equal(total, fused["scores"])
+    got = B.metok_prune_by_scores(fused["scores"].clone(), hidden, pf["S"], 0, grp, budgets)
+    torch.cuda.synchronize()
+    n = int(fused["S_out"].item())
+    assert int(got["S_out"].item()) == n and int(got["status"].item()) == 0
+    assert torch.equal(got["keep_idx"][:n], fused["keep_idx"][:n])
+    assert torch.equal(got["hidden_out"][:n].view(torch.int16) if cfg.dtype == "bf16" else got["hidden_out"][:n],
+                       fused["hidden_out"][:n].view(torch.int16) if cfg.dtype == "bf16" else fused["hidden_out"][:n])
+    # selection on the summed scores against the oracle's selection (near-ties aside)
+    sel = B.metok_prune_by_scores(total, None, pf["S"], 0, grp, budgets)
+    want = O.weighted_topk(want_scores, groups, budgets, pf["S"], 0)
+    m = int(sel["S_out"].item())
+    assert m == want["S_out"]
+    P.check_index_set(sel["keep_idx"][:m].cpu().numpy(), want["keep_idx"],
+                      lambda u: u < cfg.Nv and bool(want["near_tie"][u]), "keep_idx from summed scores")

@@ -216,6 +216,9 @@ typedef struct metok_vision_params {
     int    s1_nonkey, s2_nonkey;  /* POOL: the same for non-key events (the paper: s/alpha) */
     const float* token_inv_norm;  /* NULL, or DEVICE float [T*N] from metok_segment_score_events: then the
                                      token_score argument is an INPUT and the Eq. 5 pass over V is skipped */
+    const uint8_t* key_events_given;  /* NULL, or DEVICE uint8 [k]: the key events are the caller's (non-zero =
+                                         key) instead of the ceil(alpha*k) best-scored ones -- the ablation
+                                         with randomly chosen key events; event_is_key returns them */
 } metok_vision_params;
 
 METOK_API int    metok_compress_vision_bound(int T, int N, int k, const metok_vision_params* p);

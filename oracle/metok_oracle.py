@@ -253,11 +253,14 @@ def merge_assign(V: np.ndarray, N: int, event_offsets: np.ndarray, is_key_token:
 
 def compress_vision(V: np.ndarray, t: np.ndarray, event_offsets: np.ndarray, alpha: float,
                     keep_key: float, keep_nonkey: float, dtype: str,
-                    event_agg: int = AGG_MEAN) -> Dict[str, np.ndarray]:
-    """a2 + a3 + a4 chained, as the library's stage-1 call runs them."""
+                    event_agg: int = AGG_MEAN, key_events_given: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """a2 + a3 + a4 chained, as the library's stage-1 call runs them.  `key_events_given` (bool [k])
+    replaces Eq. 5's choice of key events: the ablation with randomly chosen key events."""
     T, N, _ = V.shape
     s = token_relevance(V, t)
     ev = key_events(s, T, N, event_offsets, alpha, event_agg)
+    if key_events_given is not None:
+        ev["event_is_key"] = np.asarray(key_events_given).astype(ev["event_is_key"].dtype)
     sel = key_token_topk(s, N, event_offsets, ev["event_is_key"], keep_key, keep_nonkey)
     mer = merge_assign(V, N, event_offsets, sel["is_key_token"], dtype)
     out = {"token_score": s}

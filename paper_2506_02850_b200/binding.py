@@ -31,7 +31,7 @@ _vp, _i, _sz, _f, _d = _c.c_void_p, _c.c_int, _c.c_size_t, _c.c_float, _c.c_doub
 class VisionParams(_c.Structure):
     _fields_ = [("alpha", _d), ("event_agg", _i), ("mode", _i), ("keep_key", _d), ("keep_nonkey", _d),
                 ("beta", _d), ("s1", _i), ("s2", _i), ("s1_nonkey", _i), ("s2_nonkey", _i),
-                ("token_inv_norm", _vp)]
+                ("token_inv_norm", _vp), ("key_events_given", _vp)]
 
 
 class PruneLevel(_c.Structure):
@@ -228,7 +228,7 @@ def metok_segment_score_events(feats: torch.Tensor, k: int, text_emb: torch.Tens
 def vision_params(alpha: float, keep_key: float = 1.0, keep_nonkey: float = 1.0, event_agg: int = AGG_MEAN,
                   mode: int = MODE_TOPK_MERGE, beta: float = 0.5, s1: int = 2, s2: int = 3,
                   s1_nonkey: int = 4, s2_nonkey: int = 6) -> VisionParams:
-    return VisionParams(alpha, event_agg, mode, keep_key, keep_nonkey, beta, s1, s2, s1_nonkey, s2_nonkey, None)
+    return VisionParams(alpha, event_agg, mode, keep_key, keep_nonkey, beta, s1, s2, s1_nonkey, s2_nonkey, None, None)
 
 
 def metok_compress_vision_bound(T: int, N: int, k: int, p: VisionParams) -> int:
@@ -241,9 +241,11 @@ def metok_compress_vision_bound(T: int, N: int, k: int, p: VisionParams) -> int:
 def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text_emb: torch.Tensor,
                           p: VisionParams, cap: Optional[int] = None,
                           out: Optional[Dict[str, torch.Tensor]] = None,
-                          scored: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+                          scored: Optional[Dict[str, torch.Tensor]] = None,
+                          key_events: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
     """`scored` (the result of metok_segment_score_events on the same feats and text) makes the call
-    skip its own scoring pass over `feats`."""
+    skip its own scoring pass over `feats`; `key_events` (uint8 [k] on the device) replaces the
+    call's own choice of key events."""
     feats = _cuda_contig(feats, "feats")
     event_offsets = _cuda_contig(event_offsets, "event_offsets")
     text_emb = _cuda_contig(text_emb, "text_emb")
@@ -271,6 +273,12 @@ def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text
         out["token_score"] = scored["token_score"]
         p = VisionParams.from_buffer_copy(p)
         p.token_inv_norm = scored["token_inv_norm"].data_ptr()
+    if key_events is not None:
+        key_events = _cuda_contig(key_events, "key_events")
+        if key_events.dtype != torch.uint8 or key_events.numel() != k:
+            raise ValueError("key_events must be uint8 [k]")
+        p = VisionParams.from_buffer_copy(p)
+        p.key_events_given = key_events.data_ptr()
     need = L.metok_compress_vision_workspace_bytes(_dt(feats), T, N, d, k, cap, _c.byref(p))
     ws = workspace(need, dev)
     st = L.metok_compress_vision(_ptr(feats), _dt(feats), T, N, d, _ptr(event_offsets), k, _ptr(text_emb),

@@ -113,6 +113,7 @@ struct PlanParams {
     int Tn, N, k, n_key_events, event_agg, mode, tile_rows, chunk_cols;
     int grid, s1, s2, s1_nonkey, s2_nonkey;     // POOL: side of the token grid and the four strides
     double keep_key, keep_nonkey, beta;
+    const uint8_t* key_given;                   // the caller's key events, or null
 };
 
 // The workspace regions that later kernels of the call expect cleared: written here, at the start of
@@ -215,8 +216,9 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
             const float w = s_score[j];
             rank += (w > v) || (w == v && j < e);
         }
-        event_is_key[e] = (uint8_t)(rank < pp.n_key_events);
-        s_key[e] = (unsigned char)(rank < pp.n_key_events);
+        const bool key = pp.key_given ? pp.key_given[e] != 0 : rank < pp.n_key_events;
+        event_is_key[e] = (uint8_t)key;
+        s_key[e] = (unsigned char)key;
     }
     __syncthreads();
     if (pp.mode == METOK_MODE_TOPK_MERGE) {
@@ -1272,6 +1274,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     pp.event_agg = p->event_agg; pp.mode = p->mode; pp.tile_rows = mma ? kMmaBM : kMergeTM;
     pp.chunk_cols = kMmaBN;
     pp.keep_key = p->keep_key; pp.keep_nonkey = p->keep_nonkey; pp.beta = p->beta;
+    pp.key_given = p->key_events_given;
     pp.grid = 1;
     while (pp.grid * pp.grid < N) ++pp.grid;
     pp.s1 = p->s1; pp.s2 = p->s2; pp.s1_nonkey = p->s1_nonkey; pp.s2_nonkey = p->s2_nonkey;

@@ -46,13 +46,15 @@ def segment_case(V: np.ndarray, dtype: str, k: int, sim_mode: int = 0) -> Dict[s
 
 
 def compress_case(V: np.ndarray, t: np.ndarray, offs: np.ndarray, dtype: str, alpha: float, keep_key: float,
-                  keep_nonkey: float, event_agg: int = 0, check_features: bool = True) -> Dict[str, object]:
+                  keep_nonkey: float, event_agg: int = 0, check_features: bool = True,
+                  key_events: Optional[np.ndarray] = None) -> Dict[str, object]:
     T, N, d = V.shape
-    want = O.compress_vision(V, t, offs, alpha, keep_key, keep_nonkey, dtype, event_agg)
+    want = O.compress_vision(V, t, offs, alpha, keep_key, keep_nonkey, dtype, event_agg, key_events_given=key_events)
     p = B.vision_params(alpha, keep_key, keep_nonkey, event_agg)
     Vd = P.to_torch(V, dtype)
+    given = None if key_events is None else torch.from_numpy(np.asarray(key_events).astype(np.uint8)).cuda()
     got = B.metok_compress_vision(Vd, torch.from_numpy(np.asarray(offs, dtype=np.int32)).cuda(),
-                                  P.to_torch(t, dtype), p)
+                                  P.to_torch(t, dtype), p, key_events=given)
     torch.cuda.synchronize()
     rep: Dict[str, object] = {}
     assert int(got["status"].item()) == 0, "device-side wait timed out"

@@ -610,3 +610,19 @@ def test_head_sharded_scores_then_selection(name, world):
     assert m == want["S_out"]
     P.check_index_set(sel["keep_idx"][:m].cpu().numpy(), want["keep_idx"],
                       lambda u: u < cfg.Nv and bool(want["near_tie"][u]), "keep_idx from summed scores")
+
+
+def test_ablation_key_events_given_by_the_caller():
+    """Randomly chosen key events (the paper's Table 4 ablation) as an argument: the per-event
+    ratios follow the caller's mask, everything else as usual."""
+    cfg = W.CONFIGS["frames32"]
+    vis = vis_of("frames32")
+    rng = np.random.default_rng(17)
+    for mask in (rng.random(cfg.k) < 0.5, np.zeros(cfg.k, dtype=bool), np.ones(cfg.k, dtype=bool)):
+        rep = R.compress_case(vis["V"], vis["t"], vis["event_offsets"], cfg.dtype, cfg.alpha, 0.3, 0.05,
+                              key_events=mask)
+        assert "event_class_flip" not in rep
+        assert rep["key_mismatches"] <= rep["key_near_ties"] and rep["assign_mismatches"] <= rep["assign_near_ties"]
+        want_n = sum(max(1, math.ceil((0.3 if mask[e] else 0.05) * (vis["event_offsets"][e + 1] - vis["event_offsets"][e])
+                                      * cfg.N - 1e-9)) for e in range(cfg.k))
+        assert rep["n_out"] == want_n

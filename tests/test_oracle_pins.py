@@ -592,3 +592,22 @@ def test_prune_schedule_planted_order_and_printed_ratios():
         assert set(non_vis) <= set(k.tolist())                 # every non-visual position survives
     assert want_alive[1].size == math.ceil(0.3025 * N0[0] - 1e-9) and want_alive[2].size == 0
     assert np.all(group[want_alive[1]] == 0)                   # no non-key token passes the second level
+
+
+def test_given_key_events_replace_the_scored_ones():
+    """The random-key-event ablation: a caller's key-event mask only changes which per-event ratio
+    applies (brute-force count of the budgets), and the scored mask given back reproduces the default."""
+    rng = np.random.default_rng(21)
+    T, N, d = 9, 16, 12
+    offs = np.array([0, 2, 5, 9], dtype=np.int32)
+    V = rng.standard_normal((T, N, d))
+    t = rng.standard_normal(d)
+    base = O.compress_vision(V, t, offs, 0.5, 0.5, 0.1, "f32")
+    same = O.compress_vision(V, t, offs, 0.5, 0.5, 0.1, "f32", key_events_given=base["event_is_key"])
+    assert np.array_equal(base["out_src"], same["out_src"]) and np.array_equal(base["assign"], same["assign"])
+    flipped = ~base["event_is_key"].astype(bool)
+    other = O.compress_vision(V, t, offs, 0.5, 0.5, 0.1, "f32", key_events_given=flipped)
+    assert np.array_equal(other["event_is_key"].astype(bool), flipped)
+    want = sum(max(1, math.ceil((0.5 if flipped[e] else 0.1) * (offs[e + 1] - offs[e]) * N - 1e-9)) for e in range(3))
+    assert other["n_out"] == want and other["n_out"] != base["n_out"]
+    assert np.array_equal(other["token_score"], base["token_score"])          # the scores themselves do not change

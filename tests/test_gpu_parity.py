@@ -626,3 +626,66 @@ def test_ablation_key_events_given_by_the_caller():
         want_n = sum(max(1, math.ceil((0.3 if mask[e] else 0.05) * (vis["event_offsets"][e + 1] - vis["event_offsets"][e])
                                       * cfg.N - 1e-9)) for e in range(cfg.k))
         assert rep["n_out"] == want_n
+
+
+def test_benchmark_launch_configuration_equals_eager_calls_at_full_size():
+    """The configuration the benchmark times -- the 128-frame workload, two videos in flight on
+    streams of their own, K/V compaction on a side stream, all captured in one CUDA graph -- leaves
+    bit for bit what the same calls leave when made eagerly one after the other (those are the calls
+    the parity tests above compare with the oracle at this size)."""
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    _vis_cache.clear()
+    torch.cuda.empty_cache()
+    cfg = W.CONFIGS["frames128"]
+    dev = torch.device("cuda", 0)
+    ref = bench.Workload(cfg, dev, host_copies=False)
+    lanes_w = [ref.twin(), ref.twin()]
+    ref.step(); ref.step()                                      # two eager passes (the K/V cache is compacted twice)
+    for w in lanes_w:
+        w.step()                                                # first pass eagerly: allocates the outputs
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in lanes_w]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        main = torch.cuda.current_stream()
+        for st in streams:
+            st.wait_stream(main)
+        for w, st in zip(lanes_w, streams):
+            with torch.cuda.stream(st):
+                w.step()
+        for st in streams:
+            main.wait_stream(st)
+    graph.replay()                                              # second pass of both videos, concurrently
+    torch.cuda.synchronize()
+
+    def same(a, b):
+        a = a.view(torch.int16) if a.dtype == torch.bfloat16 else a
+        b = b.view(torch.int16) if b.dtype == torch.bfloat16 else b
+        return torch.equal(a, b)
+
+    for w in lanes_w:
+        o, r = w.out, ref.out
+        for name in ("sims", "boundaries", "event_offsets", "frame_event", "token_score"):
+            assert same(o["seg"][name], r["seg"][name]), name
+        n = int(r["cv"]["n_out"].item())
+        assert int(o["cv"]["n_out"].item()) == n
+        for name in ("out_feats", "out_src", "out_event", "out_members"):
+            assert same(o["cv"][name][:n], r["cv"][name][:n]), name
+        assert same(o["cv"]["assign"], r["cv"]["assign"])
+        for i in range(len(ref.stages)):
+            a, b = o[f"pf{i}"], r[f"pf{i}"]
+            s = int(b["S_out"].item())
+            assert int(a["S_out"].item()) == s and int(a["status"].item()) == 0
+            assert same(a["scores"], b["scores"]) and same(a["keep_idx"][:s], b["keep_idx"][:s])
+            assert same(a["hidden_out"][:s], b["hidden_out"][:s])
+        nl = r["kv"]["new_len"].cpu().tolist()
+        assert o["kv"]["new_len"].cpu().tolist() == nl
+        for layer in (0, cfg.L // 2, cfg.L - 1):
+            m = nl[layer]
+            assert same(o["kv"]["keep_idx"][layer, :m], r["kv"]["keep_idx"][layer, :m])
+            assert same(w.ks[layer][:, :m], ref.ks[layer][:, :m]) and same(w.vs[layer][:, :m], ref.vs[layer][:, :m])
+    del graph, lanes_w, ref
+    torch.cuda.empty_cache()

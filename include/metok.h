@@ -122,7 +122,8 @@ METOK_API int metok_segment_events(const void* feats, int dtype, int T, int N, i
  *     Larger problems return METOK_ERR_TOO_LARGE and launch nothing.
  *   - The first call on each device looks up the array's device address (a
  *     driver query, no allocation).  Make that first call outside any CUDA
- *     stream capture; later calls only launch kernels.
+ *     stream capture: while `stream` is being captured such a first call returns
+ *     METOK_ERR_UNSUPPORTED and does nothing.  Later calls only launch kernels.
  *   - All calls on one device share the one array.  Nothing in it has to start at
  *     zero (each call overwrites every entry it later reads), but two calls that
  *     overlap on the GPU -- different streams, or one stream per thread -- race
@@ -358,8 +359,12 @@ METOK_API int metok_prefill_prune_schedule(const metok_prune_level* levels, int 
  *             (outputs for PAPER / TOPK, inputs for GIVEN)
  *   new_len   DEVICE int32 [L] (output; equals keep_len)
  *
- *   A GIVEN list that is not strictly ascending or reaches S_cur gives undefined
- *   cache contents (lists are not validated on the device).
+ *   GIVEN lists are checked on the device before any row is indexed through them
+ *   (0 <= keep_len[l] <= S_cur, entries strictly ascending inside [0, S_cur)).  A
+ *   layer whose list fails is left untouched, reports new_len[l] = S_cur, and the
+ *   device status word (first int32 of ws, valid after the stream is synchronised)
+ *   reads METOK_ERR_INVALID_ARG; the other layers are compacted as usual.  The
+ *   status word reads METOK_OK otherwise.
  *   Errors: INVALID_ARG (null/misaligned, sizes < 1, S_cur > S_cap, span outside
  *   [0,S_cur], ratio outside [0,1], l1 < 0, unknown policy); UNSUPPORTED
  *   (dh*sizeof(elem) % 16 != 0); WORKSPACE.

@@ -133,12 +133,6 @@ def segment_events(V: np.ndarray, k: int, sim_mode: int = SIM_FLATTEN) -> Dict[s
     sims = frame_similarity(V, sim_mode)
     out = split_events(sims, k)
     out["sims"] = sims
-    # deciding gap of the selection, for the near-tie protocol
-    if 1 < k <= sims.size:
-        srt = np.sort(sims)
-        out["gap"] = float(srt[k - 1] - srt[k - 2]) if k - 1 < sims.size else float("inf")
-    else:
-        out["gap"] = float("inf")
     return out
 
 

@@ -492,7 +492,7 @@ def metok_kv_compact(k_layers: Sequence[torch.Tensor], v_layers: Sequence[torch.
                             vis_start, n_vis, _ptr(scores), per_layer, _ptr(keep_idx), _ptr(keep_len),
                             _ptr(new_len), _ptr(ws), ws.numel(), _stream())
     _check("metok_kv_compact", st)
-    return {"keep_idx": keep_idx, "keep_len": keep_len, "new_len": new_len}
+    return {"keep_idx": keep_idx, "keep_len": keep_len, "new_len": new_len, "status": ws[:4].view(torch.int32)}
 
 
 def metok_version() -> int:

@@ -57,9 +57,33 @@ kv_paper_lists_kernel(int S_cur, int vis_start, int n_vis, int l1, int32_t* __re
     if (threadIdx.x == 0) { keep_len[layer] = n; new_len[layer] = n; }
 }
 
-__global__ void copy_len_kernel(const int32_t* __restrict__ a, int32_t* __restrict__ b, int n) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) b[i] = a[i];
+// GIVEN policy: the caller's lists are checked before anything is indexed through them.  One CTA
+// per layer reads only the list itself: 0 <= length <= S_cur, entries strictly ascending inside
+// [0, S_cur).  valid[layer] says whether the layer may be compacted; a layer with a bad list is
+// left untouched and reports S_cur rows.
+__global__ void __launch_bounds__(256)
+kv_check_lists_kernel(int S_cur, const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ keep_len,
+                      int32_t* __restrict__ new_len, int32_t* __restrict__ valid) {
+    __shared__ int s_bad;
+    const int layer = blockIdx.x;
+    const int n = keep_len[layer];
+    if (threadIdx.x == 0) s_bad = (n < 0 || n > S_cur) ? 1 : 0;
+    __syncthreads();
+    if (!s_bad) {
+        const int32_t* keep = keep_idx + (size_t)layer * S_cur;
+        int bad = 0;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int v = keep[i];
+            const int prev = i > 0 ? keep[i - 1] : -1;
+            bad |= (v <= prev) | (v >= S_cur);           // prev >= -1, so v > prev also gives v >= 0
+        }
+        if (bad) s_bad = 1;                               // same value from every writer
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        valid[layer] = s_bad ? 0 : 1;
+        new_len[layer] = s_bad ? S_cur : n;
+    }
 }
 
 // ---- fast path ------------------------------------------------------------------
@@ -100,11 +124,25 @@ __device__ __forceinline__ SlabId slab_of(int slab, int Hkv) {
 __global__ void __launch_bounds__(kKvFastThreads)
 kv_stage_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row_chunks,
                 const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ keep_len, int stage_rows,
-                int32_t* __restrict__ haz, uint4* __restrict__ stage) {
+                int32_t* __restrict__ haz, uint4* __restrict__ stage, const int32_t* __restrict__ valid,
+                int n_layers, int32_t* __restrict__ status) {
     grid_dep_wait();
     __shared__ int s_h;
     const SlabId id = slab_of(blockIdx.y, Hkv);
     const int layer = layer0 + id.ll;
+    const bool lead = blockIdx.x == 0 && id.which == 0 && id.head == 0 && threadIdx.x == 0;   // one thread per layer
+    // the call's status word: a rejected list (GIVEN policy) is an invalid argument
+    if (layer0 == 0 && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        int st = METOK_OK;
+        if (valid)
+            for (int l = 0; l < n_layers; ++l)
+                if (!valid[l]) st = METOK_ERR_INVALID_ARG;
+        *status = st;
+    }
+    if (valid && !valid[layer]) {                          // nothing is indexed through a rejected list
+        if (lead) haz[layer] = -2;
+        return;
+    }
     const int32_t* keep = keep_idx + (size_t)layer * S_cur;
     const int n = keep_len[layer];
     if (threadIdx.x < 32) {
@@ -114,7 +152,7 @@ kv_stage_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row_
     __syncthreads();
     const int h = s_h;
     const bool fast = h <= stage_rows;
-    if (blockIdx.x == 0 && id.which == 0 && id.head == 0 && threadIdx.x == 0) haz[layer] = fast ? h : -1;
+    if (lead) haz[layer] = fast ? h : -1;
     if (!fast || h == 0) return;
     const uint4* base = reinterpret_cast<const uint4*>(id.which ? ptrs.v[id.ll] : ptrs.k[id.ll]) +
                         (size_t)id.head * S_cap * row_chunks;
@@ -178,7 +216,7 @@ kv_gather_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row
     const int head = slab % Hkv;
     const int which = (slab / Hkv) & 1;
     const int ll = slab / (2 * Hkv);
-    if (haz[layer0 + ll] >= 0) return;                   // the fast path took this layer (uniform per cluster)
+    if (haz[layer0 + ll] != -1) return;                  // the fast path took this layer, or its list was rejected (uniform per cluster)
     uint4* base = reinterpret_cast<uint4*>(which ? ptrs.v[ll] : ptrs.k[ll]) + (size_t)head * S_cap * row_chunks;
     const int32_t* keep = keep_idx + (size_t)(layer0 + ll) * S_cur;
     const int n = keep_len[layer0 + ll];
@@ -230,13 +268,17 @@ kv_gather_kernel(KvPtrs ptrs, int layer0, int Hkv, int S_cap, int S_cur, int row
 }
 
 struct KvWs {
+    int32_t* status;          // device status word, first in the workspace
     int32_t* haz;
+    int32_t* valid;           // GIVEN policy: per layer, whether the caller's list passed the check
     uint4* stage;
     int stage_rows;
 };
 static KvWs carve_kv(Carver& cv, int L, int Hkv, int S_cur, int row_chunks) {
     KvWs w;
+    w.status = cv.take<int32_t>(64);
     w.haz = cv.take<int32_t>((size_t)L);
+    w.valid = cv.take<int32_t>((size_t)L);
     const size_t per_row = (size_t)L * 2 * Hkv * row_chunks * sizeof(uint4);
     size_t rows = kKvStageBudget / per_row;
     if (rows > (size_t)S_cur) rows = (size_t)S_cur;
@@ -279,9 +321,12 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
     }
     const int eb = dtype == METOK_F32 ? 4 : 2;
     if (((long long)dh * eb) % 16 != 0) return METOK_ERR_UNSUPPORTED;
-    if (!ws || ws_bytes < metok_kv_compact_workspace_bytes(dtype, L, Hkv, S_cur, dh, policy, n_vis))
+    if (!ws || ws_bytes < metok_kv_compact_workspace_bytes(dtype, L, Hkv, S_cur, dh, policy, n_vis) || !aligned16(ws))
         return METOK_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int row_chunks = (int)((long long)dh * eb / 16);
+    Carver cv(ws);
+    const KvWs w = carve_kv(cv, L, Hkv, S_cur, row_chunks);
 
     // an upper bound, known on the host, of the length of every list that drops anything
     // (-1: not known); lists that keep all rows cause no copying
@@ -305,14 +350,12 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
         kept_bound = budget + (S_cur - n_vis);
     } else {
         {
-            METOK_TIMED("copy_len_kernel", st);
-            copy_len_kernel<<<ceil_div(L, 256), 256, 0, st>>>(keep_len, new_len, L);
+            METOK_TIMED("kv_check_lists_kernel", st);
+            kv_check_lists_kernel<<<L, 256, 0, st>>>(S_cur, keep_idx, keep_len, new_len, w.valid);
         }
         METOK_LAUNCH_CHECK();
     }
-    const int row_chunks = (int)((long long)dh * eb / 16);
-    Carver cv(ws);
-    const KvWs w = carve_kv(cv, L, Hkv, S_cur, row_chunks);
+    const int32_t* valid = policy == METOK_KV_GIVEN ? w.valid : nullptr;
     for (int l0 = 0; l0 < L; l0 += kKvMaxLayersPerLaunch) {
         const int nl = (L - l0) < kKvMaxLayersPerLaunch ? (L - l0) : kKvMaxLayersPerLaunch;
         KvPtrs ptrs;
@@ -324,7 +367,8 @@ extern "C" int metok_kv_compact(void* const* k_layers, void* const* v_layers, in
         {
             METOK_TIMED("kv_stage_kernel", st);
             launch_chained(kv_stage_kernel, dim3(dim3(kKvStageSplit, slabs)), dim3(kKvFastThreads), 0, st, 
-                ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len, w.stage_rows, w.haz, w.stage);
+                ptrs, l0, Hkv, S_cap, S_cur, row_chunks, keep_idx, keep_len, w.stage_rows, w.haz, w.stage, valid, L,
+                w.status);
         }
         METOK_LAUNCH_CHECK();
         {

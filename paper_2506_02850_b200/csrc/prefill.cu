@@ -510,10 +510,10 @@ static AttnDims make_dims(int Hq, int Hkv, int Lt, int S, int dh, int vis_start,
     return dm;
 }
 
-// The tensor-core scoring path takes bf16 with head dim 64 or 128; METOK_FORCE_SIMT=1 in
+// The tensor-core scoring path takes bf16 with head dim 64 or 128; METOK_DEBUG_FORCE_SIMT=1 in
 // the environment selects the CUDA-core kernels (debugging aid).
 static bool use_mma_attn(int dtype, int dh) {
-    static const bool force_simt = [] { const char* e = getenv("METOK_FORCE_SIMT"); return e && e[0] == '1'; }();
+    static const bool force_simt = [] { const char* e = getenv("METOK_DEBUG_FORCE_SIMT"); return e && e[0] == '1'; }();
     return !force_simt && dtype == METOK_BF16 && (dh == 64 || dh == 128);
 }
 
@@ -601,11 +601,12 @@ extern "C" size_t metok_prefill_prune_workspace_bytes(int dtype, int Hq, int Hkv
     return cv.total();
 }
 
-extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const void* hidden, int dtype, int Hq,
-                                   int Hkv, int Lt, int S, int dh, int D, int vis_start, int n_vis,
-                                   const int32_t* token_group, int G, const int32_t* group_budget,
-                                   float softmax_scale, float* scores, int32_t* keep_idx, int32_t* S_out,
-                                   void* hidden_out, void* ws, size_t ws_bytes, void* stream) {
+// Every check of metok_prefill_prune that needs no device: arguments, shapes, alignment, workspace.
+static int validate_prefill_prune(const void* q_text, const void* k_all, const void* hidden, int dtype, int Hq,
+                                  int Hkv, int Lt, int S, int dh, int D, int vis_start, int n_vis,
+                                  const int32_t* token_group, int G, const int32_t* group_budget,
+                                  float softmax_scale, const float* scores, const int32_t* keep_idx,
+                                  const int32_t* S_out, const void* hidden_out, const void* ws, size_t ws_bytes) {
     if (!q_text || !k_all || !token_group || !group_budget || !scores || !keep_idx || !S_out)
         return METOK_ERR_INVALID_ARG;
     if ((hidden == nullptr) != (hidden_out == nullptr)) return METOK_ERR_INVALID_ARG;
@@ -625,6 +626,19 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
     if (hidden && ((long long)D * eb) % 16 != 0) return METOK_ERR_UNSUPPORTED;
     const size_t need = metok_prefill_prune_workspace_bytes(dtype, Hq, Hkv, Lt, S, dh, n_vis);
     if (!ws || ws_bytes < need || !aligned16(ws)) return METOK_ERR_WORKSPACE;
+    return METOK_OK;
+}
+
+extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const void* hidden, int dtype, int Hq,
+                                   int Hkv, int Lt, int S, int dh, int D, int vis_start, int n_vis,
+                                   const int32_t* token_group, int G, const int32_t* group_budget,
+                                   float softmax_scale, float* scores, int32_t* keep_idx, int32_t* S_out,
+                                   void* hidden_out, void* ws, size_t ws_bytes, void* stream) {
+    const int vrc = validate_prefill_prune(q_text, k_all, hidden, dtype, Hq, Hkv, Lt, S, dh, D, vis_start, n_vis,
+                                           token_group, G, group_budget, softmax_scale, scores, keep_idx, S_out,
+                                           hidden_out, ws, ws_bytes);
+    if (vrc != METOK_OK) return vrc;
+    const int eb = dtype == METOK_F32 ? 4 : 2;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
     AttnDims dm = make_dims(Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale);
@@ -744,8 +758,12 @@ schedule_init_kernel(const int32_t* __restrict__ token_group, int n_vis, int n0_
 __global__ void __launch_bounds__(256)
 schedule_propagate_kernel(const int32_t* __restrict__ keep_idx, int vis_start, int n_cur, int n_next,
                           const int32_t* __restrict__ group, const int32_t* __restrict__ origin,
-                          int32_t* __restrict__ group_next, int32_t* __restrict__ origin_next) {
+                          int32_t* __restrict__ group_next, int32_t* __restrict__ origin_next,
+                          const int32_t* __restrict__ level_status, int32_t* __restrict__ status) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    // a level that gave up on a wait leaves its code in its own status word, which the next level
+    // clears: the first failure is kept in the caller's
+    if (i == 0 && *level_status != METOK_OK && *status == METOK_OK) *status = *level_status;
     if (i >= n_next) return;
     int j = keep_idx[vis_start + i] - vis_start;
     j = j < 0 ? 0 : (j >= n_cur ? n_cur - 1 : j);            // only reached with a wrong N0 (status says so)
@@ -794,8 +812,22 @@ extern "C" int metok_prefill_prune_schedule(const metok_prune_level* levels, int
         if (sizes[s] < 1) return METOK_ERR_INVALID_ARG;
         if (!levels[s].token_group || !levels[s].origin) return METOK_ERR_INVALID_ARG;
     }
+    // every level's arguments, shapes and workspace are checked before the first launch
+    for (int s = 0; s < n_levels; ++s) {
+        const metok_prune_level& lv = levels[s];
+        int32_t budget[2];
+        rc = metok_retention_budgets(alpha, r, s + 1, N0, budget);
+        if (rc != METOK_OK) return rc;
+        rc = validate_prefill_prune(lv.q_text, lv.k_all, lv.hidden, dtype, Hq, Hkv, Lt, S - n_vis + sizes[s], dh, D,
+                                    vis_start, sizes[s], lv.token_group, 2, budget, softmax_scale, lv.scores,
+                                    lv.keep_idx, lv.S_out, lv.hidden_out, ws, ws_bytes);
+        if (rc != METOK_OK) return rc;
+    }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    schedule_init_kernel<<<1, 1024, 0, st>>>(levels[0].token_group, n_vis, N0[0], N0[1], levels[0].origin, status);
+    {
+        METOK_TIMED("schedule_init_kernel", st);
+        schedule_init_kernel<<<1, 1024, 0, st>>>(levels[0].token_group, n_vis, N0[0], N0[1], levels[0].origin, status);
+    }
     METOK_LAUNCH_CHECK();
     for (int s = 0; s < n_levels; ++s) {
         const metok_prune_level& lv = levels[s];
@@ -807,12 +839,17 @@ extern "C" int metok_prefill_prune_schedule(const metok_prune_level* levels, int
                                  lv.token_group, 2, budget, softmax_scale, lv.scores, lv.keep_idx, lv.S_out,
                                  lv.hidden_out, ws, ws_bytes, stream);
         if (rc != METOK_OK) return rc;
-        if (s + 1 < n_levels) {
-            const metok_prune_level& nx = levels[s + 1];
-            schedule_propagate_kernel<<<ceil_div(sizes[s + 1], 256), 256, 0, st>>>(
-                lv.keep_idx, vis_start, sizes[s], sizes[s + 1], lv.token_group, lv.origin, nx.token_group, nx.origin);
-            METOK_LAUNCH_CHECK();
+        // the level's status word (start of the workspace, cleared again by the next level) is folded
+        // into the caller's; this kernel also hands classes and origins to the next level
+        const bool more = s + 1 < n_levels;
+        const metok_prune_level& nx = levels[more ? s + 1 : s];
+        {
+            METOK_TIMED("schedule_propagate_kernel", st);
+            schedule_propagate_kernel<<<more ? ceil_div(sizes[s + 1], 256) : 1, 256, 0, st>>>(
+                lv.keep_idx, vis_start, sizes[s], more ? sizes[s + 1] : 0, lv.token_group, lv.origin, nx.token_group,
+                nx.origin, reinterpret_cast<const int32_t*>(ws), status);
         }
+        METOK_LAUNCH_CHECK();
     }
     return METOK_OK;
 }

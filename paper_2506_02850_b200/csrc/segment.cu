@@ -145,6 +145,9 @@ seg_meandot_kernel(const float* __restrict__ mean, int Tn, int d, float* __restr
     }
 }
 
+// Order-preserving key of a similarity; NaN (a non-finite frame) ranks above everything.
+__device__ __forceinline__ uint32_t sim_key(float f) { return f != f ? 0xFFFFFFFFu : float_key(f); }
+
 // Adds the slab partials in slab order, forms the cosines, picks the k-1 smallest
 // (rank by counting; ties to the lower index) and writes boundaries, CSR offsets
 // and per-frame event ids.  One CTA of 1024 threads; T <= kMaxFrames.
@@ -209,10 +212,12 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
     for (int i = tid; i < Tn; i += nthr) {
         int flag = 0;
         if (i < Tn - 1 && nb > 0) {
-            const float v = s_sim[i];
+            // integer keys give a total order even with non-finite similarities (a NaN ranks as the
+            // largest value), so exactly k-1 boundaries are flagged whatever the input holds
+            const uint32_t v = sim_key(s_sim[i]);
             int rank = 0;
             for (int j = 0; j < Tn - 1; ++j) {
-                const float w = s_sim[j];
+                const uint32_t w = sim_key(s_sim[j]);
                 rank += (w < v) || (w == v && j < i);
             }
             flag = rank < nb;
@@ -240,7 +245,7 @@ seg_finish_kernel(const float* __restrict__ part_dot, const float* __restrict__ 
     int run = before + incl - local;                       // boundaries before frame lo
     for (int i = lo; i < hi; ++i) {
         frame_event[i] = run;                              // event id = boundaries strictly before i
-        if (s_flag[i] && run < nb) {                       // (NaN similarities could over-flag)
+        if (s_flag[i] && run < nb) {
             boundaries[run] = i;
             event_offsets[run + 1] = i + 1;
             ++run;
@@ -729,11 +734,16 @@ static void* g_seg_scratch_addr[kMaxDevices] = {nullptr};    // device address o
 
 // `g_seg_scratch` in host code is only a handle; the address kernels can use has to be
 // asked for, once per device, with that device current.
-static int static_scratch_address(void** out) {
+static int static_scratch_address(void** out, cudaStream_t st) {
     int dev = -1;
     METOK_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return METOK_ERR_UNSUPPORTED;
     if (!g_seg_scratch_addr[dev]) {
+        // the look-up is not a stream operation: made while `st` is being captured it could end the
+        // caller's capture, so the first call on a device has to come before any capture
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        METOK_CUDA_TRY(cudaStreamIsCapturing(st, &cs));
+        if (cs != cudaStreamCaptureStatusNone) return METOK_ERR_UNSUPPORTED;
         void* p = nullptr;
         METOK_CUDA_TRY(cudaGetSymbolAddress(&p, g_seg_scratch));
         g_seg_scratch_addr[dev] = p;
@@ -753,7 +763,7 @@ extern "C" int metok_segment_events_static(const void* feats, int dtype, int T, 
     const size_t need = metok_segment_events_workspace_bytes(dtype, T, N, d, sim_mode);
     if (need > metok::kStaticScratchBytes) return METOK_ERR_TOO_LARGE;
     void* scratch = nullptr;
-    const int rc = metok::static_scratch_address(&scratch);
+    const int rc = metok::static_scratch_address(&scratch, reinterpret_cast<cudaStream_t>(stream));
     if (rc != METOK_OK) return rc;
     return metok_segment_events(feats, dtype, T, N, d, k, sim_mode, sims, boundaries, event_offsets, frame_event,
                                 scratch, metok::kStaticScratchBytes, stream);

@@ -1230,9 +1230,9 @@ static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, b
 }
 
 // The tensor-core merge path needs bf16 rows that TMA can address (16-byte row pitch);
-// METOK_FORCE_SIMT=1 in the environment selects the CUDA-core kernels (debugging aid).
+// METOK_DEBUG_FORCE_SIMT=1 in the environment selects the CUDA-core kernels (debugging aid).
 static bool use_mma_path(int d) {
-    static const bool force_simt = [] { const char* e = getenv("METOK_FORCE_SIMT"); return e && e[0] == '1'; }();
+    static const bool force_simt = [] { const char* e = getenv("METOK_DEBUG_FORCE_SIMT"); return e && e[0] == '1'; }();
     return !force_simt && d % 8 == 0;
 }
 

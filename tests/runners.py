@@ -27,10 +27,9 @@ def segment_case(V: np.ndarray, dtype: str, k: int, sim_mode: int = 0) -> Dict[s
     gb, wb = got["boundaries"].cpu().numpy(), want["boundaries"]
     if not np.array_equal(gb, wb):
         # only excusable when the (k-1)-th and k-th smallest similarities nearly tie
-        scale = max(float(np.max(np.abs(want["sims"]))), 1e-300)
         srt = np.sort(want["sims"])
         tau = srt[k - 2]
-        near = np.abs(want["sims"] - tau) < O.NEAR_TIE * scale
+        near = O.near_threshold(want["sims"], tau)
         rep["mismatches"] = P.check_index_set(gb, wb, lambda i: bool(near[i]), "boundaries")
         rep["near_ties"] = int(near.sum())
     else:
@@ -75,7 +74,7 @@ def compress_case(V: np.ndarray, t: np.ndarray, offs: np.ndarray, dtype: str, al
     if not np.array_equal(gk, wk):
         es = want["event_score"]
         tau = np.sort(es)[::-1][int(wk.sum()) - 1]
-        near = np.abs(es - tau) < O.NEAR_TIE * max(float(np.max(np.abs(es))), 1e-300)
+        near = O.near_threshold(es, tau)
         P.check_index_set(np.nonzero(gk)[0], np.nonzero(wk)[0], lambda i: bool(near[i]), "event_is_key")
         rep["event_class_flip"] = True
         return rep                                            # budgets differ downstream: nothing else is comparable
@@ -164,7 +163,7 @@ def pool_case(V: np.ndarray, t: np.ndarray, offs: np.ndarray, dtype: str, alpha:
             seg = fs[int(offs[e]):int(offs[e + 1])]
             nk = int(want["frame_is_key"][int(offs[e]):int(offs[e + 1])].sum())
             tau = np.sort(seg)[::-1][nk - 1]
-            assert abs(fs[f] - tau) < O.NEAR_TIE * max(float(np.max(np.abs(seg))), 1e-300), f"frame {f} flipped outside the near-tie band"
+            assert bool(O.near_threshold(seg, tau)[f - int(offs[e])]), f"frame {f} flipped outside the near-tie band"
         return rep
     assert n_out == want["n_out"]
     assert np.array_equal(frame_of, want["out_frame"])
@@ -248,11 +247,30 @@ def kv_case(cfg: W.Config, policy: int, layers: Optional[int] = None, per_layer_
     got = B.metok_kv_compact(ks, vs, S_cur, policy, 0, n_vis, l1=l1, **kwargs)
     torch.cuda.synchronize()
     new_len = got["new_len"].cpu().numpy()
+    assert int(got["status"].item()) == 0
     assert np.array_equal(new_len, [len(w) for w in want])
     assert np.array_equal(got["keep_len"].cpu().numpy(), new_len)
     keep_idx = got["keep_idx"].cpu().numpy()
     for layer in range(L):
         assert np.array_equal(keep_idx[layer, : new_len[layer]], want[layer]), layer   # scores are tie-free
+    # every (layer, K|V, head) slab bit for bit: the payload is regenerated on the device from its hash
+    # and gathered with the ORACLE's list
+    checked = 0
+    for layer in range(L):
+        n = int(new_len[layer])
+        if n == 0:
+            continue
+        idx = torch.from_numpy(np.asarray(want[layer], dtype=np.int64)).to(dev)
+        for which in (0, 1):
+            for head in range(cfg.Hkv):
+                src = W.payload_torch(W.kv_salt(cfg, layer, which, head), S_cur, cfg.dh, cfg.dtype, dev)
+                t = (vs if which else ks)[layer][head, :n]
+                exp = src[idx]
+                if cfg.dtype == "bf16":
+                    t, exp = t.view(torch.int16), exp.view(torch.int16)
+                assert torch.equal(t, exp), (layer, which, head)
+                checked += 1
+    # a few slabs also against rows regenerated on the host (the numpy form of the hash)
     rng = np.random.default_rng(99)
     slabs = [(int(rng.integers(0, L)), int(rng.integers(0, 2)), int(rng.integers(0, cfg.Hkv)))
              for _ in range(sample_slabs)]
@@ -267,4 +285,4 @@ def kv_case(cfg: W.Config, policy: int, layers: Optional[int] = None, per_layer_
             assert np.array_equal(P.bits(t), expect), (layer, which, head)
         else:
             assert np.array_equal(t.cpu().numpy(), expect), (layer, which, head)
-    return {"kept_rows": int(new_len.sum()), "slabs_checked": len(slabs)}
+    return {"kept_rows": int(new_len.sum()), "slabs_checked": checked, "slabs_checked_on_host": len(slabs)}

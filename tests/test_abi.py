@@ -21,6 +21,26 @@ def lib():
     return B.lib()
 
 
+_real = {}
+
+
+def device_pointers():
+    """(pointer, pointer + 4, a second pointer) for arguments of calls that must be rejected before any
+    launch.  Without a CUDA device they are made-up addresses (nothing can be launched anyway); with
+    one they point into a real zero-filled 64 MiB allocation, so that a validation regression would
+    launch on valid memory instead of a wild pointer."""
+    try:
+        import torch
+        if torch.cuda.is_available():
+            if "buf" not in _real:
+                _real["buf"] = torch.zeros(1 << 26, dtype=torch.uint8, device="cuda")
+            base = _real["buf"].data_ptr()
+            return base, base + 4, base + (1 << 20)
+    except Exception:
+        pass
+    return 0x10000, 0x10004, 0x20000
+
+
 def declared_symbols():
     text = open(HEADER).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
@@ -84,9 +104,10 @@ def test_compress_bound_and_workspace(lib):
 
 def test_validation_rejects_before_any_launch(lib):
     """Bad arguments return INVALID_ARG / UNSUPPORTED / WORKSPACE without touching the GPU
-    (the pointers below are fake; a launch would fault, a validated rejection cannot)."""
-    fake = ctypes.c_void_p(0x10000)
-    odd = ctypes.c_void_p(0x10004)
+    (see device_pointers for what the non-null pointers are)."""
+    p0, p_odd, p1 = device_pointers()
+    fake = ctypes.c_void_p(p0)
+    odd = ctypes.c_void_p(p_odd)
     null = ctypes.c_void_p(0)
     seg = lib.metok_segment_events
     ok_args = [fake, B.BF16, 8, 16, 64, 2, 0, fake, fake, fake, fake, fake, 1 << 20, null]
@@ -138,7 +159,7 @@ def test_validation_rejects_before_any_launch(lib):
     assert pcall(14, neg) == -1
 
     kv = lib.metok_kv_compact
-    ptrs = (ctypes.c_void_p * 2)(0x10000, 0x20000)
+    ptrs = (ctypes.c_void_p * 2)(p0, p1)
     kbase = [ptrs, ptrs, B.BF16, 2, 4, 160, 160, 128, B.KV_TOPK, 0, 0.1, 0, 144, fake, 0, fake, fake, fake,
              fake, 1 << 20, null]
     def kcall(idx, val):
@@ -151,7 +172,7 @@ def test_validation_rejects_before_any_launch(lib):
     assert kcall(13, null) == -1                              # TOPK needs scores
     assert kcall(7, 100) == -2                                # 200-byte rows
     assert kcall(18, null) == -3
-    badptrs = (ctypes.c_void_p * 2)(0x10000, 0)
+    badptrs = (ctypes.c_void_p * 2)(p0, 0)
     assert kcall(0, badptrs) == -1
 
 
@@ -171,10 +192,11 @@ def test_prune_schedule_sizes_and_validation(lib):
         assert B.metok_prune_schedule_sizes(3, alpha, r, N0) == want
     with pytest.raises(B.MetokError):
         B.metok_prune_schedule_sizes(4, 0.5, 0.5, (1, 1))
-    fake, null = ctypes.c_void_p(0x10000), ctypes.c_void_p(0)
+    p0 = device_pointers()[0]
+    fake, null = ctypes.c_void_p(p0), ctypes.c_void_p(0)
     lv = (B.PruneLevel * 3)()
     for s in range(3):
-        lv[s] = B.PruneLevel(*([0x10000] * 9))
+        lv[s] = B.PruneLevel(*([p0] * 9))
     n0 = (ctypes.c_int32 * 2)(200, 100)
     fn = lib.metok_prefill_prune_schedule
     args = [lv, 3, B.BF16, 28, 4, 16, 316, 128, 3584, 0, 300, 0.5, 0.55, n0, 0.088, fake, fake, 1 << 26, null]
@@ -190,3 +212,36 @@ def test_prune_schedule_sizes_and_validation(lib):
     assert call(13, n0_empty) == -1
     assert lib.metok_prefill_prune_schedule_workspace_bytes(3, B.BF16, 28, 4, 16, 316, 128, 300, 0.5, 0.55, n0) > 0
     assert lib.metok_prefill_prune_schedule_workspace_bytes(3, B.BF16, 28, 4, 16, 316, 128, 299, 0.5, 0.55, n0) == 0
+
+
+def test_prune_schedule_checks_every_level_before_the_first_launch(lib):
+    """A bad argument at a later level (null q_text at level 2, a misaligned K at level 3, a workspace
+    too small for the largest level) is rejected with nothing launched: the library's own launch
+    counter stays at zero."""
+    p0, p_odd, _ = device_pointers()
+    null = ctypes.c_void_p(0)
+    n0 = (ctypes.c_int32 * 2)(200, 100)
+    fn = lib.metok_prefill_prune_schedule
+    names = [f[0] for f in B.PruneLevel._fields_]
+
+    def levels(**bad):
+        lv = (B.PruneLevel * 3)()
+        for s in range(3):
+            lv[s] = B.PruneLevel(*([p0] * 9))
+        for key, (s, val) in bad.items():
+            assert key in names
+            setattr(lv[s], key, val)
+        return lv
+
+    def call(lv, ws_bytes=1 << 26):
+        assert lib.metok_profile_begin() == 0
+        rc = fn(lv, 3, B.BF16, 28, 4, 16, 316, 128, 3584, 0, 300, 0.5, 0.55, n0, 0.088, ctypes.c_void_p(p0),
+                ctypes.c_void_p(p0), ws_bytes, null)
+        launched = lib.metok_profile_end(None, 0)
+        return rc, launched
+
+    assert call(levels(q_text=(1, None))) == (-1, 0)
+    assert call(levels(k_all=(2, p_odd))) == (-1, 0)
+    assert call(levels(keep_idx=(1, None))) == (-1, 0)
+    assert call(levels(hidden_out=(2, None))) == (-1, 0)      # hidden without hidden_out
+    assert call(levels(), ws_bytes=4096) == (-3, 0)

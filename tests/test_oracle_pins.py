@@ -611,3 +611,91 @@ def test_given_key_events_replace_the_scored_ones():
     want = sum(max(1, math.ceil((0.5 if flipped[e] else 0.1) * (offs[e + 1] - offs[e]) * N - 1e-9)) for e in range(3))
     assert other["n_out"] == want and other["n_out"] != base["n_out"]
     assert np.array_equal(other["token_score"], base["token_score"])          # the scores themselves do not change
+
+
+def test_near_threshold_band_members_known_by_construction():
+    """The band that excuses a top-k mismatch is |s - tau| < 1e-3 * max(|tau|, 1e-3 * max|s|).
+    Hand-built vectors whose band members are known: a band ten times too wide, a band taken
+    relative to the largest score instead of the threshold, or a missing floor each fail."""
+    # threshold 1.0: 1 +- 5e-4 inside, 1 +- 2e-3 outside, and the threshold itself inside
+    s = np.array([50.0, 1.002, 1.0005, 1.0, 0.9995, 0.998, -1.0, 0.0])
+    assert O.near_threshold(s, 1.0).tolist() == [False, False, True, True, True, False, False, False]
+    # relative to |tau|, not to max|s| = 50 (that band would be 5e-2 wide and take in 1.002 and 0.998)
+    assert O.near_threshold(s, 1.0).sum() == 3
+    # a negative threshold uses its magnitude
+    assert O.near_threshold(np.array([-2.0, -2.001, -2.003, 2.0]), -2.0).tolist() == [True, True, False, False]
+    # threshold near zero: the band is floored at 1e-3 * 1e-3 * max|s| = 4e-6 here
+    s0 = np.array([4.0, 1e-7, 3e-6, -3e-6, 5e-6, -5e-6, 0.0])
+    assert O.near_threshold(s0, 0.0).tolist() == [False, True, True, True, False, False, True]
+    assert O.near_threshold(s0, 1e-7).tolist() == [False, True, True, True, False, False, True]
+    # just inside and just outside one band width (1.024 at a threshold of 1024)
+    assert O.near_threshold(np.array([1024.0, 1025.0, 1025.05, 1022.95]), 1024.0).tolist() == [True, True, False, False]
+    # width scales with the threshold: the same absolute gap is inside at 100, outside at 1
+    assert O.near_threshold(np.array([100.0, 100.05]), 100.0).tolist() == [True, True]
+    assert O.near_threshold(np.array([1.0, 1.05]), 1.0).tolist() == [True, False]
+    assert O.NEAR_TIE == 1e-3
+
+
+def test_key_token_and_class_topk_report_the_band_of_their_own_threshold():
+    """key_token_topk and weighted_topk must hand near_threshold the LAST KEPT score of the segment
+    or class (not the first dropped one, not another segment's)."""
+    # one event of 8 tokens, budget 4: kept {10, 9, 8, 7.001}; 7.0 is dropped, 0.07 % below the cut
+    ts = np.array([10.0, 9.0, 8.0, 7.001, 7.0, 6.9, 1.0, 0.5])
+    out = O.key_token_topk(ts, 8, np.array([0, 1]), np.array([1], dtype=np.uint8), 0.5, 0.5)
+    assert out["key_idx"].tolist() == [0, 1, 2, 3]
+    assert out["near_tie"].tolist() == [False, False, False, True, True, False, False, False]
+    # two classes with their own cuts: class 0 cut at 5.0 (4.998 near, 4.9 not), class 1 cut at 0.5
+    sc = np.array([9.0, 5.0, 4.998, 4.9, 0.9, 0.5, 0.5004, 0.2])
+    grp = np.array([0, 0, 0, 0, 1, 1, 1, 1])
+    w = O.weighted_topk(sc, grp, [2, 3], 8, 0)
+    assert w["keep_idx"].tolist() == [0, 1, 4, 5, 6]
+    assert w["near_tie"].tolist() == [False, True, True, False, False, True, True, False]
+
+
+def test_merge_margin_closed_form():
+    """margin = (best - second best cosine) / |best| over the keys of the token's own event.
+    Three keys at known angles from a non-key token: cosines cos(10 deg), cos(20 deg), cos(60 deg) by
+    construction, so the margin is known in closed form; a margin taken from the wrong two
+    columns (best vs worst, second vs third) or divided by the second gives another number."""
+    def unit(deg):
+        return np.array([math.cos(math.radians(deg)), math.sin(math.radians(deg)), 0.0, 0.0])
+    a = unit(0.0) * 3.0                                     # the non-key token (norm must not matter)
+    k1, k2, k3 = unit(60.0) * 0.5, unit(10.0) * 2.0, unit(-20.0) * 7.0
+    # event 0: tokens a, k1, k2, k3; event 1: a copy of a whose only key is far away (one key: margin inf)
+    V = np.stack([a, k1, k2, k3, a, unit(90.0)]).reshape(6, 1, 4)
+    offs = np.array([0, 4, 6])
+    is_key = np.array([0, 1, 1, 1, 0, 1], dtype=np.uint8)
+    out = O.merge_assign(V, 1, offs, is_key, "f32")
+    c10, c20, c60 = (math.cos(math.radians(x)) for x in (10.0, 20.0, 60.0))
+    assert out["assign"][0] == 1                            # slot of k2 (the 10-degree key)
+    assert math.isclose(out["margin"][0], (c10 - c20) / c10, rel_tol=1e-12)
+    assert abs(out["margin"][0] - (c10 - c60) / c10) > 0.3   # not best-vs-worst
+    assert math.isinf(out["margin"][4]) and out["assign"][4] == 3
+    assert all(math.isinf(out["margin"][j]) for j in (1, 2, 3, 5))     # key tokens decide nothing
+    # near-tie by construction: second key 1e-4 (relative) below the best -> inside the 1e-3 band;
+    # 1e-2 below -> outside
+    for rel, inside in ((1e-4, True), (1e-2, False)):
+        ang = math.degrees(math.acos(c10 * (1.0 - rel)))
+        V2 = np.stack([a, unit(10.0), unit(-ang)]).reshape(3, 1, 4)
+        o2 = O.merge_assign(V2, 1, np.array([0, 3]), np.array([0, 1, 1], dtype=np.uint8), "f32")
+        assert math.isclose(o2["margin"][0], rel, rel_tol=1e-6)
+        assert (o2["margin"][0] < O.NEAR_TIE) == inside
+    # negative best cosine: the margin divides by its magnitude and stays positive
+    V3 = np.stack([a, unit(120.0), unit(150.0)]).reshape(3, 1, 4)
+    o3 = O.merge_assign(V3, 1, np.array([0, 3]), np.array([0, 1, 1], dtype=np.uint8), "f32")
+    c120, c150 = math.cos(math.radians(120.0)), math.cos(math.radians(150.0))
+    assert o3["assign"][0] == 0 and math.isclose(o3["margin"][0], (c120 - c150) / abs(c120), rel_tol=1e-12)
+
+
+def test_split_events_non_finite_similarity_ranks_last():
+    """A frame with a non-finite feature gives NaN similarities on both sides; they count as the
+    LARGEST values (never a boundary while finite candidates remain), ties to the lower index."""
+    sims = np.array([0.9, 0.1, np.nan, np.nan, 0.5, 0.2, 0.95])
+    assert O.split_events(sims, 3)["boundaries"].tolist() == [1, 5]
+    assert O.split_events(sims, 6)["boundaries"].tolist() == [0, 1, 4, 5, 6]
+    assert O.split_events(sims, 7)["boundaries"].tolist() == [0, 1, 2, 4, 5, 6]     # then the lower NaN
+    V = np.random.default_rng(3).standard_normal((6, 2, 4))
+    V[3, 1, 2] = np.inf
+    out = O.segment_events(V, 3)
+    assert np.isnan(out["sims"][2]) and np.isnan(out["sims"][3]) and np.isfinite(out["sims"][[0, 1, 4]]).all()
+    assert not set(out["boundaries"].tolist()) & {2, 3}

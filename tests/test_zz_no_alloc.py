@@ -55,3 +55,31 @@ def test_static_scratch_rejects_problems_beyond_its_capacity():
                                              ints.data_ptr(), ints.data_ptr(), ints.data_ptr(), None)
     assert st == -6
     assert b"capacity" in B.lib().metok_status_string(st)
+
+
+def test_static_entry_point_allocates_nothing():
+    """The raw C call with outputs allocated beforehand: neither the driver's free-memory figure nor
+    torch's allocator moves across it (the device address of the built-in array is already known
+    after a first call)."""
+    rng = np.random.default_rng(6)
+    T, N, d, k = 24, 36, 128, 5
+    V = torch.from_numpy(rng.standard_normal((T, N, d)).astype(np.float32)).cuda()
+    want = B.metok_segment_events(V, k)
+    B.metok_segment_events_static(V, k)                        # first call on this device, if none came before
+    sims = torch.empty(T - 1, dtype=torch.float32, device="cuda")
+    bnd = torch.empty(k - 1, dtype=torch.int32, device="cuda")
+    offs = torch.empty(k + 1, dtype=torch.int32, device="cuda")
+    fe = torch.empty(T, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    st = B.lib().metok_segment_events_static(V.data_ptr(), B.F32, T, N, d, k, B.SIM_FLATTEN, sims.data_ptr(),
+                                             bnd.data_ptr(), offs.data_ptr(), fe.data_ptr(),
+                                             torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert st == 0
+    assert free1 == free0
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
+    assert torch.equal(sims, want["sims"]) and torch.equal(bnd, want["boundaries"])
+    assert torch.equal(offs, want["event_offsets"]) and torch.equal(fe, want["frame_event"])

@@ -605,8 +605,8 @@ merge_assign_simt_kernel(const T* __restrict__ feats, int d, int N, const int32_
 // persistent CTA takes every gridDim-th unit.
 //   warp 0   : TMA producer -- per 64-wide K step one 256x64 (or, for an event's last
 //              rows, 128x64) tile of V (rows are contiguous in V) and the chunk's key
-//              rows from the compact key buffer (64-row boxes), 3-stage ring that runs
-//              on across units;
+//              rows from the compact key buffer (one or two boxes), 3-stage ring that
+//              runs on across units;
 //   warp 1   : allocates TMEM, issues tcgen05.mma (M=128, N=16..256, K=16), two per K
 //              slice (one per row half), and commits to the ring / accumulator barriers;
 //   warps 2-9: epilogue, four warps per row half -- read the accumulator with
@@ -645,7 +645,8 @@ __device__ __forceinline__ MergeUnit merge_unit(int u, const int32_t* __restrict
 
 __global__ void __launch_bounds__(kMmaThreads, 1)
 merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_half,
-                        const __grid_constant__ CUtensorMap tmB, int d, int N,
+                        const __grid_constant__ CUtensorMap tmB64, const __grid_constant__ CUtensorMap tmB128,
+                        const __grid_constant__ CUtensorMap tmB256, int d, int N,
                         const int32_t* __restrict__ ev_lo, int k, const int32_t* __restrict__ ev_out_off,
                         const int32_t* __restrict__ ev_unit_off, const int32_t* __restrict__ out_src,
                         const float* __restrict__ inv_norm, const uint8_t* __restrict__ is_key,
@@ -664,8 +665,6 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-    auto a_addr = [&](int s) { return smem_base + (uint32_t)s * (kMmaABytes + kMmaBBytes); };
-    auto b_addr = [&](int s) { return a_addr(s) + kMmaABytes; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
@@ -685,60 +684,80 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
 
+    // The two single-thread loops below run once per K step with nothing to hide their latency:
+    // stage and phase are counted (no division), addresses and descriptor words only move by adds.
     if (warp == 0) {
         if (lane == 0) {
             prefetch_tmap(&tmA);
             prefetch_tmap(&tmA_half);
-            prefetch_tmap(&tmB);
-            int it = 0;
+            prefetch_tmap(&tmB64);
+            prefetch_tmap(&tmB128);
+            prefetch_tmap(&tmB256);
+            int s = 0, issued = 0;
+            uint32_t ph = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
                 const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
-                const int nbox = (mu.nvalid + 63) >> 6;
+                // a copy costs the copy engine a fixed time per box on top of the time per row, so the
+                // chunk's key rows come in as few boxes as cover them: 64, 128, 128 + 64 or 256 rows
+                const int nbox = (mu.nvalid + 63) >> 6;                // 64-row boxes that would cover the keys: 1..4
+                const CUtensorMap* b0 = nbox == 1 ? &tmB64 : nbox == 4 ? &tmB256 : &tmB128;
+                const bool b1 = nbox == 3;                             // a 64-row box after the 128-row one
                 const bool two = mu.row_end - mu.row0 > 128;           // both row halves hold rows of the event
-                for (int ks = 0; ks < ksteps; ++ks, ++it) {
-                    const int s = it % kMmaStages;
-                    const uint32_t ph = (uint32_t)(it / kMmaStages) & 1u;
-                    if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t fb = smem_u32(&full_bar[s]);
-                    mbar_arrive_expect_tx(fb, (two ? kMmaABytes : kMmaABytes / 2) + (uint32_t)nbox * kMmaBoxBytes);
-                    tma_load_2d(a_addr(s), two ? &tmA : &tmA_half, ks * kMmaBK, mu.row0, fb);
-                    for (int j = 0; j < nbox; ++j)
-                        tma_load_2d(b_addr(s) + (uint32_t)j * kMmaBoxBytes, &tmB, ks * kMmaBK, mu.col0 + j * 64, fb);
+                const CUtensorMap* a0 = two ? &tmA : &tmA_half;
+                const uint32_t tx = (two ? kMmaABytes : kMmaABytes / 2) + (uint32_t)nbox * kMmaBoxBytes;
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t fb = smem_u32(&full_bar[0]) + 8u * s;
+                    const uint32_t a_dst = smem_base + (uint32_t)s * (kMmaABytes + kMmaBBytes);
+                    mbar_arrive_expect_tx(fb, tx);
+                    tma_load_2d(a_dst, a0, ks * kMmaBK, mu.row0, fb);
+                    tma_load_2d(a_dst + kMmaABytes, b0, ks * kMmaBK, mu.col0, fb);
+                    if (b1) tma_load_2d(a_dst + kMmaABytes + 2u * kMmaBoxBytes, &tmB64, ks * kMmaBK, mu.col0 + 128, fb);
+                    ++issued;
+                    if (++s == kMmaStages) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {
                 // let the copies already issued land before the CTA's shared memory goes away
-                for (int back = 1; back <= kMmaStages && back <= it; ++back) {
-                    const int j = it - back;
+                for (int back = 1; back <= kMmaStages && back <= issued; ++back) {
+                    const int j = issued - back;
                     mbar_wait(smem_u32(&full_bar[j % kMmaStages]), (uint32_t)(j / kMmaStages) & 1u, abort_flag);
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            int it = 0, n = 0;
+            int s = 0, n = 0;
+            uint32_t ph = 0;
             bool ok = true;
+            const uint32_t a_lo0 = desc_k128_lo(smem_base);
+            constexpr uint32_t kStageWords = (kMmaABytes + kMmaBBytes) >> 4, kBWords = kMmaABytes >> 4,
+                               kHalfWords = (kMmaABytes / 2) >> 4;
             for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++n) {
                 const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
                 const bool two = mu.row_end - mu.row0 > 128;
                 if (!mbar_wait(smem_u32(&tempty_bar), ((uint32_t)n & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t idesc = make_idesc_bf16(128, (mu.nvalid + 15) & ~15);
-                for (int ks = 0; ks < ksteps; ++ks, ++it) {
-                    const int s = it % kMmaStages;
-                    const uint32_t ph = (uint32_t)(it / kMmaStages) & 1u;
-                    if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag)) { ok = false; break; }
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
+                    const uint32_t a_lo = a_lo0 + (uint32_t)s * kStageWords, b_lo = a_lo + kBWords;
+                    const uint32_t acc0 = ks != 0 ? 1u : 0u;
+                    if (two) {                                       // rows 128..255 of the tile: 16 KiB further on
 #pragma unroll
-                    for (int kk = 0; kk < kMmaBK / 16; ++kk) {
-                        const uint64_t bd = make_desc_k128(b_addr(s) + kk * 32);
-                        umma_bf16(tmem_base, make_desc_k128(a_addr(s) + kk * 32), bd, idesc, (ks | kk) != 0 ? 1u : 0u);
-                        if (two)                                     // rows 128..255 of the tile: 16 KiB further on
-                            umma_bf16(tmem_base + kMmaBN, make_desc_k128(a_addr(s) + kMmaABytes / 2 + kk * 32), bd, idesc,
-                                      (ks | kk) != 0 ? 1u : 0u);
+                        for (int kk = 0; kk < kMmaBK / 16; ++kk) {
+                            umma_bf16_words(tmem_base, a_lo + 2 * kk, b_lo + 2 * kk, idesc, kk ? 1u : acc0);
+                            umma_bf16_words(tmem_base + kMmaBN, a_lo + kHalfWords + 2 * kk, b_lo + 2 * kk, idesc, kk ? 1u : acc0);
+                        }
+                    } else {
+#pragma unroll
+                        for (int kk = 0; kk < kMmaBK / 16; ++kk)
+                            umma_bf16_words(tmem_base, a_lo + 2 * kk, b_lo + 2 * kk, idesc, kk ? 1u : acc0);
                     }
-                    umma_commit(smem_u32(&empty_bar[s]));          // frees the stage when these MMAs retire
+                    umma_commit(smem_u32(&empty_bar[0]) + 8u * s);   // frees the stage when these MMAs retire
+                    if (++s == kMmaStages) { s = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit(smem_u32(&tfull_bar));         // both accumulators of this unit complete
             }
@@ -1346,14 +1365,19 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         if (r2 != METOK_OK) return r2;
         r2 = make_tmap_bf16_2d(&tmA_half, feats, (uint64_t)Nv, (uint64_t)d, kMmaBM / 2);
         if (r2 != METOK_OK) return r2;
+        CUtensorMap tmB128, tmB256;
         r2 = make_tmap_bf16_2d(&tmB, w.key_rows, (uint64_t)cap + 64, (uint64_t)d, 64);
+        if (r2 != METOK_OK) return r2;
+        r2 = make_tmap_bf16_2d(&tmB128, w.key_rows, (uint64_t)cap + 64, (uint64_t)d, 128);
+        if (r2 != METOK_OK) return r2;
+        r2 = make_tmap_bf16_2d(&tmB256, w.key_rows, (uint64_t)cap + 64, (uint64_t)d, 256);
         if (r2 != METOK_OK) return r2;
         METOK_CUDA_TRY(cudaFuncSetAttribute(merge_assign_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)kMmaSmemBytes));
         {
             METOK_TIMED("merge_assign_mma_kernel", st);
             launch_chained(merge_assign_mma_kernel, dim3(kNumSMs), dim3(kMmaThreads), kMmaSmemBytes, st, 
-                tmA, tmA_half, tmB, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, inv_norm, w.is_key, w.best64,
+                tmA, tmA_half, tmB, tmB128, tmB256, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, inv_norm, w.is_key, w.best64,
                 w.status);
         }
         METOK_LAUNCH_CHECK();

@@ -604,9 +604,13 @@ merge_assign_simt_kernel(const T* __restrict__ feats, int d, int N, const int32_
 // fewer bytes per flop than a 128 x 256 one.  The units of all events form one list; a
 // persistent CTA takes every gridDim-th unit.
 //   warp 0   : TMA producer -- per 64-wide K step one 256x64 (or, for an event's last
-//              rows, 128x64) tile of V (rows are contiguous in V) and the chunk's key
-//              rows from the compact key buffer (one or two boxes), 3-stage ring that
+//              rows, 128x64) tile of V (rows are contiguous in V), 3-stage ring that
 //              runs on across units;
+//   warps 10-13: key producers -- the chunk's key rows are rows of V scattered over the
+//              event, so their 128-byte slices come by 16-byte asynchronous copies
+//              straight from V into the ring, written in the 128-byte swizzle the MMA
+//              expects (eight threads per row, sixteen rows per thread and K step); the
+//              copies of a stage report to the stage's barrier when they have landed;
 //   warp 1   : allocates TMEM, issues tcgen05.mma (M=128, N=16..256, K=16), two per K
 //              slice (one per row half), and commits to the ring / accumulator barriers;
 //   warps 2-9: epilogue, four warps per row half -- read the accumulator with
@@ -618,7 +622,8 @@ merge_assign_simt_kernel(const T* __restrict__ feats, int d, int N, const int32_
 // Every wait is bounded; on a timeout the CTA unwinds and writes METOK_ERR_TIMEOUT.
 // --------------------------------------------------------------------------- //
 constexpr int kMmaBM = 256, kMmaBK = 64, kMmaBN = 256, kMmaStages = 3;
-constexpr int kMmaThreads = 320;
+constexpr int kMmaThreads = 448;
+constexpr int kMmaKeyThreads = 128;                        // warps 10-13
 constexpr uint32_t kMmaABytes = kMmaBM * kMmaBK * 2;       // 32 KiB
 constexpr uint32_t kMmaBBytes = kMmaBN * kMmaBK * 2;       // 32 KiB
 constexpr uint32_t kMmaBoxBytes = 64 * kMmaBK * 2;         // one 64-row key box
@@ -645,8 +650,7 @@ __device__ __forceinline__ MergeUnit merge_unit(int u, const int32_t* __restrict
 
 __global__ void __launch_bounds__(kMmaThreads, 1)
 merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_half,
-                        const __grid_constant__ CUtensorMap tmB64, const __grid_constant__ CUtensorMap tmB128,
-                        const __grid_constant__ CUtensorMap tmB256, int d, int N,
+                        const __nv_bfloat16* __restrict__ feats, int d, int N,
                         const int32_t* __restrict__ ev_lo, int k, const int32_t* __restrict__ ev_out_off,
                         const int32_t* __restrict__ ev_unit_off, const int32_t* __restrict__ out_src,
                         const float* __restrict__ inv_norm, const uint8_t* __restrict__ is_key,
@@ -667,7 +671,9 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMmaStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        // a stage is full when the tile of V has landed (one arrival with its byte count) and every
+        // key-producer thread's copies have (one arrival each)
+        for (int s = 0; s < kMmaStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1 + kMmaKeyThreads); mbar_init(smem_u32(&empty_bar[s]), 1); }
         mbar_init(smem_u32(&tfull_bar), 1);
         mbar_init(smem_u32(&tempty_bar), 8);
         mbar_init(smem_u32(&drain_bar), 1);
@@ -690,30 +696,19 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         if (lane == 0) {
             prefetch_tmap(&tmA);
             prefetch_tmap(&tmA_half);
-            prefetch_tmap(&tmB64);
-            prefetch_tmap(&tmB128);
-            prefetch_tmap(&tmB256);
             int s = 0, issued = 0;
             uint32_t ph = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
                 const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
-                // a copy costs the copy engine a fixed time per box on top of the time per row, so the
-                // chunk's key rows come in as few boxes as cover them: 64, 128, 128 + 64 or 256 rows
-                const int nbox = (mu.nvalid + 63) >> 6;                // 64-row boxes that would cover the keys: 1..4
-                const CUtensorMap* b0 = nbox == 1 ? &tmB64 : nbox == 4 ? &tmB256 : &tmB128;
-                const bool b1 = nbox == 3;                             // a 64-row box after the 128-row one
                 const bool two = mu.row_end - mu.row0 > 128;           // both row halves hold rows of the event
                 const CUtensorMap* a0 = two ? &tmA : &tmA_half;
-                const uint32_t tx = (two ? kMmaABytes : kMmaABytes / 2) + (uint32_t)nbox * kMmaBoxBytes;
+                const uint32_t tx = two ? kMmaABytes : kMmaABytes / 2;
                 for (int ks = 0; ks < ksteps; ++ks) {
                     if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t fb = smem_u32(&full_bar[0]) + 8u * s;
-                    const uint32_t a_dst = smem_base + (uint32_t)s * (kMmaABytes + kMmaBBytes);
                     mbar_arrive_expect_tx(fb, tx);
-                    tma_load_2d(a_dst, a0, ks * kMmaBK, mu.row0, fb);
-                    tma_load_2d(a_dst + kMmaABytes, b0, ks * kMmaBK, mu.col0, fb);
-                    if (b1) tma_load_2d(a_dst + kMmaABytes + 2u * kMmaBoxBytes, &tmB64, ks * kMmaBK, mu.col0 + 128, fb);
+                    tma_load_2d(smem_base + (uint32_t)s * (kMmaABytes + kMmaBBytes), a0, ks * kMmaBK, mu.row0, fb);
                     ++issued;
                     if (++s == kMmaStages) { s = 0; ph ^= 1u; }
                 }
@@ -742,6 +737,7 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 const uint32_t idesc = make_idesc_bf16(128, (mu.nvalid + 15) & ~15);
                 for (int ks = 0; ks < ksteps; ++ks) {
                     if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, ph, abort_flag)) { ok = false; break; }
+                    fence_proxy_async();                             // the key rows were written by ordinary (non-bulk) copies
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + (uint32_t)s * kStageWords, b_lo = a_lo + kBWords;
                     const uint32_t acc0 = ks != 0 ? 1u : 0u;
@@ -766,6 +762,44 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 mbar_wait(smem_u32(&drain_bar), 0u, abort_flag);
             }
         }
+    } else if (warp >= 10) {
+        // Key producers.  Thread pt copies 16-byte chunk c = pt % 8 of the rows r = pt / 8 + 16 i,
+        // i = 0..15, of the chunk's keys: eight consecutive threads read the 128 contiguous bytes of
+        // one row's K slice.  In the swizzled tile row r lies at r * 128 bytes and its chunk c at
+        // position c ^ (r % 8).  Rows past the chunk's keys up to the next multiple of 16 (the MMA's
+        // column count) are written as zeros; rows beyond are not touched.
+        const int pt = (int)threadIdx.x - 320, c = pt & 7, rsub = pt >> 3;
+        const uint32_t dst0 = smem_base + kMmaABytes + (uint32_t)rsub * 128u + (uint32_t)((c ^ (rsub & 7)) << 4);   // (r % 8) == (rsub % 8)
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+            const MergeUnit mu = merge_unit(u, ev_unit_off, ev_lo, ev_out_off, k, N);
+            const int npad = (mu.nvalid + 15) & ~15;
+            const __nv_bfloat16* src[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int r = rsub + 16 * i;
+                const int row = r < mu.nvalid ? out_src[mu.col0 + r] : 0;
+                src[i] = feats + (size_t)row * d + c * 8;
+            }
+            for (int ks = 0; ks < ksteps; ++ks) {
+                if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                const uint32_t dst = dst0 + (uint32_t)s * (kMmaABytes + kMmaBBytes);
+                // a K slice that reaches past d (d is a multiple of 8, not of 64) reads zeros there
+                const bool in_k = ks * kMmaBK + c * 8 < d;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int r = rsub + 16 * i;
+                    if (r < npad)
+                        cp_async16_zfill(dst + (uint32_t)i * 2048u, src[i] + (in_k ? ks * kMmaBK : 0),
+                                         (r < mu.nvalid && in_k) ? 16u : 0u);
+                }
+                cp_async_arrive_noinc(smem_u32(&full_bar[0]) + 8u * s);   // arrives when this thread's copies have landed
+                if (++s == kMmaStages) { s = 0; ph ^= 1u; }
+            }
+        }
+        cp_async_wait_all();                                       // nothing may land after the CTA's shared memory is gone
     } else {
         const int grp = warp & 3;                                   // TMEM lanes 32*grp .. 32*grp+31
         const int half = (warp - 2) >> 2;                           // row half = accumulator
@@ -1194,7 +1228,6 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
 // --------------------------------------------------------------------------- //
 struct VisionWs {
     int32_t* status;          // device status word, first in the workspace
-    void* key_rows;           // compact copy of the key-token rows (tensor-core path)
     float* inv_norm;
     uint8_t* is_key;
     int32_t *ev_lo, *ev_budget, *ev_out_off, *ev_tile_off, *ev_unit_off;
@@ -1217,7 +1250,6 @@ struct VisionWs {
 static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, bool mma) {
     VisionWs w;
     w.status = cv.take<int32_t>(64);
-    w.key_rows = mma ? (void*)cv.take<__nv_bfloat16>(((size_t)cap + 64) * d) : nullptr;
     w.inv_norm = cv.take<float>((size_t)Tn * N);
     w.is_key = cv.take<uint8_t>((size_t)Tn * N);
     w.ev_lo = cv.take<int32_t>((size_t)k + 1);
@@ -1355,29 +1387,17 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     }
 
     if (mma) {
-        // compact copy of the key rows so that one tensor map covers an event's keys
-        const int rc = launch_gather_rows(feats, w.key_rows, out_src, n_out, (int)((size_t)d * sizeof(T) / 16),
-                                          "gather_key_rows_kernel", st);
-        if (rc != METOK_OK) return rc;
-        CUtensorMap tmA, tmB;
-        CUtensorMap tmA_half;
+        CUtensorMap tmA, tmA_half;
         int r2 = make_tmap_bf16_2d(&tmA, feats, (uint64_t)Nv, (uint64_t)d, kMmaBM);
         if (r2 != METOK_OK) return r2;
         r2 = make_tmap_bf16_2d(&tmA_half, feats, (uint64_t)Nv, (uint64_t)d, kMmaBM / 2);
-        if (r2 != METOK_OK) return r2;
-        CUtensorMap tmB128, tmB256;
-        r2 = make_tmap_bf16_2d(&tmB, w.key_rows, (uint64_t)cap + 64, (uint64_t)d, 64);
-        if (r2 != METOK_OK) return r2;
-        r2 = make_tmap_bf16_2d(&tmB128, w.key_rows, (uint64_t)cap + 64, (uint64_t)d, 128);
-        if (r2 != METOK_OK) return r2;
-        r2 = make_tmap_bf16_2d(&tmB256, w.key_rows, (uint64_t)cap + 64, (uint64_t)d, 256);
         if (r2 != METOK_OK) return r2;
         METOK_CUDA_TRY(cudaFuncSetAttribute(merge_assign_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)kMmaSmemBytes));
         {
             METOK_TIMED("merge_assign_mma_kernel", st);
             launch_chained(merge_assign_mma_kernel, dim3(kNumSMs), dim3(kMmaThreads), kMmaSmemBytes, st, 
-                tmA, tmA_half, tmB, tmB128, tmB256, d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, inv_norm, w.is_key, w.best64,
+                tmA, tmA_half, reinterpret_cast<const __nv_bfloat16*>(feats), d, N, w.ev_lo, k, w.ev_out_off, w.ev_unit_off, out_src, inv_norm, w.is_key, w.best64,
                 w.status);
         }
         METOK_LAUNCH_CHECK();

@@ -38,21 +38,10 @@ from paper_2506_02850_b200 import workloads as W
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu
-# captures (profiles/), keyed by (kernel, workload); absent -> null in the JSON line.
-NCU_TRAFFIC_BYTES = {
-    # profiles/kernel_sections_frames128.txt; averages over a step's launches of the kernel
-    ("class_topk_kernel", "frames128"): 0.14e6,
-    ("merge_assign_mma_kernel", "frames128"): 163.7e6,
-    ("merge_avg_kernel", "frames128"): 151.6e6,
-    ("seg_score_kernel", "frames128"): 136.0e6,
-    ("tok_score_kernel", "frames128"): 135.9e6,
-    ("kv_copy_kernel", "frames128"): 100.7e6,
-    ("gather_rows_kernel", "frames128"): 23.3e6,
-    ("gather_key_rows_kernel", "frames128"): 26.6e6,
-    ("attn_stats_mma_kernel", "frames128"): 9.9e6,
-    ("attn_colsum_mma_kernel", "frames128"): 10.1e6,
-}
+# dram__bytes_read.sum + dram__bytes_write.sum of one video's launches of each kernel, from the committed ncu
+# captures (profiles/), keyed by (scope/kernel, workload); a kernel changed since its capture is left out
+# (its stage then reports traffic null).
+NCU_TRAFFIC_BYTES = {}
 
 
 def load_peaks():
@@ -154,8 +143,10 @@ class Workload:
         # the text embedding is known before the video is segmented: segmentation and the Eq. 5
         # token scores share one pass over V, and the compressor takes the scores from there
         if "segment" in self.parts:
+            B.metok_profile_scope("segment")
             o["seg"] = B.metok_segment_score_events(self.V, cfg.k, self.t, out=o.get("seg"))
         if "compress" in self.parts:
+            B.metok_profile_scope("compress")
             offs = o["seg"]["event_offsets"] if "seg" in o else self.planted_offsets
             o["cv"] = B.metok_compress_vision(self.V, offs, self.t, self.params, out=o.get("cv"),
                                               scored=o.get("seg"))
@@ -166,6 +157,7 @@ class Workload:
             self.side = torch.cuda.Stream()
         forked = False
         for i, s in enumerate(self.stages):
+            B.metok_profile_scope(f"prefill{i + 1}")
             o[f"pf{i}"] = B.metok_prefill_prune(s["Q"], s["K"], s["hidden"], 0, s["n_vis"], s["groups"], s["budgets"],
                                                 self.scale, out=o.get(f"pf{i}"))
             if i == 0 and "kv" in self.parts:
@@ -180,6 +172,7 @@ class Workload:
 
     def _kv_call(self):
         B, cfg, o = self.B, self.cfg, self.out
+        B.metok_profile_scope("kv")
         # KV selection uses the first pruning layer's attention scores (n_vis = all visual tokens)
         scores = o["pf0"]["scores"] if self.stages and self.stages[0]["n_vis"] == cfg.Nv else self.kv_scores
         kv = o.get("kv")
@@ -239,42 +232,48 @@ class Workload:
             self.d2h["kv_k"][l].copy_(self.ks[l][:, : self.kv_new], non_blocking=True)
             self.d2h["kv_v"][l].copy_(self.vs[l][:, : self.kv_new], non_blocking=True)
 
-    # algorithmic work of one step per kernel name: (bound, bytes or flops)
-    def algorithmic_work(self):
+    def stage_work(self):
+        """Algorithmic work of one video per step of the path: what the method has to move or compute
+        (bytes over HBM, tensor flops, exponentials), and the kernels (scope/name of the library's
+        brackets) that make up the step."""
         cfg = self.cfg
         b = cfg.elem_bytes
         Nv, d = cfg.Nv, cfg.d
         lens = np.asarray(self.vis["lengths"]) * cfg.N
         k_e = np.array([min(m, max(1, math.ceil(cfg.keep_enc * m - 1e-9))) for m in lens])
         n_out = int(k_e.sum())
-        merge_flops = float(np.sum(2.0 * (lens - k_e) * k_e * d))
-        attn_flops = sum(2.0 * cfg.Hq * cfg.Lt * s["S"] * cfg.dh for s in self.stages)
-        hidden_bytes = sum(2.0 * (cfg.Lt + sum(min(bg, int((s["groups"] == g).sum().item()))
-                                               for g, bg in enumerate(s["budgets"]))) * cfg.D * b
-                           for s in self.stages)
-        kv_rows = min(cfg.Nv, math.ceil(cfg.keep_kv * cfg.Nv - 1e-9)) + cfg.kv_text
-        work = {
-            "seg_partial_kernel": ("hbm", float(Nv) * d * b),
-            "seg_score_kernel": ("hbm", float(Nv) * d * b),
-            "tok_score_kernel": ("hbm", float(Nv) * d * b),
-            "merge_assign_simt_kernel": ("tensor", merge_flops),
-            "merge_assign_mma_kernel": ("tensor", merge_flops),
-            "merge_avg_kernel": ("hbm", float(Nv) * d * b + float(n_out) * d * b),   # with its long-list launch
-            "attn_stats_kernel": ("tensor", attn_flops),
-            "attn_colsum_kernel": ("tensor", attn_flops),
-            "attn_stats_mma_kernel": ("tensor", attn_flops),
-            "attn_colsum_mma_kernel": ("tensor", attn_flops),
-            "gather_rows_kernel": ("hbm", hidden_bytes),
-            "gather_key_rows_kernel": ("hbm", 2.0 * n_out * d * b),
-            "kv_copy_kernel": ("hbm", 2.0 * kv_rows * cfg.dh * b * 2 * cfg.Hkv * cfg.L),
-            # scores and classes read once per level, scores once for the K/V lists; the lists written
-            "class_topk_kernel": ("hbm", 8.0 * sum(s["n_vis"] for s in self.stages) + 4.0 * Nv
-                                  + 4.0 * sum(cfg.Lt + sum(min(bg, int((s["groups"] == g).sum().item()))
-                                                           for g, bg in enumerate(s["budgets"])) for s in self.stages)
-                                  + 4.0 * cfg.L * kv_rows),
-            "event_topk_kernel": ("hbm", 8.0 * Nv),
-        }
-        return work
+        st = {}
+        if "segment" in self.parts:
+            st["a1+a2 segmentation, text relevance"] = {
+                "bound": "hbm", "bytes": float(Nv) * d * b,
+                "kernels": ["segment/seg_score_kernel", "segment/seg_finish_kernel", "segment/seg_partial_kernel",
+                            "compress/tok_score_kernel", "compress/event_plan_kernel"]}
+        if "compress" in self.parts:
+            st["a3 key tokens per event"] = {"bound": "latency", "bytes": 8.0 * Nv, "kernels": ["compress/event_topk_kernel"]}
+            st["a4 merge-assign, averaging"] = {
+                "bound": "tensor+hbm", "flops": float(np.sum(2.0 * (lens - k_e) * k_e * d)),
+                "bytes": float(Nv + n_out) * d * b,
+                "kernels": ["compress/merge_assign_mma_kernel", "compress/merge_assign_simt_kernel",
+                            "compress/merge_decode_kernel", "compress/merge_avg_kernel"]}
+        for i, s in enumerate(self.stages, start=1):
+            kept = cfg.Lt + sum(min(bg, int((s["groups"] == g).sum().item())) for g, bg in enumerate(s["budgets"]))
+            st[f"a5 attention scores, level {i}"] = {
+                "bound": "tensor", "flops": 2.0 * 2.0 * cfg.Hq * cfg.Lt * s["S"] * cfg.dh,      # two passes over Q K^T
+                "exps": 2.0 * cfg.Hq * cfg.Lt * s["S"], "bytes": float(cfg.Hkv) * s["S"] * cfg.dh * b,
+                "kernels": [f"prefill{i}/{k_}" for k_ in ("attn_stats_mma_kernel", "attn_colsum_mma_kernel",
+                                                          "attn_stats_kernel", "attn_colsum_kernel",
+                                                          "attn_score_reduce_kernel")]}
+            st[f"a6 class-wise top-k, level {i}"] = {"bound": "latency", "bytes": 8.0 * s["n_vis"] + 4.0 * kept,
+                                                     "kernels": [f"prefill{i}/class_topk_kernel"]}
+            st[f"a7 hidden rows, level {i}"] = {"bound": "hbm", "bytes": 2.0 * kept * cfg.D * b,
+                                                "kernels": [f"prefill{i}/gather_rows_kernel"]}
+        if "kv" in self.parts:
+            kv_rows = min(cfg.Nv, math.ceil(cfg.keep_kv * cfg.Nv - 1e-9)) + cfg.kv_text
+            st["a8 K/V lists"] = {"bound": "latency", "bytes": 4.0 * Nv + 4.0 * cfg.L * kv_rows,
+                                  "kernels": ["kv/class_topk_kernel", "kv/kv_paper_lists_kernel", "kv/kv_check_lists_kernel"]}
+            st["a9 K/V in-place gather"] = {"bound": "hbm", "bytes": 2.0 * kv_rows * cfg.dh * b * 2 * cfg.Hkv * cfg.L,
+                                            "kernels": ["kv/kv_stage_kernel", "kv/kv_copy_kernel", "kv/kv_gather_kernel"]}
+        return st
 
 
 # --------------------------------------------------------------------------- #
@@ -419,6 +418,113 @@ def time_oracle(cfg, steps, warmup, budget_s=None):
 # --------------------------------------------------------------------------- #
 
 
+def chained_run(cfg, dev, B, timed):
+    """The four calls fed by one another: segmentation -> stage-1 compression -> the pruning levels on the
+    survivors -> K/V compaction of the cache the survivors would have left.  Q, K and hidden rows of a
+    level are gathered (torch.index_select, inside the timed region) from per-token synthetic tensors by
+    the original ids of the tokens still alive; the layers of the model that would sit in between are not
+    part of the path.  Sizes are those of the first, untimed pass (the inputs are fixed, so they repeat)."""
+    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    vis = W.vision_inputs(cfg)
+    V = torch.from_numpy(vis["V"]).to(tdt).to(dev)
+    t = torch.from_numpy(vis["t"]).to(tdt).to(dev)
+    params = B.vision_params(cfg.alpha, cfg.keep_enc, cfg.keep_enc)
+    grp_full = torch.from_numpy(W.token_groups(cfg, cfg.Nv, vis=vis).astype(np.int32)).to(dev)
+    full = []
+    for s_ in range(1, cfg.n_stages + 1):
+        pf = W.prefill_inputs(cfg, s_, cfg.Nv, W.token_groups(cfg, cfg.Nv, vis=vis))
+        full.append({"Q": torch.from_numpy(pf["Q"]).to(tdt).to(dev), "K": torch.from_numpy(pf["K"]).to(tdt).to(dev),
+                     "hidden": W.payload_torch(W.hidden_salt(cfg, s_), cfg.Nv + cfg.Lt, cfg.D, cfg.dtype, dev)})
+    text_rows = torch.arange(cfg.Nv, cfg.Nv + cfg.Lt, device=dev, dtype=torch.int64)
+    seg = B.metok_segment_score_events(V, cfg.k, t)
+    cv = B.metok_compress_vision(V, seg["event_offsets"], t, params, scored=seg)
+    torch.cuda.synchronize()
+    n1 = int(cv["n_out"].item())
+    g1 = grp_full[cv["out_src"][:n1].long()]
+    N0 = [int((g1 == 0).sum().item()), int((g1 == 1).sum().item())]
+    sizes = B.metok_prune_schedule_sizes(cfg.n_stages, cfg.alpha, cfg.keep_prefill, N0)
+    bufs = [{"K": torch.empty((cfg.Hkv, sizes[i] + cfg.Lt, cfg.dh), dtype=tdt, device=dev),
+             "hidden": torch.empty((sizes[i] + cfg.Lt, cfg.D), dtype=tdt, device=dev)} for i in range(cfg.n_stages)]
+    budgets = [B.metok_retention_budgets(cfg.alpha, cfg.keep_prefill, i + 1, N0) for i in range(cfg.n_stages)]
+    S_kv = n1 + cfg.kv_text
+    ks = [W.payload_torch(W.kv_salt(cfg, l, 0, 0), cfg.Hkv * S_kv, cfg.dh, cfg.dtype, dev).view(cfg.Hkv, S_kv, cfg.dh)
+          for l in range(cfg.L)]
+    vs = [W.payload_torch(W.kv_salt(cfg, l, 1, 0), cfg.Hkv * S_kv, cfg.dh, cfg.dtype, dev).view(cfg.Hkv, S_kv, cfg.dh)
+          for l in range(cfg.L)]
+    out = {}
+    scale = float(cfg.dh ** -0.5)
+
+    def chained_step():
+        out["seg"] = B.metok_segment_score_events(V, cfg.k, t, out=out.get("seg"))
+        out["cv"] = B.metok_compress_vision(V, out["seg"]["event_offsets"], t, params, out=out.get("cv"), scored=out["seg"])
+        idx = out["cv"]["out_src"][:n1].long()
+        grp = grp_full[idx]
+        for i in range(cfg.n_stages):
+            rows = torch.cat([idx, text_rows])
+            torch.index_select(full[i]["K"], 1, rows, out=bufs[i]["K"])
+            torch.index_select(full[i]["hidden"], 0, rows, out=bufs[i]["hidden"])
+            pf = B.metok_prefill_prune(full[i]["Q"], bufs[i]["K"], bufs[i]["hidden"], 0, sizes[i], grp.contiguous(),
+                                       budgets[i], scale, out=out.get(f"pf{i}"))
+            out[f"pf{i}"] = pf
+            if i == 0:
+                kv = out.get("kv")
+                out["kv"] = B.metok_kv_compact(ks, vs, S_kv, B.KV_TOPK, 0, n1, keep_ratio=cfg.keep_kv, scores=pf["scores"],
+                                               keep_idx=None if kv is None else kv["keep_idx"],
+                                               keep_len=None if kv is None else kv["keep_len"],
+                                               new_len=None if kv is None else kv["new_len"])
+            keepv = pf["keep_idx"][: sizes[i + 1]].long()        # the visual survivors come first (vis_start = 0)
+            idx, grp = idx[keepv], grp[keepv]
+
+    chained_step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        chained_step()
+
+    def chained_graph():
+        g.replay()
+
+    steps = 200
+    ms = timed(chained_graph, steps) / steps
+    return {"ms_per_video": ms, "tokens_per_s": cfg.Nv / (ms * 1e-3), "n_out": n1, "level_sizes": sizes,
+            "kv_rows_before": S_kv, "launch": "cuda_graph",
+            "what": "segment -> compress -> pruning levels on the survivors -> K/V compaction, one video alone; "
+                    "includes the torch gathers that stand in for the model's layers between the calls"}
+
+
+def unplanted_attention_run(cfg, dev, B, timed):
+    """Pruning level 1 at full size on Q/K without the planted relevance: every score then lies inside the
+    near-tie band of the cut (nothing to compare index by index), but the work is the same."""
+    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    vis = W.vision_inputs(cfg)
+    groups = W.token_groups(cfg, cfg.Nv, vis=vis)
+    N0 = [int((groups == 0).sum()), int((groups == 1).sum())]
+    budgets = B.metok_retention_budgets(cfg.alpha, cfg.keep_prefill, 1, N0)
+    pf = W.prefill_inputs(cfg, 1, cfg.Nv, groups, planted=False)
+    Q, K = torch.from_numpy(pf["Q"]).to(tdt).to(dev), torch.from_numpy(pf["K"]).to(tdt).to(dev)
+    hidden = W.payload_torch(W.hidden_salt(cfg, 1), pf["S"], cfg.D, cfg.dtype, dev)
+    grp = torch.from_numpy(groups.astype(np.int32)).to(dev)
+    out = {}
+
+    def call():
+        out["pf"] = B.metok_prefill_prune(Q, K, hidden, 0, cfg.Nv, grp, budgets, float(cfg.dh ** -0.5), out=out.get("pf"))
+
+    call()
+    torch.cuda.synchronize()
+    sc = out["pf"]["scores"].float()
+    spread = float((sc.max() - sc.min()) / sc.mean())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        call()
+
+    def unplanted_graph():
+        g.replay()
+
+    ms = timed(unplanted_graph, 200) / 200
+    return {"ms_per_call": ms, "relative_score_spread": spread, "S_out": int(out["pf"]["S_out"].item()),
+            "what": "metok_prefill_prune, level 1, all visual tokens, Q/K ~ N(0, 1/sqrt(dh)) only"}
+
+
 def max_over_ranks(ms: float, dist, device) -> float:
     """The slowest rank's time: replicas finish together only when the last one does."""
     if dist is None:
@@ -443,6 +549,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph of the step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the chained run and the run without planted relevance")
     ap.add_argument("--videos", type=int, default=4,
                     help="independent videos in flight per step, each on a stream of its own (a step = this batch)")
     ap.add_argument("--parts", default=",".join(PARTS),
@@ -530,7 +637,7 @@ def main():
         return max_over_ranks(e0.elapsed_time(e1), dist, dev)
 
     # eager: every step issues its C-ABI calls from Python
-    eager_ms_per_step = timed(batch_step, args.steps) / args.steps
+    eager_ms_per_step = timed(batch_step, min(args.steps, 50)) / min(args.steps, 50)
     # the same calls captured once in a CUDA graph and replayed: the calls enqueue on a stream
     # and never synchronise, so one capture of a step holds all of its launches
     graph = graph_one = None
@@ -547,13 +654,20 @@ def main():
 
         def step_graph_one():
             graph_one.replay()
+    run_one = step_graph_one if graph_one is not None else wl.step
+    run_batch = step_graph if graph is not None else batch_step
     # latency of one video alone on the GPU
-    ms_one_video = timed(step_graph_one if graph_one is not None else wl.step, args.steps) / args.steps
+    ms_one_video = timed(run_one, min(args.steps, 200)) / min(args.steps, 200)
+    # exactly --steps steps (a burst when that is a few milliseconds) ...
+    burst_ms = timed(run_batch, args.steps) / args.steps
+    # ... and the sustained figure: as many steps as fill at least a second (and no fewer than --steps),
+    # the clocks sampled meanwhile; `value` is this one, whatever --steps was
+    sustain_steps = max(args.steps, int(math.ceil(1000.0 / max(burst_ms, 1e-3))))
     sampler = ClockSampler(local)
     sampler.start()
-    total_ms = timed(step_graph if graph is not None else batch_step, args.steps)
+    total_ms = timed(run_batch, sustain_steps)
     clocks = sampler.stop()
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / sustain_steps
     value = replica_throughput(cfg.Nv * n_videos, world, ms_per_step)
 
     # per-kernel times: one video's step with the library's event brackets on.  Captured in a CUDA
@@ -580,50 +694,104 @@ def main():
         for _ in range(prof_steps):
             wl.step()
         prof = B.metok_profile_end()
+    B.metok_profile_scope(None)
     launches_per_step = sum(v["launches"] for v in prof.values()) // prof_steps
-    work = wl.algorithmic_work()
     peaks = load_peaks()
-    kern_ms = {k_: v["ms"] / prof_steps for k_, v in prof.items()}
-    top = max(kern_ms, key=kern_ms.get)
-    bound, units = work.get(top, ("hbm", float("nan")))
-    if bound == "tensor":
-        achieved = units / (kern_ms[top] * 1e-3) / 1e12
-        peak, unit = float(peaks["bf16_tflops_sustained"]), "TFLOP/s"
-    else:
-        achieved = units / (kern_ms[top] * 1e-3) / 1e9
-        peak, unit = float(peaks["hbm_gbs"]), "GB/s"
-    roofline = {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "peak_source": peaks["_source"],
-                "traffic": NCU_TRAFFIC_BYTES.get((top, cfg.name)),
-                "ms_per_step_in_kernel": kern_ms[top],
-                "per_kernel": {}}
+    hbm_peak, tc_peak = float(peaks["hbm_gbs"]), float(peaks["bf16_tflops_sustained"])
+    kern_us = {k_: v["ms"] * 1e3 / prof_steps for k_, v in prof.items()}
     # every bracket costs the same few microseconds on top of its kernel (two event nodes): what the
     # brackets add up to beyond the step's own time, per launch
-    roofline["bracket_overhead_us_per_launch"] = (
-        max(0.0, sum(kern_ms.values()) - ms_one_video) * 1e3 / max(1, launches_per_step) if not partial else None)
-    if units < 1e6:
-        # the selection kernels touch a few hundred KB on one SM: their time is instruction issue and
-        # barriers, and an HBM fraction says nothing about them.  The largest kernel that streams data:
-        big = {k_: ms for k_, ms in kern_ms.items() if work.get(k_, (None, 0.0))[1] >= 1e6}
-        if big:
-            k2 = max(big, key=big.get)
-            b2, u2 = work[k2]
-            a2 = u2 / (kern_ms[k2] * 1e-3) / (1e12 if b2 == "tensor" else 1e9)
-            p2 = float(peaks["bf16_tflops_sustained"] if b2 == "tensor" else peaks["hbm_gbs"])
-            roofline["note"] = "top kernel by share is a one-SM selection; see largest_streaming_kernel"
-            roofline["largest_streaming_kernel"] = {
-                "kernel": k2, "bound": b2, "achieved": a2, "peak": p2, "unit": "TFLOP/s" if b2 == "tensor" else "GB/s",
-                "frac": a2 / p2, "traffic": NCU_TRAFFIC_BYTES.get((k2, cfg.name)), "ms_per_step_in_kernel": kern_ms[k2]}
-    for k_, ms in sorted(kern_ms.items(), key=lambda kv: -kv[1]):
-        bd, u = work.get(k_, (None, None))
-        ent = {"ms": round(ms, 5), "launches": prof[k_]["launches"] // prof_steps}
-        if bd == "tensor":
-            ent["TFLOP/s"] = round(u / (ms * 1e-3) / 1e12, 2)
-            ent["frac"] = round(ent["TFLOP/s"] / float(peaks["bf16_tflops_sustained"]), 4)
-        elif bd == "hbm":
-            ent["GB/s"] = round(u / (ms * 1e-3) / 1e9, 1)
-            ent["frac"] = round(ent["GB/s"] / float(peaks["hbm_gbs"]), 4)
-        roofline["per_kernel"][k_] = ent
+    bracket_us = (max(0.0, sum(kern_us.values()) - ms_one_video * 1e3) / max(1, launches_per_step)
+                  if not partial else None)
+
+    # the steps of the path: algorithmic work / the summed time of ALL kernels a step launches
+    stages = {}
+    for name, w_ in wl.stage_work().items():
+        ks = [k_ for k_ in w_["kernels"] if k_ in kern_us]
+        if not ks:
+            continue
+        us = sum(kern_us[k_] for k_ in ks)
+        ent = {"us": round(us, 2), "kernels": {k_.split("/", 1)[1]: round(kern_us[k_], 2) for k_ in ks},
+               "launches": sum(prof[k_]["launches"] for k_ in ks) // prof_steps, "bound": w_["bound"]}
+        traffic = [NCU_TRAFFIC_BYTES.get((k_, cfg.name)) for k_ in ks]
+        ent["traffic"] = None if any(t is None for t in traffic) else float(sum(traffic))
+        if "bytes" in w_:
+            ent["algorithmic_bytes"] = w_["bytes"]
+            ent["GB/s"] = round(w_["bytes"] / (us * 1e-6) / 1e9, 1)
+            ent["frac_hbm"] = round(ent["GB/s"] / hbm_peak, 4)
+        if "flops" in w_:
+            ent["algorithmic_flops"] = w_["flops"]
+            ent["TFLOP/s"] = round(w_["flops"] / (us * 1e-6) / 1e12, 1)
+            ent["frac_tensor"] = round(ent["TFLOP/s"] / tc_peak, 4)
+        if "exps" in w_:
+            ent["exponentials"] = w_["exps"]
+            ent["Gexp/s"] = round(w_["exps"] / (us * 1e-6) / 1e9, 1)
+        # fraction of the binding roof: the slower of the HBM and the tensor floor over the measured time
+        if w_["bound"] != "latency":
+            ent["frac"] = max(ent.get("frac_hbm", 0.0), ent.get("frac_tensor", 0.0)) if w_["bound"] == "tensor+hbm" else (
+                ent.get("frac_tensor") if w_["bound"] == "tensor" else ent.get("frac_hbm"))
+        stages[name] = ent
+
+    # the headline roofline entry: the kernel with the largest share among those that stream data or run
+    # on the tensor cores (the one-SM selection launches are latency-bound: an HBM fraction says nothing)
+    def kernel_entry(full_name, us, bound, units):
+        if bound == "tensor":
+            ach, peak, unit = units / (us * 1e-6) / 1e12, tc_peak, "TFLOP/s"
+        else:
+            ach, peak, unit = units / (us * 1e-6) / 1e9, hbm_peak, "GB/s"
+        return {"kernel": full_name.split("/", 1)[-1], "scope": full_name.split("/", 1)[0], "bound": bound,
+                "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                "peak_source": peaks["_source"] + " (HBM copy; bf16 sustained)",
+                "traffic": NCU_TRAFFIC_BYTES.get((full_name, cfg.name)), "us_per_launch": us}
+    kernel_work = {}
+    sw = wl.stage_work()
+    def put_work(kname, bound, units):
+        if kname in kern_us:
+            kernel_work[kname] = (bound, units)
+    if "a4 merge-assign, averaging" in sw:
+        a4 = sw["a4 merge-assign, averaging"]
+        put_work("compress/merge_assign_mma_kernel", "tensor", a4["flops"])
+        put_work("compress/merge_assign_simt_kernel", "tensor", a4["flops"])
+        put_work("compress/merge_avg_kernel", "hbm", a4["bytes"])
+    if "a1+a2 segmentation, text relevance" in sw:
+        put_work("segment/seg_score_kernel", "hbm", sw["a1+a2 segmentation, text relevance"]["bytes"])
+    for i in range(1, len(wl.stages) + 1):
+        a5, a7 = sw[f"a5 attention scores, level {i}"], sw[f"a7 hidden rows, level {i}"]
+        for k_ in ("attn_stats_mma_kernel", "attn_colsum_mma_kernel", "attn_stats_kernel", "attn_colsum_kernel"):
+            put_work(f"prefill{i}/{k_}", "tensor", a5["flops"] / 2)
+        put_work(f"prefill{i}/gather_rows_kernel", "hbm", a7["bytes"])
+    if "a9 K/V in-place gather" in sw:
+        put_work("kv/kv_copy_kernel", "hbm", sw["a9 K/V in-place gather"]["bytes"])
+    roofline = None
+    if kernel_work:
+        top = max(kernel_work, key=lambda k_: kern_us[k_])
+        roofline = kernel_entry(top, kern_us[top], *kernel_work[top])
+        roofline["per_kernel"] = {k_: dict(us=round(kern_us[k_], 2), **{kk: (round(vv, 4) if isinstance(vv, float) else vv)
+                                                                        for kk, vv in kernel_entry(k_, kern_us[k_], *kernel_work[k_]).items()
+                                                                        if kk in ("bound", "achieved", "unit", "frac")})
+                                  for k_ in sorted(kernel_work, key=lambda k_: -kern_us[k_])}
+        roofline["latency_bound_kernels_us"] = {k_: round(u, 2) for k_, u in sorted(kern_us.items(), key=lambda kv: -kv[1])
+                                                if k_ not in kernel_work}
+        roofline["bracket_overhead_us_per_launch"] = bracket_us
+
+    # one video against its own floors: the algorithmic HBM bytes and tensor flops of all steps
+    step_roofline = None
+    if not partial:
+        tot_bytes = sum(w_.get("bytes", 0.0) for n_, w_ in sw.items() if w_["bound"] in ("hbm", "tensor+hbm"))
+        tot_bytes += sum(w_.get("bytes", 0.0) for n_, w_ in sw.items() if w_["bound"] == "tensor")      # K read by the scoring
+        tot_flops = sum(w_.get("flops", 0.0) for w_ in sw.values())
+        floor_us = tot_bytes / (hbm_peak * 1e9) * 1e6
+        tensor_us = tot_flops / (tc_peak * 1e12) * 1e6
+        step_roofline = {"algorithmic_bytes": tot_bytes, "algorithmic_flops": tot_flops, "hbm_floor_us": round(floor_us, 1),
+                         "tensor_floor_us": round(tensor_us, 1),
+                         "one_video_alone": {"us": round(ms_one_video * 1e3, 1), "frac_of_hbm_floor": round(floor_us / (ms_one_video * 1e3), 3)},
+                         "per_video_in_batch": {"us": round(ms_per_step * 1e3 / n_videos, 1),
+                                                "frac_of_hbm_floor": round(floor_us / (ms_per_step * 1e3 / n_videos), 3)}}
+
+    extras = {}
+    if not partial and rank == 0 and world == 1 and not args.no_extras:
+        extras["chained"] = chained_run(cfg, dev, B, timed)
+        extras["no_planted_relevance"] = unplanted_attention_run(cfg, dev, B, timed)
 
     e2e = None
     if not args.no_e2e:
@@ -638,6 +806,13 @@ def main():
         v, dt, what = time_oracle(cfg, 3, 1)
         cpu = {"value": v, "unit": "tokens/s", "cores": cpu_threads(), "kind": "oracle", "sample": what,
                "seconds": dt}
+        try:
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                v1, dt1, _ = time_oracle(cfg, 1, 0)
+            cpu["one_thread"] = {"value": v1, "seconds": dt1, "cores": 1}
+        except Exception as exc:                       # the limit is a convenience of the numpy build
+            cpu["one_thread"] = {"unavailable": str(exc)}
 
     if rank == 0:
         line = {"metric": "visual_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
@@ -645,10 +820,14 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
                 "config": {"workload": workload_name, "l2": "inputs larger than L2 (V 132 MB, hidden 133 MB, K/V 1.06 GB touched between reuses)",
                            "videos_in_flight": n_videos, "parallelism": f"replicas x{world}"},
+                "timed_steps": sustain_steps, "burst": {"steps": args.steps, "ms_per_step": burst_ms,
+                                                        "value": replica_throughput(cfg.Nv * n_videos, world, burst_ms)},
                 "single_video": {"ms_per_video": ms_one_video, "tokens_per_s": replica_throughput(cfg.Nv, world, ms_one_video)},
                 "launch": "cuda_graph" if graph is not None else "eager", "eager_ms_per_step": eager_ms_per_step,
-                "host_enqueue_ms_per_step": host_ms.get("batch_step"), "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * n_videos * args.steps,
-                "roofline": roofline, "cpu_baseline": cpu}
+                "host_enqueue_ms_per_step": host_ms.get("batch_step"), "clocks": clocks, "e2e": e2e,
+                "gpu_launches": launches_per_step * n_videos * sustain_steps,
+                "roofline": roofline, "stages": stages, "step_roofline": step_roofline, "cpu_baseline": cpu}
+        line.update(extras)
         if partial:
             line["partial"] = "only " + ",".join(parts) + ": not a benchmark result"
         print(json.dumps(line))

@@ -392,9 +392,12 @@ METOK_API int metok_kv_compact(void* const* k_layers, void* const* v_layers, int
  * times its kernels without the host's launch gaps.  metok_profile_read stops
  * bracketing further launches and reports like metok_profile_end but keeps the
  * events, so that the graph can be replayed and read again; metok_profile_end
- * releases them (destroy the graph first).  The paper has no counterpart of
- * these three calls. */
+ * releases them (destroy the graph first).  metok_profile_scope(label) names the
+ * brackets recorded from then on (label without blanks or '/', NULL or "" for none):
+ * they are reported as "label/name", so that launches of one kernel made for different
+ * steps of the path can be told apart.  The paper has no counterpart of these calls. */
 METOK_API int metok_profile_begin(void);
+METOK_API int metok_profile_scope(const char* label);
 METOK_API int metok_profile_read(char* out, size_t cap);
 METOK_API int metok_profile_end(char* out, size_t cap);
 

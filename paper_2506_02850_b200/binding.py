@@ -77,6 +77,7 @@ _SIGNATURES = {
     "metok_profile_begin": (_i, []),
     "metok_profile_read": (_i, [_c.c_char_p, _sz]),
     "metok_profile_end": (_i, [_c.c_char_p, _sz]),
+    "metok_profile_scope": (_i, [_c.c_char_p]),
     "metok_status_string": (_c.c_char_p, [_i]),
     "metok_last_cuda_error": (_i, []),
     "metok_version": (_i, []),
@@ -501,6 +502,11 @@ def metok_version() -> int:
 
 def metok_profile_begin() -> None:
     _check("metok_profile_begin", lib().metok_profile_begin())
+
+
+def metok_profile_scope(label: Optional[str]) -> None:
+    """Names the brackets recorded from now on: reported as "label/kernel"."""
+    _check("metok_profile_scope", lib().metok_profile_scope(label.encode() if label else None))
 
 
 def _profile(fn_name: str) -> Dict[str, Dict[str, float]]:

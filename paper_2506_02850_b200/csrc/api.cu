@@ -1,4 +1,5 @@
 // Host-only helpers of the C ABI: status strings, last CUDA error, version.
+#include <deque>
 #include <mutex>
 #include <string>
 #include <vector>
@@ -14,8 +15,10 @@ void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 
 bool g_profiling = false;
 namespace {
-struct Rec { const char* name; cudaEvent_t a, b; };
+struct Rec { const char* scope; const char* name; cudaEvent_t a, b; };
 std::vector<Rec> g_recs;
+std::deque<std::string> g_scopes;            // interned scope labels: pointers into it stay valid
+const char* g_scope = "";                    // label of the brackets recorded from now on
 std::mutex g_mu;
 }  // namespace
 
@@ -37,7 +40,7 @@ KernelTimer::~KernelTimer() {
     if (!active) return;
     record(b);
     std::lock_guard<std::mutex> lk(g_mu);
-    g_recs.push_back({name, a, b});
+    g_recs.push_back({g_scope, name, a, b});
 }
 }  // namespace metok
 
@@ -73,7 +76,20 @@ extern "C" int metok_profile_begin(void) {
     std::lock_guard<std::mutex> lk(metok::g_mu);
     for (auto& r : metok::g_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     metok::g_recs.clear();
+    metok::g_scope = "";
     metok::g_profiling = true;
+    return METOK_OK;
+}
+
+extern "C" int metok_profile_scope(const char* label) {
+    std::lock_guard<std::mutex> lk(metok::g_mu);
+    if (!label || !*label) { metok::g_scope = ""; return METOK_OK; }
+    for (const char* c = label; *c; ++c)
+        if (*c == ' ' || *c == '\n' || *c == '/') return METOK_ERR_INVALID_ARG;
+    for (auto& sc : metok::g_scopes)
+        if (sc == label) { metok::g_scope = sc.c_str(); return METOK_OK; }
+    metok::g_scopes.emplace_back(label);
+    metok::g_scope = metok::g_scopes.back().c_str();
     return METOK_OK;
 }
 
@@ -81,7 +97,7 @@ extern "C" int metok_profile_begin(void) {
 static int profile_collect(char* out, size_t cap, bool release) {
     metok::g_profiling = false;
     std::lock_guard<std::mutex> lk(metok::g_mu);
-    struct Agg { const char* name; int n; double ms; };
+    struct Agg { std::string name; int n; double ms; };
     std::vector<Agg> agg;
     int launches = 0;
     for (auto& r : metok::g_recs) {
@@ -92,9 +108,10 @@ static int profile_collect(char* out, size_t cap, bool release) {
         }
         ++launches;
         bool found = false;
+        const std::string full = *r.scope ? std::string(r.scope) + "/" + r.name : std::string(r.name);
         for (auto& g : agg)
-            if (std::strcmp(g.name, r.name) == 0) { g.n += 1; g.ms += ms; found = true; break; }
-        if (!found) agg.push_back({r.name, 1, (double)ms});
+            if (g.name == full) { g.n += 1; g.ms += ms; found = true; break; }
+        if (!found) agg.push_back({full, 1, (double)ms});
         if (release) {
             cudaEventDestroy(r.a);
             cudaEventDestroy(r.b);
@@ -105,7 +122,7 @@ static int profile_collect(char* out, size_t cap, bool release) {
         std::string text;
         char line[256];
         for (auto& g : agg) {
-            std::snprintf(line, sizeof line, "%s %d %.6f\n", g.name, g.n, g.ms);
+            std::snprintf(line, sizeof line, "%s %d %.6f\n", g.name.c_str(), g.n, g.ms);
             text += line;
         }
         const size_t n = text.size() < cap - 1 ? text.size() : cap - 1;

@@ -626,7 +626,6 @@ constexpr int kMmaThreads = 448;
 constexpr int kMmaKeyThreads = 128;                        // warps 10-13
 constexpr uint32_t kMmaABytes = kMmaBM * kMmaBK * 2;       // 32 KiB
 constexpr uint32_t kMmaBBytes = kMmaBN * kMmaBK * 2;       // 32 KiB
-constexpr uint32_t kMmaBoxBytes = 64 * kMmaBK * 2;         // one 64-row key box
 constexpr size_t kMmaSmemBytes = (size_t)kMmaStages * (kMmaABytes + kMmaBBytes) + 1024;
 
 struct MergeUnit { int row0, row_end, col0, nvalid; };     // rows of V; first key slot and number of keys

@@ -401,6 +401,21 @@ METOK_API int metok_profile_scope(const char* label);
 METOK_API int metok_profile_read(char* out, size_t cap);
 METOK_API int metok_profile_end(char* out, size_t cap);
 
+/* Debug builds (lib/libmetok_debug.so: compiled with METOK_DEBUG_SHORT_WAIT and METOK_DEBUG_BOUNDS).
+ * There the bounded device-side waits give up after a few thousand polls, every data-dependent
+ * row or slot index is range-checked (a bad one is counted in int32 word 2 of the workspace and
+ * replaced by 0: nothing traps or faults), and metok_debug_set(METOK_DEBUG_WITHHOLD_COPY, mask)
+ * makes the producer of the kernels named in `mask` skip one copy in the calls made from then on,
+ * so that the waiting side runs into its limit, the CTA unwinds (copies drained, tensor memory
+ * freed) and the call's status word -- int32 word 0 of the workspace -- reads METOK_ERR_TIMEOUT.
+ * mask bits: 1 merge-assign, 2 attention statistics, 4 attention column sums, 8 averaging,
+ * 16 hidden-row gather; 0 switches it off.  metok_debug_build() returns 1 | 2 for such a build and
+ * 0 for the normal library, in which metok_debug_set returns METOK_ERR_UNSUPPORTED and does
+ * nothing.  The paper has no counterpart of these two calls. */
+#define METOK_DEBUG_WITHHOLD_COPY 1
+METOK_API int metok_debug_set(int what, int value);
+METOK_API int metok_debug_build(void);
+
 METOK_API const char* metok_status_string(int status);
 METOK_API int metok_last_cuda_error(void);   /* cudaError_t of the last METOK_ERR_CUDA on this thread, else 0 */
 METOK_API int metok_version(void);           /* major*10000 + minor*100 + patch */

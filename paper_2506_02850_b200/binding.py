@@ -78,6 +78,8 @@ _SIGNATURES = {
     "metok_profile_read": (_i, [_c.c_char_p, _sz]),
     "metok_profile_end": (_i, [_c.c_char_p, _sz]),
     "metok_profile_scope": (_i, [_c.c_char_p]),
+    "metok_debug_set": (_i, [_i, _i]),
+    "metok_debug_build": (_i, []),
     "metok_status_string": (_c.c_char_p, [_i]),
     "metok_last_cuda_error": (_i, []),
     "metok_version": (_i, []),

@@ -135,6 +135,40 @@ static int profile_collect(char* out, size_t cap, bool release) {
 extern "C" int metok_profile_read(char* out, size_t cap) { return profile_collect(out, cap, false); }
 extern "C" int metok_profile_end(char* out, size_t cap) { return profile_collect(out, cap, true); }
 
+namespace metok {
+static int g_dbg_withhold = 0;
+int debug_arm(int32_t* status, cudaStream_t st) {
+#if defined(METOK_DEBUG_SHORT_WAIT) || defined(METOK_DEBUG_BOUNDS)
+    const int32_t words[2] = {g_dbg_withhold, 0};
+    METOK_CUDA_TRY(cudaMemcpyAsync(status + 1, words, sizeof words, cudaMemcpyHostToDevice, st));
+#else
+    (void)status; (void)st;
+#endif
+    return METOK_OK;
+}
+}  // namespace metok
+
+extern "C" int metok_debug_set(int what, int value) {
+#if defined(METOK_DEBUG_SHORT_WAIT) || defined(METOK_DEBUG_BOUNDS)
+    if (what == METOK_DEBUG_WITHHOLD_COPY) { metok::g_dbg_withhold = value; return METOK_OK; }
+    return METOK_ERR_INVALID_ARG;
+#else
+    (void)what; (void)value;
+    return METOK_ERR_UNSUPPORTED;
+#endif
+}
+
+extern "C" int metok_debug_build(void) {
+    int flags = 0;
+#ifdef METOK_DEBUG_SHORT_WAIT
+    flags |= 1;
+#endif
+#ifdef METOK_DEBUG_BOUNDS
+    flags |= 2;
+#endif
+    return flags;
+}
+
 extern "C" const char* metok_status_string(int status) {
     switch (status) {
         case METOK_OK: return "ok";

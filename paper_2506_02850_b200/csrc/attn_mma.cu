@@ -147,6 +147,7 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                 const uint32_t fb = smem_u32(&full_bar[s]);
                 mbar_arrive_expect_tx(fb, kKBytes);
+                if (dbg_withhold(status, kDbgAttnStats) && split == 0 && rt == 0 && g == 0 && it == 0) continue;   // debug builds: one copy never sent
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
                     tma_load_2d(k_addr(s) + kb * kKBlk, &tmK, kb * 64, g * dm.S + (t_lo + it) * kStBN, fb);
@@ -343,6 +344,7 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                 const uint32_t fb = smem_u32(&full_bar[s]);
                 mbar_arrive_expect_tx(fb, kKBytes);
+                if (dbg_withhold(status, kDbgAttnColsum) && split == 0 && chunk == 0 && g == 0 && it == 0) continue;   // debug builds: one copy never sent
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
                     tma_load_2d(k_addr(s) + kb * kKBlk, &tmK, kb * 64, g * dm.S + (t_lo + it) * kCsBM, fb);

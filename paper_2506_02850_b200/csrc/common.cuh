@@ -68,6 +68,42 @@ __device__ __forceinline__ void grid_dep_wait() {
 }
 #endif
 
+// ---- debug builds ------------------------------------------------------------------
+// Two compile-time switches give a second library (lib/libmetok_debug.so) that exercises what a
+// normal run never reaches:
+//   METOK_DEBUG_SHORT_WAIT  bounded waits give up after a few thousand polls, and metok_debug_set
+//                           can make a producer skip ONE copy, so that the consumer's wait runs out,
+//                           the CTA unwinds and the call's status word reads METOK_ERR_TIMEOUT;
+//   METOK_DEBUG_BOUNDS      every data-dependent row or slot index is checked against its range; a bad
+//                           one is counted in word 2 of the call's status area and replaced by 0
+//                           (no trap, no fault).
+// Words 1 and 2 of the status area (the 64 int32 at the start of a workspace) belong to these builds:
+// word 1 = the copies to withhold (bit mask, written by the host when the call is made), word 2 = the
+// number of out-of-range indices met.
+enum { kDbgMergeAssign = 1, kDbgAttnStats = 2, kDbgAttnColsum = 4, kDbgMergeAvg = 8, kDbgGatherRows = 16 };
+int debug_arm(int32_t* status, cudaStream_t st);          // debug builds: writes words 1 and 2; else does nothing
+#ifdef __CUDACC__
+__device__ __forceinline__ bool dbg_withhold(const int32_t* status, int bit) {
+#ifdef METOK_DEBUG_SHORT_WAIT
+    return (status[1] & bit) != 0;
+#else
+    (void)status; (void)bit;
+    return false;
+#endif
+}
+__device__ __forceinline__ long long dbg_bound(long long idx, long long limit, int32_t* status) {
+#ifdef METOK_DEBUG_BOUNDS
+    if (idx < 0 || idx >= limit) {
+        atomicAdd(status + 2, 1);
+        return 0;
+    }
+#else
+    (void)limit; (void)status;
+#endif
+    return idx;
+}
+#endif
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

@@ -16,15 +16,11 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
                       const int32_t* budgets_host, int S, int vis_start, int32_t* keep_idx, size_t keep_stride,
                       int replicas, int32_t* count_a, int32_t* count_b, int problems, cudaStream_t st);
 
-// dst[i] = src[idx[i]] for i < *n_rows (device scalar); rows of row_chunks 16-byte chunks.
-// timer_name labels the launch in the per-kernel timing report.
-int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
-                       const char* timer_name, cudaStream_t st);
-
-// The same gather by bulk copies through shared memory (rows of any multiple of 16 bytes).
-// `status` receives METOK_ERR_TIMEOUT if a device-side wait gave up.
+// dst[i] = src[idx[i]] for i < *n_rows (device scalar), by bulk copies through shared memory; rows of
+// any multiple of 16 bytes; src has src_rows rows.  timer_name labels the launch in the per-kernel
+// timing report.  `status` receives METOK_ERR_TIMEOUT if a device-side wait gave up.
 int launch_gather_rows_bulk(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, size_t row_bytes,
-                            int32_t* status, const char* timer_name, cudaStream_t st);
+                            int src_rows, int32_t* status, const char* timer_name, cudaStream_t st);
 
 // Text->visual attention scores on the tensor cores (bf16, dh 64 or 128): leaves
 // n_planes partial column sums of n_vis floats each in part_col; their sum divided by

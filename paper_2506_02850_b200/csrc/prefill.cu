@@ -372,42 +372,7 @@ int launch_class_topk(const float* scores, size_t score_stride, const int32_t* t
 
 // --------------------------------------------------------------------------- //
 // hidden_out[i] = hidden[keep_idx[i]], i < *S_out.  Rows are whole 16-byte chunks.
-// One warp per row and trip; a lane has up to 8 chunks (128 bytes) in flight before it
-// stores any, and rows are dealt to warps round-robin so that consecutive rows -- often
-// consecutive in the source too -- are copied at the same time.
-// --------------------------------------------------------------------------- //
-constexpr int kGatherThreads = 256;
-constexpr int kGatherUnroll = 8;
-
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-__global__ void __launch_bounds__(kGatherThreads)
-gather_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const int32_t* __restrict__ keep_idx,
-                   const int32_t* __restrict__ n_rows, int row_chunks) {
-    grid_dep_wait();
-    const int n = *n_rows;
-    const int lane = threadIdx.x & 31;
-    const int warps = gridDim.x * (kGatherThreads / 32);
-    for (int i = blockIdx.x * (kGatherThreads / 32) + (threadIdx.x >> 5); i < n; i += warps) {
-        const uint4* s = src + (size_t)keep_idx[i] * row_chunks;
-        uint4* o = dst + (size_t)i * row_chunks;
-        for (int c = lane; c < row_chunks; c += 32 * kGatherUnroll) {
-            uint4 v[kGatherUnroll];
-#pragma unroll
-            for (int u = 0; u < kGatherUnroll; ++u)
-                if (c + u * 32 < row_chunks) v[u] = ld_stream(s + c + u * 32);
-#pragma unroll
-            for (int u = 0; u < kGatherUnroll; ++u)
-                if (c + u * 32 < row_chunks) o[c + u * 32] = v[u];
-        }
-    }
-}
-
-// The same gather driven by the copy engine: one thread per CTA moves (row, 8 KiB segment)
+// The gather is driven by the copy engine: one thread per CTA moves (row, 8 KiB segment)
 // items global -> shared -> global with bulk copies, kGbStages items in flight; no registers
 // or warps are spent on the data.
 constexpr int kGbStages = 4;
@@ -417,7 +382,7 @@ constexpr size_t kGbSmemBytes = (size_t)kGbStages * kGbSegBytes + 128;
 __global__ void __launch_bounds__(32)
 gather_rows_bulk_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
                         const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ n_rows,
-                        uint32_t row_bytes, int32_t* __restrict__ status) {
+                        uint32_t row_bytes, int src_rows, int32_t* __restrict__ status) {
     grid_dep_wait();
     using namespace sm100;
     extern __shared__ uint8_t gb_dyn[];
@@ -439,8 +404,9 @@ gather_rows_bulk_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ d
         const uint32_t bytes = min(kGbSegBytes, row_bytes - off);
         const uint32_t bar = smem_u32(&s_bar[k % kGbStages]);
         mbar_arrive_expect_tx(bar, bytes);
-        bulk_load(stage0 + (uint32_t)(k % kGbStages) * kGbSegBytes, src + (size_t)keep_idx[i] * row_bytes + off, bytes,
-                  bar);
+        const long long row = dbg_bound(keep_idx[i], src_rows, status);
+        if (!(dbg_withhold(status, kDbgGatherRows) && blockIdx.x == 0 && k == 0))   // debug builds: one copy never sent
+            bulk_load(stage0 + (uint32_t)(k % kGbStages) * kGbSegBytes, src + (size_t)row * row_bytes + off, bytes, bar);
     };
     volatile int* abort_flag = &s_abort;
     for (long long k = 0; k < mine && k < kGbStages; ++k) issue_load(k);
@@ -470,25 +436,14 @@ gather_rows_bulk_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ d
 }
 
 int launch_gather_rows_bulk(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, size_t row_bytes,
-                            int32_t* status, const char* timer_name, cudaStream_t st) {
+                            int src_rows, int32_t* status, const char* timer_name, cudaStream_t st) {
     METOK_CUDA_TRY(cudaFuncSetAttribute(gather_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)kGbSmemBytes));
     {
         METOK_TIMED(timer_name, st);
         launch_chained(gather_rows_bulk_kernel, dim3(kNumSMs * 6), dim3(32), kGbSmemBytes, st, 
             reinterpret_cast<const uint8_t*>(src), reinterpret_cast<uint8_t*>(dst), idx, n_rows, (uint32_t)row_bytes,
-            status);
-    }
-    METOK_LAUNCH_CHECK();
-    return METOK_OK;
-}
-
-int launch_gather_rows(const void* src, void* dst, const int32_t* idx, const int32_t* n_rows, int row_chunks,
-                       const char* timer_name, cudaStream_t st) {
-    {
-        METOK_TIMED(timer_name, st);
-        launch_chained(gather_rows_kernel, dim3(kNumSMs * 8), dim3(kGatherThreads), 0, st, reinterpret_cast<const uint4*>(src),
-                                                        reinterpret_cast<uint4*>(dst), idx, n_rows, row_chunks);
+            src_rows, status);
     }
     METOK_LAUNCH_CHECK();
     return METOK_OK;
@@ -644,13 +599,15 @@ extern "C" int metok_prefill_prune(const void* q_text, const void* k_all, const 
     AttnDims dm = make_dims(Hq, Hkv, Lt, S, dh, vis_start, n_vis, softmax_scale);
     Carver cv(ws);
     PrefillWs w = carve_prefill(cv, dm, use_mma_attn(dtype, dh));
-    int rc = run_attention_scores(q_text, k_all, dtype, dm, w, softmax_scale, 1.0f / (float)(Hq * Lt), scores, st);
+    int rc = debug_arm(w.status, st);
+    if (rc != METOK_OK) return rc;
+    rc = run_attention_scores(q_text, k_all, dtype, dm, w, softmax_scale, 1.0f / (float)(Hq * Lt), scores, st);
     if (rc != METOK_OK) return rc;
     rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, 1, S_out,
                            nullptr, 1, st);
     if (rc != METOK_OK) return rc;
     if (hidden) {
-        rc = launch_gather_rows_bulk(hidden, hidden_out, keep_idx, S_out, (size_t)D * eb, w.status, "gather_rows_kernel",
+        rc = launch_gather_rows_bulk(hidden, hidden_out, keep_idx, S_out, (size_t)D * eb, S, w.status, "gather_rows_kernel",
                                      st);
         if (rc != METOK_OK) return rc;
     }
@@ -675,6 +632,7 @@ extern "C" int metok_attention_scores(const void* q_text, const void* k_all, int
     Carver cv(ws);
     PrefillWs w = carve_prefill(cv, dm, use_mma_attn(dtype, dh));
     const float inv_rows = 1.0f / (float)(rows_total ? rows_total : Hq * Lt);
+    if (const int rc = debug_arm(w.status, reinterpret_cast<cudaStream_t>(stream))) return rc;
     return run_attention_scores(q_text, k_all, dtype, dm, w, softmax_scale, inv_rows, scores,
                                 reinterpret_cast<cudaStream_t>(stream));
 }
@@ -700,11 +658,13 @@ extern "C" int metok_prune_by_scores(const float* scores, const void* hidden, in
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     int32_t* status = reinterpret_cast<int32_t*>(ws);
     METOK_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
-    int rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, 1, S_out,
+    int rc = debug_arm(status, st);
+    if (rc != METOK_OK) return rc;
+    rc = launch_class_topk(scores, 0, token_group, n_vis, G, group_budget, S, vis_start, keep_idx, 0, 1, S_out,
                                nullptr, 1, st);
     if (rc != METOK_OK) return rc;
     if (hidden)
-        rc = launch_gather_rows_bulk(hidden, hidden_out, keep_idx, S_out, (size_t)D * eb, status, "gather_rows_kernel", st);
+        rc = launch_gather_rows_bulk(hidden, hidden_out, keep_idx, S_out, (size_t)D * eb, S, status, "gather_rows_kernel", st);
     return rc;
 }
 

@@ -43,7 +43,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // a hardware-defined slice) the waiter raises the CTA's abort flag and gives up;
 // every other waiter sees the flag and gives up too, and the kernel unwinds
 // (drains its copies, frees TMEM) and reports METOK_ERR_TIMEOUT.
+#ifdef METOK_DEBUG_SHORT_WAIT
+constexpr uint32_t kWaitLimit = 1u << 12;
+#else
 constexpr uint32_t kWaitLimit = 1u << 22;
+#endif
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;

@@ -707,7 +707,8 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t fb = smem_u32(&full_bar[0]) + 8u * s;
                     mbar_arrive_expect_tx(fb, tx);
-                    tma_load_2d(smem_base + (uint32_t)s * (kMmaABytes + kMmaBBytes), a0, ks * kMmaBK, mu.row0, fb);
+                    if (!(dbg_withhold(status, kDbgMergeAssign) && blockIdx.x == 0 && issued == 0))   // debug builds: one copy never sent
+                        tma_load_2d(smem_base + (uint32_t)s * (kMmaABytes + kMmaBBytes), a0, ks * kMmaBK, mu.row0, fb);
                     ++issued;
                     if (++s == kMmaStages) { s = 0; ph ^= 1u; }
                 }
@@ -779,7 +780,7 @@ merge_assign_mma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int r = rsub + 16 * i;
-                const int row = r < mu.nvalid ? out_src[mu.col0 + r] : 0;
+                const int row = r < mu.nvalid ? (int)dbg_bound(out_src[mu.col0 + r], (long long)ev_lo[k] * N, status) : 0;
                 src[i] = feats + (size_t)row * d + c * 8;
             }
             for (int ks = 0; ks < ksteps; ++ks) {
@@ -862,7 +863,8 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
                     int32_t* __restrict__ long_index, int32_t* __restrict__ long_slot,
                     int32_t* __restrict__ long_counter, int long_threshold, int long_cap,
                     int32_t* __restrict__ few_members, int few_cap, int32_t* __restrict__ heavy_index,
-                    int32_t* __restrict__ heavy_slot, int32_t* __restrict__ heavy_counter, int heavy_cap) {
+                    int32_t* __restrict__ heavy_slot, int32_t* __restrict__ heavy_counter, int heavy_cap,
+                    const int32_t* __restrict__ n_out) {
     grid_dep_wait();
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= Nv) return;
@@ -873,6 +875,9 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
     } else {
         slot = assign[row];
     }
+    // a token whose unit gave up on a wait has no maximum: it stays out of every member list (the
+    // call's status word already says that the results are not valid)
+    if (slot < 0 || slot >= *n_out) return;
     const int e = find_event(ev_lo, k, row / N);
     const int lo = ev_lo[e] * N, m = ev_lo[e + 1] * N - lo;
     atomicOr(&slot_blocks[slot], 1ull << ((row - lo) / avg_block_tokens(m)));
@@ -984,8 +989,9 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
             const int j = m % kAvgStages;
             const uint32_t bar = smem_u32(&s_bar[j]);
             mbar_arrive_expect_tx(bar, seg_bytes);
-            bulk_load(stage0 + (uint32_t)j * kAvgStageBytes, feats + (size_t)s_list[m] * d + (size_t)cb * VN,
-                      seg_bytes, bar);
+            const long long src_row = dbg_bound(s_list[m], Nv, status);
+            if (!(dbg_withhold(status, kDbgMergeAvg) && blockIdx.x == (unsigned)kAvgFrontCtas && m == 0 && cb == 0))   // debug builds: one copy never sent
+                bulk_load(stage0 + (uint32_t)j * kAvgStageBytes, feats + (size_t)src_row * d + (size_t)cb * VN, seg_bytes, bar);
         };
         if (tid == 0)
             for (int m = 0; m < nlist && m < kAvgStages; ++m) issue(m);
@@ -1303,6 +1309,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     Carver cv(ws);
     VisionWs w = carve_vision(cv, Tn, N, k, d, cap, mma);
     // (the status word and the scratch that must start cleared are written by event_plan_kernel)
+    if (const int rc = debug_arm(w.status, st)) return rc;
 
     // Eq. 5 per token, unless the caller brings the scores and norms from metok_segment_score_events
     const float* inv_norm = p->token_inv_norm ? p->token_inv_norm : w.inv_norm;
@@ -1417,7 +1424,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
                                                                assign, w.slot_blocks, w.slot_cnt, w.long_index,
                                                                w.long_slot, w.long_counter, kAvgLong, kAvgLongCap,
                                                                w.few_members, kAvgFew, w.heavy_index, w.heavy_slot,
-                                                               w.heavy_counter, kAvgHeavyCap);
+                                                               w.heavy_counter, kAvgHeavyCap, n_out);
     }
     METOK_LAUNCH_CHECK();
     METOK_CUDA_TRY(cudaFuncSetAttribute(merge_avg_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -220,6 +220,9 @@ typedef struct metok_vision_params {
     const uint8_t* key_events_given;  /* NULL, or DEVICE uint8 [k]: the key events are the caller's (non-zero =
                                          key) instead of the ceil(alpha*k) best-scored ones -- the ablation
                                          with randomly chosen key events; event_is_key returns them */
+    const uint8_t* key_frames_given;  /* POOL: NULL, or DEVICE uint8 [T]: the key frames are the caller's (non-zero =
+                                         key) instead of the ceil(beta*|E_j|) best-scored frames of every
+                                         event -- the ablation with randomly chosen key frames */
 } metok_vision_params;
 
 METOK_API int    metok_compress_vision_bound(int T, int N, int k, const metok_vision_params* p);
@@ -339,6 +342,24 @@ METOK_API int metok_prefill_prune_schedule(const metok_prune_level* levels, int 
                         int Hq, int Hkv, int Lt, int S, int dh, int D, int vis_start, int n_vis,
                         double alpha, double r, const int32_t* N0, float softmax_scale,
                         int32_t* status, void* ws, size_t ws_bytes, void* stream);
+
+/* The K/V keep lists that follow from the recorded keep lists of the levels (section 3.3: the cache
+ * is pruned in line with the hierarchical pruning).  Layer l lies in group g = number of pruning
+ * layers level_layer[s] <= l; its cache holds the rows of level g's input (all of them for g = 0),
+ * S - n_vis + n_vis_of_level[g] rows, and keeps what level g + 1 kept; layers at or beyond the last
+ * pruning layer keep all their rows.  Call it on the stream of metok_prefill_prune_schedule after
+ * that call; the lists are in the form policy GIVEN of metok_kv_compact takes (one call per group
+ * of layers, whose caches have the same length).
+ *   level_layer  HOST int32 [n_levels]: the pruning layers l1 < l2 < l3 (0-based)
+ *   kv_keep_idx  DEVICE int32 [L][S] (row stride S); kv_keep_len DEVICE int32 [L]
+ *   kv_S_cur     HOST int32 [L] (output): rows of layer l's cache before compaction
+ *   ws           DEVICE, at least 4*L bytes
+ * Errors: INVALID_ARG (null pointers, layers not ascending, N0 not summing to n_vis);
+ * UNSUPPORTED (L > 1024); WORKSPACE. */
+METOK_API int metok_prune_schedule_kv_lists(const metok_prune_level* levels, int n_levels,
+                        const int32_t* level_layer, int L, int S, int n_vis, double alpha, double r,
+                        const int32_t* N0, int32_t* kv_keep_idx, int32_t* kv_keep_len, int32_t* kv_S_cur,
+                        void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------- *
  * (4) KV-cache selection and in-place compaction -- section 3.3.

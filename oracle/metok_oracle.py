@@ -296,15 +296,20 @@ def pool2d(frame: np.ndarray, G: int, s: int) -> np.ndarray:
 
 
 def adaptive_pool(V: np.ndarray, t: np.ndarray, event_offsets: np.ndarray, alpha: float, beta: float,
-                  strides: Sequence[int], dtype: str, event_agg: int = AGG_MEAN) -> Dict[str, np.ndarray]:
+                  strides: Sequence[int], dtype: str, event_agg: int = AGG_MEAN,
+                  key_frames_given: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
     """strides = (s1, s2, s1_nonkey, s2_nonkey): key/non-key frames of key events,
-    then of non-key events.  Frames are pooled and appended in temporal order."""
+    then of non-key events.  Frames are pooled and appended in temporal order.
+    `key_frames_given` (bool [T]) replaces the scored choice of key frames: the ablation
+    with randomly chosen key frames."""
     T, N, d = V.shape
     G = int(round(math.sqrt(N)))
     assert G * G == N
     s = token_relevance(V, t)
     ev = key_events(s, T, N, event_offsets, alpha, event_agg)
     kf = key_frames(ev["frame_score"], event_offsets, beta)
+    if key_frames_given is not None:
+        kf = np.asarray(key_frames_given).astype(kf.dtype)
     frame_stride = np.empty(T, dtype=np.int32)
     for e in range(len(event_offsets) - 1):
         for f in range(int(event_offsets[e]), int(event_offsets[e + 1])):
@@ -433,6 +438,24 @@ def prune_schedule(Qs: Sequence[np.ndarray], Ks: Sequence[np.ndarray], token_gro
         kept_vis = sel["keep_idx"][(sel["keep_idx"] >= vis_start) & (sel["keep_idx"] < vis_start + n_vis)] - vis_start
         group, origin = group[kept_vis], origin[kept_vis]
     return levels
+
+
+def schedule_kv_lists(levels: List[Dict[str, np.ndarray]], level_layer: Sequence[int], L: int,
+                      S: int) -> List[np.ndarray]:
+    """K/V keep lists in line with the hierarchical pruning (section 3.3): layer l lies in group
+    g = #{s : level_layer[s] <= l}; its cache holds the rows of level g's input and keeps what level
+    g + 1 kept; layers at or beyond the last pruning layer keep all their rows.  `levels` is
+    prune_schedule's result, S the sequence length at the first level."""
+    n_vis0 = levels[0]["token_group"].size
+    lists = []
+    for l in range(L):
+        g = sum(1 for x in level_layer if x <= l)
+        if g < len(levels):
+            lists.append(np.asarray(levels[g]["keep_idx"], dtype=np.int32))
+        else:
+            kept_vis = int(levels[-1]["S_out"]) - (S - n_vis0)      # visual tokens the last level left
+            lists.append(np.arange(S - n_vis0 + kept_vis, dtype=np.int32))
+    return lists
 
 
 # --------------------------------------------------------------------------- #

@@ -31,7 +31,7 @@ _vp, _i, _sz, _f, _d = _c.c_void_p, _c.c_int, _c.c_size_t, _c.c_float, _c.c_doub
 class VisionParams(_c.Structure):
     _fields_ = [("alpha", _d), ("event_agg", _i), ("mode", _i), ("keep_key", _d), ("keep_nonkey", _d),
                 ("beta", _d), ("s1", _i), ("s2", _i), ("s1_nonkey", _i), ("s2_nonkey", _i),
-                ("token_inv_norm", _vp), ("key_events_given", _vp)]
+                ("token_inv_norm", _vp), ("key_events_given", _vp), ("key_frames_given", _vp)]
 
 
 class PruneLevel(_c.Structure):
@@ -78,6 +78,7 @@ _SIGNATURES = {
     "metok_profile_read": (_i, [_c.c_char_p, _sz]),
     "metok_profile_end": (_i, [_c.c_char_p, _sz]),
     "metok_profile_scope": (_i, [_c.c_char_p]),
+    "metok_prune_schedule_kv_lists": (_i, [_vp, _i, _vp, _i, _i, _i, _d, _d, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "metok_debug_set": (_i, [_i, _i]),
     "metok_debug_build": (_i, []),
     "metok_status_string": (_c.c_char_p, [_i]),
@@ -231,7 +232,8 @@ def metok_segment_score_events(feats: torch.Tensor, k: int, text_emb: torch.Tens
 def vision_params(alpha: float, keep_key: float = 1.0, keep_nonkey: float = 1.0, event_agg: int = AGG_MEAN,
                   mode: int = MODE_TOPK_MERGE, beta: float = 0.5, s1: int = 2, s2: int = 3,
                   s1_nonkey: int = 4, s2_nonkey: int = 6) -> VisionParams:
-    return VisionParams(alpha, event_agg, mode, keep_key, keep_nonkey, beta, s1, s2, s1_nonkey, s2_nonkey, None, None)
+    return VisionParams(alpha, event_agg, mode, keep_key, keep_nonkey, beta, s1, s2, s1_nonkey, s2_nonkey, None, None,
+                        None)
 
 
 def metok_compress_vision_bound(T: int, N: int, k: int, p: VisionParams) -> int:
@@ -245,10 +247,11 @@ def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text
                           p: VisionParams, cap: Optional[int] = None,
                           out: Optional[Dict[str, torch.Tensor]] = None,
                           scored: Optional[Dict[str, torch.Tensor]] = None,
-                          key_events: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+                          key_events: Optional[torch.Tensor] = None,
+                          key_frames: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
     """`scored` (the result of metok_segment_score_events on the same feats and text) makes the call
     skip its own scoring pass over `feats`; `key_events` (uint8 [k] on the device) replaces the
-    call's own choice of key events."""
+    call's own choice of key events, `key_frames` (uint8 [T], mode POOL) that of key frames."""
     feats = _cuda_contig(feats, "feats")
     event_offsets = _cuda_contig(event_offsets, "event_offsets")
     text_emb = _cuda_contig(text_emb, "text_emb")
@@ -282,6 +285,12 @@ def metok_compress_vision(feats: torch.Tensor, event_offsets: torch.Tensor, text
             raise ValueError("key_events must be uint8 [k]")
         p = VisionParams.from_buffer_copy(p)
         p.key_events_given = key_events.data_ptr()
+    if key_frames is not None:
+        key_frames = _cuda_contig(key_frames, "key_frames")
+        if key_frames.dtype != torch.uint8 or key_frames.numel() != T:
+            raise ValueError("key_frames must be uint8 [T]")
+        p = VisionParams.from_buffer_copy(p)
+        p.key_frames_given = key_frames.data_ptr()
     need = L.metok_compress_vision_workspace_bytes(_dt(feats), T, N, d, k, cap, _c.byref(p))
     ws = workspace(need, dev)
     st = L.metok_compress_vision(_ptr(feats), _dt(feats), T, N, d, _ptr(event_offsets), k, _ptr(text_emb),
@@ -464,7 +473,25 @@ def metok_prefill_prune_schedule(q_texts: Sequence[torch.Tensor], k_alls: Sequen
     _check("metok_prefill_prune_schedule", st)
     for o in outs:
         o["status"] = status
+        o["_schedule"] = (arr, n_levels, S, n_vis, alpha, r, n0)
     return outs
+
+
+def metok_prune_schedule_kv_lists(levels: List[Dict[str, torch.Tensor]], level_layer: Sequence[int],
+                                  L: int) -> Dict[str, object]:
+    """K/V keep lists per layer from the keep lists recorded by metok_prefill_prune_schedule (its result is
+    `levels`): {"keep_idx": int32 [L, S], "keep_len": int32 [L], "S_cur": list of L ints}."""
+    arr, n_levels, S, n_vis, alpha, r, n0 = levels[0]["_schedule"]
+    dev = levels[0]["keep_idx"].device
+    keep_idx = torch.empty((L, S), dtype=torch.int32, device=dev)
+    keep_len = torch.zeros(L, dtype=torch.int32, device=dev)
+    s_cur = (_c.c_int32 * L)()
+    layers = (_c.c_int32 * n_levels)(*[int(v) for v in level_layer])
+    ws = workspace(4 * L, dev)
+    st = lib().metok_prune_schedule_kv_lists(arr, n_levels, layers, L, S, n_vis, alpha, r, n0, _ptr(keep_idx), _ptr(keep_len),
+                                             s_cur, _ptr(ws), ws.numel(), _stream())
+    _check("metok_prune_schedule_kv_lists", st)
+    return {"keep_idx": keep_idx, "keep_len": keep_len, "S_cur": [int(v) for v in s_cur]}
 
 
 def metok_kv_compact(k_layers: Sequence[torch.Tensor], v_layers: Sequence[torch.Tensor], S_cur: int, policy: int,

@@ -733,6 +733,64 @@ schedule_propagate_kernel(const int32_t* __restrict__ keep_idx, int vis_start, i
 
 }  // namespace metok
 
+namespace metok {
+struct KvListSrc { const int32_t* keep_idx[4]; const int32_t* S_out[4]; int S_in[4]; };   // per layer group
+// Layer l of group g (the pruning layers at or below it: g of them) holds the rows of level g's input;
+// its list is the keep list recorded by level g + 1, or everything when no level follows.
+__global__ void __launch_bounds__(256)
+schedule_kv_lists_kernel(KvListSrc src, const int32_t* __restrict__ layer_group, int stride,
+                         int32_t* __restrict__ kv_keep_idx, int32_t* __restrict__ kv_keep_len) {
+    const int layer = blockIdx.x;
+    const int g = layer_group[layer];
+    int32_t* out = kv_keep_idx + (size_t)layer * stride;
+    const int32_t* keep = src.keep_idx[g];
+    const int n = keep ? *src.S_out[g] : src.S_in[g];
+    for (int i = threadIdx.x; i < n; i += blockDim.x) out[i] = keep ? keep[i] : i;
+    if (threadIdx.x == 0) kv_keep_len[layer] = n;
+}
+}  // namespace metok
+
+extern "C" int metok_prune_schedule_kv_lists(const metok_prune_level* levels, int n_levels, const int32_t* level_layer,
+                                             int L, int S, int n_vis, double alpha, double r, const int32_t* N0,
+                                             int32_t* kv_keep_idx, int32_t* kv_keep_len, int32_t* kv_S_cur,
+                                             void* ws, size_t ws_bytes, void* stream) {
+    if (!levels || !level_layer || !N0 || !kv_keep_idx || !kv_keep_len || !kv_S_cur) return METOK_ERR_INVALID_ARG;
+    if (L < 1 || S < 1 || n_vis < 1 || n_vis > S) return METOK_ERR_INVALID_ARG;
+    int32_t sizes[4];
+    const int rc = metok_prune_schedule_sizes(n_levels, alpha, r, N0, sizes);
+    if (rc != METOK_OK) return rc;
+    if (sizes[0] != n_vis) return METOK_ERR_INVALID_ARG;
+    for (int s = 0; s < n_levels; ++s) {
+        if (!levels[s].keep_idx || !levels[s].S_out) return METOK_ERR_INVALID_ARG;
+        if (level_layer[s] < 0 || (s > 0 && level_layer[s] <= level_layer[s - 1])) return METOK_ERR_INVALID_ARG;
+    }
+    if (!ws || ws_bytes < (size_t)L * sizeof(int32_t) || !aligned16(ws)) return METOK_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    metok::KvListSrc src;
+    for (int g = 0; g < 4; ++g) {
+        src.keep_idx[g] = g < n_levels ? levels[g].keep_idx : nullptr;
+        src.S_out[g] = g < n_levels ? levels[g].S_out : nullptr;
+        src.S_in[g] = g <= n_levels ? S - n_vis + sizes[g] : 0;
+    }
+    // the group of every layer, known on the host
+    int32_t group_host[1024];
+    if (L > 1024) return METOK_ERR_UNSUPPORTED;
+    for (int l = 0; l < L; ++l) {
+        int g = 0;
+        while (g < n_levels && level_layer[g] <= l) ++g;
+        group_host[l] = g;
+        kv_S_cur[l] = src.S_in[g];
+    }
+    int32_t* group_dev = reinterpret_cast<int32_t*>(ws);
+    METOK_CUDA_TRY(cudaMemcpyAsync(group_dev, group_host, (size_t)L * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    {
+        METOK_TIMED("schedule_kv_lists_kernel", st);
+        metok::schedule_kv_lists_kernel<<<L, 256, 0, st>>>(src, group_dev, S, kv_keep_idx, kv_keep_len);
+    }
+    METOK_LAUNCH_CHECK();
+    return METOK_OK;
+}
+
 extern "C" int metok_prune_schedule_sizes(int n_levels, double alpha, double r, const int32_t* N0,
                                           int32_t* n_vis_of_level) {
     if (!N0 || !n_vis_of_level || n_levels < 1 || n_levels > 3) return METOK_ERR_INVALID_ARG;

@@ -114,6 +114,7 @@ struct PlanParams {
     int grid, s1, s2, s1_nonkey, s2_nonkey;     // POOL: side of the token grid and the four strides
     double keep_key, keep_nonkey, beta;
     const uint8_t* key_given;                   // the caller's key events, or null
+    const uint8_t* key_frames_given;            // POOL: the caller's key frames, or null
 };
 
 // The workspace regions that later kernels of the call expect cleared: written here, at the start of
@@ -278,7 +279,7 @@ event_plan_kernel(const float* __restrict__ token_score, float* __restrict__ fra
                 const float w = s_frame[j];
                 rank += (w > v) || (w == v && j < f);
             }
-            const bool key_frame = rank < (int)nk;
+            const bool key_frame = pp.key_frames_given ? pp.key_frames_given[f] != 0 : rank < (int)nk;
             frame_stride[f] = event_is_key[e] ? (key_frame ? pp.s1 : pp.s2) : (key_frame ? pp.s1_nonkey : pp.s2_nonkey);
         }
         __syncthreads();
@@ -1332,6 +1333,7 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
     pp.chunk_cols = kMmaBN;
     pp.keep_key = p->keep_key; pp.keep_nonkey = p->keep_nonkey; pp.beta = p->beta;
     pp.key_given = p->key_events_given;
+    pp.key_frames_given = p->key_frames_given;
     pp.grid = 1;
     while (pp.grid * pp.grid < N) ++pp.grid;
     pp.s1 = p->s1; pp.s2 = p->s2; pp.s1_nonkey = p->s1_nonkey; pp.s2_nonkey = p->s2_nonkey;

@@ -120,17 +120,18 @@ def compress_case(V: np.ndarray, t: np.ndarray, offs: np.ndarray, dtype: str, al
 
 
 def pool_case(V: np.ndarray, t: np.ndarray, offs: np.ndarray, dtype: str, alpha: float, beta: float,
-              strides: Sequence[int], event_agg: int = 0) -> Dict[str, object]:
+              strides: Sequence[int], event_agg: int = 0, key_frames: Optional[np.ndarray] = None) -> Dict[str, object]:
     """mode POOL (Algorithm 1) against the oracle's adaptive_pool.  Key frames are chosen by frame
     score: a frame whose score is within the near-tie band of its event's cut may flip, and then the
     layouts differ; everything the layout fixes is checked either way."""
     T, N, d = V.shape
     G = int(round(N ** 0.5))
-    want = O.adaptive_pool(V, t, offs, alpha, beta, strides, dtype, event_agg)
+    want = O.adaptive_pool(V, t, offs, alpha, beta, strides, dtype, event_agg, key_frames_given=key_frames)
     p = B.vision_params(alpha, event_agg=event_agg, mode=B.MODE_POOL, beta=beta, s1=strides[0], s2=strides[1],
                         s1_nonkey=strides[2], s2_nonkey=strides[3])
+    given = None if key_frames is None else torch.from_numpy(np.asarray(key_frames).astype(np.uint8)).cuda()
     got = B.metok_compress_vision(P.to_torch(V, dtype), torch.from_numpy(np.asarray(offs, dtype=np.int32)).cuda(),
-                                  P.to_torch(t, dtype), p)
+                                  P.to_torch(t, dtype), p, key_frames=given)
     torch.cuda.synchronize()
     rep: Dict[str, object] = {}
     P.check_scores(got["frame_score"].cpu().numpy(), want["frame_score"], dtype, "frame_score")

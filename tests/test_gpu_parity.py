@@ -607,6 +607,59 @@ def test_prefill_prune_schedule_three_levels_in_one_call(name):
         assert int(out[0]["status"].item()) == -1
 
 
+def test_kv_lists_from_the_recorded_keep_lists_and_their_compaction():
+    """The schedule's recorded keep lists as K/V lists per layer (metok_prune_schedule_kv_lists), equal to
+    the oracle's, and the caches of every layer group compacted with them (policy GIVEN) equal to the
+    oracle's gather."""
+    import dataclasses
+    cfg = dataclasses.replace(W.CONFIGS["frames32"], L=6)
+    vis = vis_of("frames32")
+    groups = W.token_groups(cfg, cfg.Nv, vis=vis)
+    N0 = [int((groups == 0).sum()), int((groups == 1).sum())]
+    r, layers = cfg.keep_prefill, [1, 3, 4]
+    sizes = B.metok_prune_schedule_sizes(3, cfg.alpha, r, N0)
+    Qs, Ks, g_s = [], [], groups
+    for s in range(1, 4):
+        pf = W.prefill_inputs(cfg, s, g_s.size, g_s)
+        Qs.append(pf["Q"]); Ks.append(pf["K"])
+        want_lv = O.prune_schedule(Qs, Ks, groups, cfg.alpha, r, 0, O.f32(cfg.dh ** -0.5))
+        k_ = want_lv[-1]["keep_idx"]
+        g_s = g_s[k_[k_ < g_s.size]]
+    S = cfg.Nv + cfg.Lt
+    got_lv = B.metok_prefill_prune_schedule([P.to_torch(q, cfg.dtype) for q in Qs], [P.to_torch(k_, cfg.dtype) for k_ in Ks],
+                                            None, 0, torch.from_numpy(groups.astype(np.int32)).cuda(), cfg.alpha, r, N0,
+                                            cfg.dh ** -0.5)
+    kv = B.metok_prune_schedule_kv_lists(got_lv, layers, cfg.L)
+    torch.cuda.synchronize()
+    want = O.schedule_kv_lists(want_lv, layers, cfg.L, S)
+    lens = kv["keep_len"].cpu().numpy()
+    same_lists = all(np.array_equal(got_lv[s]["keep_idx"][: int(got_lv[s]["S_out"].item())].cpu().numpy(), want_lv[s]["keep_idx"])
+                     for s in range(3))
+    for l in range(cfg.L):
+        grp = sum(1 for x in layers if x <= l)
+        assert kv["S_cur"][l] == S - cfg.Nv + sizes[grp]
+        assert lens[l] == want[l].size
+        if same_lists:                                       # (a near-tie may tip a level's list; the sizes hold either way)
+            assert np.array_equal(kv["keep_idx"][l, : lens[l]].cpu().numpy(), want[l]), l
+    # compaction per layer group with the lists as given ones
+    for grp_layers in ([0], [1, 2], [3], [4, 5]):
+        S_cur = kv["S_cur"][grp_layers[0]]
+        ks = [W.payload_torch(900 + l, cfg.Hkv * S_cur, cfg.dh, cfg.dtype, "cuda").view(cfg.Hkv, S_cur, cfg.dh) for l in grp_layers]
+        vs = [W.payload_torch(950 + l, cfg.Hkv * S_cur, cfg.dh, cfg.dtype, "cuda").view(cfg.Hkv, S_cur, cfg.dh) for l in grp_layers]
+        before = [(a.clone(), b.clone()) for a, b in zip(ks, vs)]
+        ki = torch.zeros((len(grp_layers), S_cur), dtype=torch.int32, device="cuda")
+        for j, l in enumerate(grp_layers):
+            ki[j, : lens[l]] = kv["keep_idx"][l, : lens[l]]
+        out = B.metok_kv_compact(ks, vs, S_cur, O.KV_GIVEN, 0, S_cur - cfg.Lt, keep_idx=ki,
+                                 keep_len=kv["keep_len"][grp_layers[0]: grp_layers[-1] + 1].clone())
+        torch.cuda.synchronize()
+        assert int(out["status"].item()) == 0
+        for j, l in enumerate(grp_layers):
+            idx = kv["keep_idx"][l, : lens[l]].long()
+            assert torch.equal(ks[j][:, : lens[l]].view(torch.int16), before[j][0][:, idx].view(torch.int16))
+            assert torch.equal(vs[j][:, : lens[l]].view(torch.int16), before[j][1][:, idx].view(torch.int16))
+
+
 def test_two_videos_on_two_streams_do_not_share_scratch():
     """Independent videos in flight on streams of their own (the benchmark's batch): each call takes
     its scratch per stream, so the results equal those of the same calls made one after the other."""
@@ -715,6 +768,19 @@ def test_head_sharded_call_at_world_size_one_equals_the_fused_call(name):
     assert n == want["S_out"]
     P.check_index_set(got["keep_idx"][:n].cpu().numpy(), want["keep_idx"],
                       lambda u: u < cfg.Nv and bool(want["near_tie"][u]), "keep_idx of the sharded call")
+
+
+def test_ablation_key_frames_given_by_the_caller():
+    """Randomly chosen key frames (the ablation of Algorithm 1's key-frame choice): the caller's mask
+    decides the strides; with a given mask no score can tip a frame, so the layout must match exactly."""
+    cfg = W.CONFIGS["frames32"]
+    vis = vis_of("frames32")
+    rng = np.random.default_rng(41)
+    given = (rng.random(cfg.T) < 0.4).astype(np.uint8)
+    rep = R.pool_case(vis["V"], vis["t"], vis["event_offsets"], cfg.dtype, cfg.alpha, 0.45, (2, 3, 4, 6), key_frames=given)
+    assert rep["stride_flips"] == 0 and rep["n_out"] > 0
+    base = R.pool_case(vis["V"], vis["t"], vis["event_offsets"], cfg.dtype, cfg.alpha, 0.45, (2, 3, 4, 6))
+    assert rep["n_out"] != base["n_out"]                      # the mask does change the layout
 
 
 def test_ablation_key_events_given_by_the_caller():

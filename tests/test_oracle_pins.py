@@ -699,3 +699,57 @@ def test_split_events_non_finite_similarity_ranks_last():
     out = O.segment_events(V, 3)
     assert np.isnan(out["sims"][2]) and np.isnan(out["sims"][3]) and np.isfinite(out["sims"][[0, 1, 4]]).all()
     assert not set(out["boundaries"].tolist()) & {2, 3}
+
+
+def test_given_key_frames_replace_the_scored_ones():
+    """The random-key-frame ablation of Algorithm 1: a caller's key-frame mask only changes which stride
+    a frame is pooled with (output sizes counted by hand), and the scored mask given back reproduces
+    the default."""
+    rng = np.random.default_rng(23)
+    T, G, d = 7, 6, 5
+    offs = np.array([0, 3, 7], dtype=np.int32)
+    V = rng.standard_normal((T, G * G, d))
+    t = rng.standard_normal(d)
+    strides = (1, 2, 3, 6)
+    base = O.adaptive_pool(V, t, offs, 0.5, 0.5, strides, "f32")
+    same = O.adaptive_pool(V, t, offs, 0.5, 0.5, strides, "f32", key_frames_given=base["frame_is_key"])
+    assert np.array_equal(base["out_feats"], same["out_feats"]) and np.array_equal(base["out_frame"], same["out_frame"])
+    given = np.array([1, 0, 0, 0, 0, 1, 1], dtype=np.uint8)
+    out = O.adaptive_pool(V, t, offs, 0.5, 0.5, strides, "f32", key_frames_given=given)
+    assert np.array_equal(out["frame_is_key"], given)
+    want_stride = [(strides[0] if given[f] else strides[1]) if out["event_is_key"][0 if f < 3 else 1]
+                   else (strides[2] if given[f] else strides[3]) for f in range(T)]
+    assert out["frame_stride"].tolist() == want_stride
+    assert out["n_out"] == sum((-(-G // s_)) ** 2 for s_ in want_stride)
+    assert np.array_equal(out["event_is_key"], base["event_is_key"])            # the events' classes do not change
+    f = 5                                                                       # a frame pooled with its given stride
+    lo = int(np.searchsorted(out["out_frame"], f))
+    assert np.allclose(out["out_feats_exact"][lo:lo + (-(-G // want_stride[f])) ** 2], O.pool2d(V[f], G, want_stride[f]))
+
+
+def test_schedule_kv_lists_by_construction():
+    """Layer groups and their lists, hand-built: 6 visual + 2 text positions, pruning layers 2 and 5 of 7."""
+    lv1 = {"keep_idx": np.array([0, 2, 3, 5, 6, 7], dtype=np.int32), "S_out": 6, "token_group": np.zeros(6, dtype=np.int32)}
+    lv2 = {"keep_idx": np.array([1, 4, 5], dtype=np.int32), "S_out": 3, "token_group": np.zeros(4, dtype=np.int32)}
+    lists = O.schedule_kv_lists([lv1, lv2], [2, 5], 7, 8)
+    assert [l.tolist() for l in lists[:2]] == [[0, 2, 3, 5, 6, 7]] * 2            # before the first pruning layer: what level 1 keeps
+    assert [l.tolist() for l in lists[2:5]] == [[1, 4, 5]] * 3                    # between the two: what level 2 keeps, in level 2's layout
+    assert [l.tolist() for l in lists[5:]] == [[0, 1, 2]] * 2                     # from the last pruning layer on: all rows that are left
+    # a real chain: every list is ascending, inside its layer's cache, and text positions always survive
+    rng = np.random.default_rng(8)
+    n_vis, Lt, Hq, dh = 40, 3, 2, 8
+    group = (rng.random(n_vis) < 0.5).astype(np.int32)
+    Qs, Ks, g = [], [], group
+    N0 = [int((group == 0).sum()), int((group == 1).sum())]
+    for s_ in range(1, 4):
+        Qs.append(rng.standard_normal((Hq, Lt, dh))); Ks.append(rng.standard_normal((1, g.size + Lt, dh)))
+        lv = O.prune_schedule(Qs, Ks, group, 0.5, 0.6, 0, 0.3)
+        k_ = lv[-1]["keep_idx"]
+        g = g[k_[k_ < g.size]]
+    lists = O.schedule_kv_lists(lv, [1, 2, 4], 6, n_vis + Lt)
+    sizes = [n_vis + Lt] + [int(x["S_out"]) for x in lv]
+    for l, lst in enumerate(lists):
+        grp = sum(1 for x in (1, 2, 4) if x <= l)
+        assert np.all(np.diff(lst) > 0) and lst[-1] < sizes[grp]
+        assert lst[-Lt:].tolist() == list(range(sizes[grp] - Lt, sizes[grp]))
+        assert lst.size == sizes[min(grp + 1, 3)]

@@ -368,8 +368,10 @@ extern "C" int metok_segment_events(const void* feats, int dtype, int T, int N, 
 // leaves an SM with 12 warps.  Here the rows land in shared memory by 16-byte
 // asynchronous copies (a ring of kFsDepth stages per warp, no registers held while in
 // flight) and the sums run on the tensor cores.  A warp owns one position and
-// EIGHT consecutive frames; a stage holds one 64-byte slice of those eight rows and of
-// the frame before them.  Lane (g, q) = (lane / 4, lane % 4) reads chunk q of frame g's
+// EIGHT consecutive frames; a stage holds 512 contiguous bytes of those eight rows and
+// of the frame before them (one copy instruction per row, 16 bytes per lane: the memory
+// system sees long pieces of a row).  A stage is consumed as eight 64-byte slices.  Lane
+// (g, q) = (lane / 4, lane % 4) reads chunk q of frame g's
 // slice: the 16 bytes, as they lie in memory (dwords m0..m3), are the A operand of
 // m16n8k16 mma, which gives row g of A the k-slots (m0, m2) and row 8 + g the slots
 // (m1, m3).  The other vector is the B operand, whose two registers pair with (m0, m2)
@@ -379,7 +381,7 @@ extern "C" int metok_segment_events(const void* feats, int dtype, int T, int N, 
 // is free as long as both operands use the same one.  Two mma per slice and vector pair,
 // accumulated over the slices of the row: at the end the lane that holds C[g][g] has the
 // complete sum of frame g, with no shuffle and no widening.  The previous frame's slice
-// is the neighbouring 64 bytes of the same stage.  Products of bf16 are exact in fp32 and
+// is the same slice of the row before it in the stage.  Products of bf16 are exact in fp32 and
 // the sums are fp32; the off-diagonal entries are never read.
 // --------------------------------------------------------------------------- //
 namespace metok {
@@ -494,14 +496,16 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-constexpr int kFsDepth = 16;                       // stages of a warp's ring
+constexpr int kFsDepth = 4;                        // stages of a warp's ring
 constexpr int kFsFrames = 8;                       // frames per warp = row groups of the mma tile
-constexpr int kFsStageBytes = (kFsFrames + 1) * 64;
+constexpr int kFsSlices = 8;                       // 64-byte slices of a row per stage: 512 contiguous bytes
+constexpr int kFsRowPitch = kFsSlices * 64 + 64;   // bytes between a stage's rows (see the bank note in the kernel)
+constexpr int kFsStageBytes = (kFsFrames + 1) * kFsRowPitch;
 
 // Shared memory: the text embedding as 16-byte chunks with the dwords in the order
-// (0, 2, 1, 3), zero-padded to whole slices; then per warp kFsDepth stages of 9 x 64 bytes
-// (slice of frame f0 - 1, then of frames f0 .. f0 + 7).
-template <bool kFull>                               // kFull: the row is a whole number of 64-byte slices
+// (0, 2, 1, 3), zero-padded to whole slices; then per warp kFsDepth stages of nine rows
+// (512 bytes of frame f0 - 1, then of frames f0 .. f0 + 7).
+template <bool kFull>                               // kFull: the row is a whole number of 512-byte pieces
 __global__ void __launch_bounds__(kFsThreads)
 seg_score_mma_kernel(const __nv_bfloat16* __restrict__ feats, const __nv_bfloat16* __restrict__ text, int Tn, int N,
                      int d, float* __restrict__ part_dot, float* __restrict__ part_nrm,
@@ -548,23 +552,30 @@ seg_score_mma_kernel(const __nv_bfloat16* __restrict__ feats, const __nv_bfloat1
     const int g = lane >> 2, q = lane & 3;
     const int f = f0 + g;                                   // this lane's frame
     const bool has_f = f < Tn;
-    const bool halo = g == 0 && f0 > 0;                     // lanes 0..3 also fetch frame f0 - 1
-    // chunk q of slice 0 of this lane's row, and of the row before the run (a valid address even if unused)
-    const uint4* src = reinterpret_cast<const uint4*>(feats) + ((size_t)(has_f ? f : 0) * N + p) * (size_t)nchunk + q;
-    const uint4* src_h = reinterpret_cast<const uint4*>(feats) + ((size_t)(halo ? f0 - 1 : 0) * N + p) * (size_t)nchunk + q;
-    const uint32_t sz = has_f ? 16u : 0u, sz_h = halo ? 16u : 0u;      // 0 bytes read = zeros written
+    // Copies: a stage holds 512 contiguous bytes (eight 64-byte slices) of each of the nine rows -- the
+    // frame before the run, then the run's eight frames.  One copy instruction moves a row's 512 bytes
+    // (16 per lane), so what reaches the memory system is long contiguous pieces of a row.  Rows of a
+    // stage lie kFsRowPitch bytes apart: with 16 words more than a multiple of 32 the 16-byte reads of
+    // the eight lanes of a quarter warp (two frames, four chunks each) fall into different banks.
+    const uint4* row0 = reinterpret_cast<const uint4*>(feats) + ((size_t)max(f0 - 1, 0) * N + p) * (size_t)nchunk;
+    const size_t frame_pitch = (size_t)N * nchunk;          // 16-byte chunks from a frame's row to the next frame's
+    const int nsuper = (nslice + kFsSlices - 1) / kFsSlices;
     unsigned char* ring = s_dyn + (size_t)nslice * 4 * sizeof(uint4) + (size_t)warp * kFsDepth * kFsStageBytes;
-    const unsigned char* mine = ring + (g + 1) * 64 + q * 16;
-    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + (uint32_t)((g + 1) * 64 + q * 16);
-    const uint32_t dst_h = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + (uint32_t)(q * 16);
+    const unsigned char* mine = ring + (g + 1) * kFsRowPitch + q * 16;
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + (uint32_t)lane * 16u;
     const uint4* tq = s_text + q;
-    // slice sl into stage `stage` (a constant where the caller is unrolled); one group per call
-    auto issue = [&](int sl, int stage) {
-        if (sl < nslice) {
-            const bool in = kFull || sl * 4 + q < nchunk;
-            const int o = in ? sl * 4 : 0;
-            cp_async16(dst + stage * kFsStageBytes, src + o, in ? sz : 0u);
-            if (g == 0) cp_async16(dst_h + stage * kFsStageBytes, src_h + o, in ? sz_h : 0u);
+    // 512-byte piece `sup` of the nine rows into stage `stage` (a constant where the caller is unrolled); one group per call
+    auto issue = [&](int sup, int stage) {
+        if (sup < nsuper) {
+            const int c = sup * 32 + lane;                  // this lane's chunk of every row
+            const bool in = c < nchunk;
+#pragma unroll
+            for (int r = 0; r <= kFsFrames; ++r) {
+                const int fr = f0 - 1 + r;                  // r = 0: the frame before the run
+                const bool ok = in && fr >= 0 && fr < Tn;
+                const uint4* src = ok ? row0 + (size_t)(fr - max(f0 - 1, 0)) * frame_pitch + c : row0;
+                cp_async16(dst + stage * kFsStageBytes + r * kFsRowPitch, src, ok ? 16u : 0u);   // 0 bytes read = zeros written
+            }
         }
         cp_async_commit();
     };
@@ -575,24 +586,30 @@ seg_score_mma_kernel(const __nv_bfloat16* __restrict__ feats, const __nv_bfloat1
     float cp[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     float ct[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll 1
-    for (int base = 0; base < nslice; base += kFsDepth) {
+    for (int base = 0; base < nsuper; base += kFsDepth) {
 #pragma unroll
         for (int j = 0; j < kFsDepth; ++j) {
-            const int sl = base + j;
-            if (sl < nslice) {                              // the same for the whole warp
-                cp_async_wait<kFsDepth - 2>();              // this lane's copies of slice sl have landed
-                __syncwarp();                               // ... and every lane's; slice sl - 1 is read by all
-                issue(sl + kFsDepth - 1, (j + kFsDepth - 1) % kFsDepth);      // into the stage that held slice sl - 1
-                const uint4 x = *reinterpret_cast<const uint4*>(mine + j * kFsStageBytes);
-                const uint4 pv = *reinterpret_cast<const uint4*>(mine + j * kFsStageBytes - 64);
-                const uint4 tt = tq[sl * 4];
-                const uint4 xs = make_uint4(x.x, x.z, x.y, x.w);
-                mma_bf16_m16n8k16(cn[0], x, xs.x, xs.y);
-                mma_bf16_m16n8k16(cn[1], x, xs.z, xs.w);
-                mma_bf16_m16n8k16(cp[0], pv, xs.x, xs.y);
-                mma_bf16_m16n8k16(cp[1], pv, xs.z, xs.w);
-                mma_bf16_m16n8k16(ct[0], x, tt.x, tt.y);
-                mma_bf16_m16n8k16(ct[1], x, tt.z, tt.w);
+            const int sup = base + j;
+            if (sup < nsuper) {                             // the same for the whole warp
+                cp_async_wait<kFsDepth - 2>();              // this lane's copies of the piece have landed
+                __syncwarp();                               // ... and every lane's; the piece before it has been read by all
+                issue(sup + kFsDepth - 1, (j + kFsDepth - 1) % kFsDepth);     // into the stage that held the piece before
+#pragma unroll
+                for (int i = 0; i < kFsSlices; ++i) {
+                    const int sl = sup * kFsSlices + i;
+                    if (kFull || sl < nslice) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(mine + j * kFsStageBytes + i * 64);
+                        const uint4 pv = *reinterpret_cast<const uint4*>(mine + j * kFsStageBytes + i * 64 - kFsRowPitch);
+                        const uint4 tt = tq[sl * 4];
+                        const uint4 xs = make_uint4(x.x, x.z, x.y, x.w);
+                        mma_bf16_m16n8k16(cn[0], x, xs.x, xs.y);
+                        mma_bf16_m16n8k16(cn[1], x, xs.z, xs.w);
+                        mma_bf16_m16n8k16(cp[0], pv, xs.x, xs.y);
+                        mma_bf16_m16n8k16(cp[1], pv, xs.z, xs.w);
+                        mma_bf16_m16n8k16(ct[0], x, tt.x, tt.y);
+                        mma_bf16_m16n8k16(ct[1], x, tt.z, tt.w);
+                    }
+                }
             }
         }
     }
@@ -651,7 +668,7 @@ static int launch_seg_score(const void* feats, const void* text, int Tn, int N, 
     if constexpr (sizeof(T) == 2) {
         const int nslice = (d / 8 + 3) / 4;
         const size_t smem_t = (size_t)nslice * 4 * sizeof(uint4) + (size_t)(kFsThreads / 32) * kFsDepth * kFsStageBytes;
-        auto kernel = (d / 8) % 4 == 0 ? seg_score_mma_kernel<true> : seg_score_mma_kernel<false>;
+        auto kernel = (d / 8) % (4 * kFsSlices) == 0 ? seg_score_mma_kernel<true> : seg_score_mma_kernel<false>;
         if (smem_t > 40 * 1024)
             METOK_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_t));
         nslab = ceil_div(N, kFsThreads / 32);              // the kernel adds the four positions of a CTA

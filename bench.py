@@ -550,6 +550,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph of the step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the chained run and the run without planted relevance")
+    ap.add_argument("--no-sustain", action="store_true",
+                    help="time exactly --steps steps (for profiler captures, where a one-second region is thousands of launches)")
     ap.add_argument("--videos", type=int, default=4,
                     help="independent videos in flight per step, each on a stream of its own (a step = this batch)")
     ap.add_argument("--parts", default=",".join(PARTS),
@@ -662,7 +664,7 @@ def main():
     burst_ms = timed(run_batch, args.steps) / args.steps
     # ... and the sustained figure: as many steps as fill at least a second (and no fewer than --steps),
     # the clocks sampled meanwhile; `value` is this one, whatever --steps was
-    sustain_steps = max(args.steps, int(math.ceil(1000.0 / max(burst_ms, 1e-3))))
+    sustain_steps = args.steps if args.no_sustain else max(args.steps, int(math.ceil(1000.0 / max(burst_ms, 1e-3))))
     sampler = ClockSampler(local)
     sampler.start()
     total_ms = timed(run_batch, sustain_steps)

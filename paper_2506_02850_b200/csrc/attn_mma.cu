@@ -33,20 +33,10 @@ constexpr int kStEpiWarps = 16;           // stats: four warps per TMEM lane qua
 constexpr int kStThreads = 64 + kStEpiWarps * 32;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegInf = -3.0e38f;       // finite stand-in: keeps (m_old - m_new) free of inf - inf
-// The exponentials of both passes are taken two at a time in half precision (exp2_sum8).  Their
-// arguments are shifted by kExpShift: a probability of 2^-13 then has the argument 0, so the ones
-// that matter among the ~16 K keys a query sees lie where a half resolves an argument to 1e-3 or
-// better; sums of four terms stay below the largest half (4 * 2^13 < 65504); results down to 2^-37
-// of a row's total are still represented.  The sums are scaled back by kExpUnshift.  In the first
-// pass the argument is relative to the running maximum, so the terms that make up the sum are the
-// ones near the shift itself.  Each term carries a relative rounding of about 2e-4; a score is the
-// mean of Hq * Lt rows of them.
-constexpr float kExpShift = 13.0f, kExpUnshift = 0.0001220703125f;
 
 constexpr int kStBM = 128;                // stats: query rows per CTA
-constexpr int kStBN = 256;                // stats: keys per tile (one accumulator)
-constexpr int kStHalf = 128;              // ... brought in as two stages of this many keys: more, smaller copies in flight
-constexpr int kStStages = 5;
+constexpr int kStBN = 256;                // stats: keys per tile
+constexpr int kStStages = 2;
 constexpr int kCsBM = 128;                // colsum: keys per tile
 constexpr int kCsMaxNQ = 256;             // colsum: query rows per chunk (multiple of 16)
 constexpr int kCsStages = 4;
@@ -100,8 +90,8 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     grid_dep_wait();
     using namespace sm100;
     constexpr int KB = DH / 64;                               // 64-element (128-byte) K blocks
-    constexpr uint32_t kQBlk = kStBM * 128, kKBlk = kStHalf * 128;
-    constexpr uint32_t kQBytes = KB * kQBlk, kKBytes = KB * kKBlk;       // a stage: kStHalf keys
+    constexpr uint32_t kQBlk = kStBM * 128, kKBlk = kStBN * 128;
+    constexpr uint32_t kQBytes = KB * kQBlk, kKBytes = KB * kKBlk;
     extern __shared__ uint8_t smem_dyn[];
     __shared__ __align__(8) uint64_t q_bar, drain_bar, full_bar[kStStages], empty_bar[kStStages], tfull_bar[2],
         tempty_bar[2];
@@ -149,9 +139,9 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb)
                 tma_load_2d(q_addr + kb * kQBlk, &tmQ, kb * 64, g * dm.R + rt * kStBM, smem_u32(&q_bar));
-            int it = 0;                                        // stages issued: two per tile
+            int it = 0;
             bool ok = true;
-            for (; it < 2 * nt; ++it) {
+            for (; it < nt; ++it) {
                 const int s = it % kStStages;
                 const uint32_t ph = (uint32_t)(it / kStStages) & 1u;
                 if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -160,7 +150,7 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 if (dbg_withhold(status, kDbgAttnStats) && split == 0 && rt == 0 && g == 0 && it == 0) continue;   // debug builds: one copy never sent
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
-                    tma_load_2d(k_addr(s) + kb * kKBlk, &tmK, kb * 64, g * dm.S + (t_lo + (it >> 1)) * kStBN + (it & 1) * kStHalf, fb);
+                    tma_load_2d(k_addr(s) + kb * kKBlk, &tmK, kb * 64, g * dm.S + (t_lo + it) * kStBN, fb);
             }
             if (!ok) {
                 // let the copies already issued land before the CTA's shared memory goes away
@@ -173,26 +163,22 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(kStBM, kStHalf);
+            constexpr uint32_t idesc = make_idesc_bf16(kStBM, kStBN);
             bool ok = mbar_wait(smem_u32(&q_bar), 0u, abort_flag);
-            int st = 0;                                        // stages consumed
             for (int it = 0; it < nt && ok; ++it) {
-                const int b = it & 1;
+                const int b = it & 1, s = it % kStStages;
                 if (!mbar_wait(smem_u32(&tempty_bar[b]), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-                for (int h = 0; h < 2 && ok; ++h, ++st) {      // the tile's two key halves: columns h * kStHalf ...
-                    const int s = st % kStStages;
-                    if (!mbar_wait(smem_u32(&full_bar[s]), (uint32_t)(st / kStStages) & 1u, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(b * kStBN + h * kStHalf);
+                if (!mbar_wait(smem_u32(&full_bar[s]), (uint32_t)(it / kStStages) & 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)b * kStBN;
 #pragma unroll
-                    for (int kk = 0; kk < DH / 16; ++kk) {
-                        const uint64_t ad = make_desc_k128(q_addr + (kk >> 2) * kQBlk + (kk & 3) * 32);
-                        const uint64_t bd = make_desc_k128(k_addr(s) + (kk >> 2) * kKBlk + (kk & 3) * 32);
-                        umma_bf16(d_tmem, ad, bd, idesc, kk != 0 ? 1u : 0u);
-                    }
-                    umma_commit(smem_u32(&empty_bar[s]));
+                for (int kk = 0; kk < DH / 16; ++kk) {
+                    const uint64_t ad = make_desc_k128(q_addr + (kk >> 2) * kQBlk + (kk & 3) * 32);
+                    const uint64_t bd = make_desc_k128(k_addr(s) + (kk >> 2) * kKBlk + (kk & 3) * 32);
+                    umma_bf16(d_tmem, ad, bd, idesc, kk != 0 ? 1u : 0u);
                 }
-                if (ok) umma_commit(smem_u32(&tfull_bar[b]));
+                umma_commit(smem_u32(&empty_bar[s]));
+                umma_commit(smem_u32(&tfull_bar[b]));
             }
             if (!ok) {                                         // wait until whatever was issued has retired
                 umma_commit(smem_u32(&drain_bar));
@@ -253,19 +239,14 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     }
                     const float cm = t16[0];
                     m_new = fmaxf(m_run, cm * sc);
-                    // 2^(logit - max + kExpShift) two per special-function instruction, in half precision:
-                    // the terms that make up the sum have arguments near kExpShift, where a half is exact to
-                    // 1e-3 or better, and the sum is of thousands of them; the shift is taken out below
-                    const float neg_m = kExpShift - m_new;
+                    const float neg_m = -m_new;
 #pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        float x[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) x[i] = fmaf(v[j + i], sc, neg_m);
-                        if (j & 8) a1 += exp2_sum8(x); else a0 += exp2_sum8(x);
+                    for (int j = 0; j < 32; j += 4) {           // every fourth exponential on the FMA pipe
+                        a0 += fast_exp2(fmaf(v[j], sc, neg_m));
+                        a1 += fast_exp2(fmaf(v[j + 1], sc, neg_m));
+                        a0 += fast_exp2(fmaf(v[j + 2], sc, neg_m));
+                        a1 += exp2_fma(fmaf(v[j + 3], sc, neg_m));
                     }
-                    a0 *= kExpUnshift;
-                    a1 *= kExpUnshift;
                 }
                 l_run = l_run * fast_exp2(m_run - m_new) + (a0 + a1);
                 m_run = m_new;
@@ -428,7 +409,7 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         M = Mn;
                     }
                 }
-                nl = kExpShift - (M + log2f(Z));                  // with the shift of the half-precision exponentials
+                nl = -(M + log2f(Z));
             }
             s_nlse[c] = nl;
             asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -448,44 +429,38 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * kCsMaxNQ);
-            // 16 columns at a time (the halves are multiples of 16), the next 16 fetched from tensor memory
-            // while these are reduced: a load the thread waited for each time was what a tile's time was
             float a0 = 0.f, a1 = 0.f;
-            const int nch = (c_hi - c_lo) >> 4;
-            uint32_t raw[2][16];
-            auto reduce16 = [&](const uint32_t (&r)[16], int c) {
-                const float4 n0 = *reinterpret_cast<const float4*>(&s_nlse[c]);
-                const float4 n1 = *reinterpret_cast<const float4*>(&s_nlse[c + 4]);
-                const float4 n2 = *reinterpret_cast<const float4*>(&s_nlse[c + 8]);
-                const float4 n3 = *reinterpret_cast<const float4*>(&s_nlse[c + 12]);
-                const float x0[8] = {fmaf(__uint_as_float(r[0]), sc, n0.x), fmaf(__uint_as_float(r[1]), sc, n0.y),
-                                     fmaf(__uint_as_float(r[2]), sc, n0.z), fmaf(__uint_as_float(r[3]), sc, n0.w),
-                                     fmaf(__uint_as_float(r[4]), sc, n1.x), fmaf(__uint_as_float(r[5]), sc, n1.y),
-                                     fmaf(__uint_as_float(r[6]), sc, n1.z), fmaf(__uint_as_float(r[7]), sc, n1.w)};
-                const float x1[8] = {fmaf(__uint_as_float(r[8]), sc, n2.x), fmaf(__uint_as_float(r[9]), sc, n2.y),
-                                     fmaf(__uint_as_float(r[10]), sc, n2.z), fmaf(__uint_as_float(r[11]), sc, n2.w),
-                                     fmaf(__uint_as_float(r[12]), sc, n3.x), fmaf(__uint_as_float(r[13]), sc, n3.y),
-                                     fmaf(__uint_as_float(r[14]), sc, n3.z), fmaf(__uint_as_float(r[15]), sc, n3.w)};
-                a0 += exp2_sum8(x0);
-                a1 += exp2_sum8(x1);
-            };
-            if (nch > 0) tmem_ld16_issue(taddr + (uint32_t)c_lo, raw[0]);
+            int c = c_lo;
 #pragma unroll 1
-            for (int i = 0; i < nch; i += 2) {
-                tmem_ld16_wait(raw[0]);
-                if (i + 1 < nch) tmem_ld16_issue(taddr + (uint32_t)(c_lo + 16 * (i + 1)), raw[1]);
-                reduce16(raw[0], c_lo + 16 * i);
-                if (i + 1 < nch) {
-                    tmem_ld16_wait(raw[1]);
-                    if (i + 2 < nch) tmem_ld16_issue(taddr + (uint32_t)(c_lo + 16 * (i + 2)), raw[0]);
-                    reduce16(raw[1], c_lo + 16 * (i + 1));
+            for (; c + 32 <= c_hi; c += 32) {
+                float v[32];
+                tmem_ld32(taddr + (uint32_t)c, v);
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float4 nl = *reinterpret_cast<const float4*>(&s_nlse[c + j]);
+                    a0 += fast_exp2(fmaf(v[j], sc, nl.x));
+                    a1 += fast_exp2(fmaf(v[j + 1], sc, nl.y));
+                    a0 += fast_exp2(fmaf(v[j + 2], sc, nl.z));
+                    a1 += exp2_fma(fmaf(v[j + 3], sc, nl.w));     // every fourth exponential on the FMA pipe
+                }
+            }
+            if (c < c_hi) {                                    // halves are multiples of 16 columns
+                float v[16];
+                tmem_ld16(taddr + (uint32_t)c, v);
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) {
+                    const float4 nl = *reinterpret_cast<const float4*>(&s_nlse[c + j]);
+                    a0 += fast_exp2(fmaf(v[j], sc, nl.x));
+                    a1 += fast_exp2(fmaf(v[j + 1], sc, nl.y));
+                    a0 += fast_exp2(fmaf(v[j + 2], sc, nl.z));
+                    a1 += exp2_fma(fmaf(v[j + 3], sc, nl.w));     // every fourth exponential on the FMA pipe
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[b]));
             const int u = (t_lo + it) * kCsBM + quad * 32 + lane;
-            if (u >= dm.vis_start && u < vis_end) plane[u - dm.vis_start] = (a0 + a1) * kExpUnshift;
+            if (u >= dm.vis_start && u < vis_end) plane[u - dm.vis_start] = a0 + a1;
         }
     }
     tc_fence_before();
@@ -501,11 +476,11 @@ int launch_dh(const void* q_text, const void* k_all, const AttnMmaDims& dm, floa
     const uint64_t qrows = (uint64_t)dm.Hq * dm.Lt, krows = (uint64_t)dm.Hkv * dm.S;
     int rc;
     if ((rc = make_tmap_bf16_2d(&tmQs, q_text, qrows, DH, kStBM)) != METOK_OK) return rc;
-    if ((rc = make_tmap_bf16_2d(&tmKs, k_all, krows, DH, kStHalf)) != METOK_OK) return rc;
+    if ((rc = make_tmap_bf16_2d(&tmKs, k_all, krows, DH, kStBN)) != METOK_OK) return rc;
     if ((rc = make_tmap_bf16_2d(&tmQc, q_text, qrows, DH, (uint32_t)dm.cs_nq)) != METOK_OK) return rc;
     if ((rc = make_tmap_bf16_2d(&tmKc, k_all, krows, DH, kCsBM)) != METOK_OK) return rc;
     constexpr int KB = DH / 64;
-    const size_t smem_st = (size_t)KB * (kStBM + kStStages * kStHalf) * 128 + 1024;
+    const size_t smem_st = (size_t)KB * (kStBM + kStStages * kStBN) * 128 + 1024;
     const size_t smem_cs = (size_t)KB * (dm.cs_nq + kCsStages * kCsBM) * 128 + 1024;
     METOK_CUDA_TRY(cudaFuncSetAttribute(attn_stats_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)smem_st));

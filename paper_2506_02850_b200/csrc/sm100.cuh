@@ -214,25 +214,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// The 16-column load split in two like the 32-column one.
-__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld16_wait(uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.wait::ld.sync.aligned;"
-        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-        :
-        : "memory");
-}
-
 // 2^x on the special-function unit (about 2 ulp; results below 2^-126 flush to zero).
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -254,39 +235,6 @@ __device__ __forceinline__ float exp2_fma(float x) {
     p = fmaf(p, f, 0.6931470036506653f);
     p = fmaf(p, f, 1.0f);
     return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
-
-// Two exponentials per special-function instruction: 2^a and 2^b for a pair of arguments packed as
-// half precision (11-bit significand: the arguments should be small in magnitude where the result
-// matters; results below 2^-24 are zero, above 65504 infinite).  pack_half2 rounds to nearest.
-__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-__device__ __forceinline__ uint32_t exp2_half2(uint32_t x) {
-    uint32_t y;
-    asm("ex2.approx.f16x2 %0, %1;" : "=r"(y) : "r"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t add_half2(uint32_t a, uint32_t b) {
-    uint32_t y;
-    asm("add.rn.f16x2 %0, %1, %2;" : "=r"(y) : "r"(a), "r"(b));
-    return y;
-}
-// lo + hi of a packed pair, as fp32
-__device__ __forceinline__ float sum_half2(uint32_t x) {
-    float lo, hi;
-    asm("{\n\t.reg .f16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}"
-        : "=f"(lo), "=f"(hi) : "r"(x));
-    return lo + hi;
-}
-// sum over eight arguments of 2^x: four packed exponentials, added pairwise in half precision (sums of
-// at most four terms), then widened
-__device__ __forceinline__ float exp2_sum8(const float (&x)[8]) {
-    const uint32_t e0 = exp2_half2(pack_half2(x[0], x[1])), e1 = exp2_half2(pack_half2(x[2], x[3]));
-    const uint32_t e2 = exp2_half2(pack_half2(x[4], x[5])), e3 = exp2_half2(pack_half2(x[6], x[7]));
-    return sum_half2(add_half2(add_half2(e0, e1), add_half2(e2, e3)));
 }
 
 // Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes

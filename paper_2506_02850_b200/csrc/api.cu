@@ -136,7 +136,9 @@ extern "C" int metok_profile_read(char* out, size_t cap) { return profile_collec
 extern "C" int metok_profile_end(char* out, size_t cap) { return profile_collect(out, cap, true); }
 
 namespace metok {
+#if defined(METOK_DEBUG_SHORT_WAIT) || defined(METOK_DEBUG_BOUNDS)
 static int g_dbg_withhold = 0;
+#endif
 int debug_arm(int32_t* status, cudaStream_t st) {
 #if defined(METOK_DEBUG_SHORT_WAIT) || defined(METOK_DEBUG_BOUNDS)
     const int32_t words[2] = {g_dbg_withhold, 0};

@@ -148,6 +148,7 @@ class Workload:
         self.kv_scores = torch.from_numpy(W.kv_scores(cfg, cfg.Nv)).to(device)
         self.out = {}
         self.side = None
+        self.up = self.down = self.consumed = None     # copy streams of the host-buffer step
         self.scale = float(cfg.dh ** -0.5)
 
     def twin(self):
@@ -161,10 +162,31 @@ class Workload:
         w.ks, w.vs = [x.clone() for x in self.ks], [x.clone() for x in self.vs]
         w.kv_scores = self.kv_scores.clone()
         w.out, w.side, w.h = {}, None, {}
+        w.up = w.down = w.consumed = None
         return w
 
     # one pass of the hot path, device-resident inputs
     def step(self):
+        self._segment_compress()
+        # The K/V lists need the first level's scores only: the compaction runs on a second stream
+        # beside pruning levels 2 and 3 and joins at the end of the step.
+        main = torch.cuda.current_stream()
+        if self.side is None:
+            self.side = torch.cuda.Stream()
+        forked = False
+        for i in range(len(self.stages)):
+            self._prefill_level(i)
+            if i == 0 and "kv" in self.parts:
+                self.side.wait_stream(main)
+                with torch.cuda.stream(self.side):
+                    self._kv_call()
+                forked = True
+        if "kv" in self.parts and not forked:
+            self._kv_call()
+        if forked:
+            main.wait_stream(self.side)
+
+    def _segment_compress(self):
         B, cfg, o = self.B, self.cfg, self.out
         # the text embedding is known before the video is segmented: segmentation and the Eq. 5
         # token scores share one pass over V, and the compressor takes the scores from there
@@ -176,25 +198,12 @@ class Workload:
             offs = o["seg"]["event_offsets"] if "seg" in o else self.planted_offsets
             o["cv"] = B.metok_compress_vision(self.V, offs, self.t, self.params, out=o.get("cv"),
                                               scored=o.get("seg"))
-        # The K/V lists need the first level's scores only: the compaction runs on a second stream
-        # beside pruning levels 2 and 3 and joins at the end of the step.
-        main = torch.cuda.current_stream()
-        if self.side is None:
-            self.side = torch.cuda.Stream()
-        forked = False
-        for i, s in enumerate(self.stages):
-            B.metok_profile_scope(f"prefill{i + 1}")
-            o[f"pf{i}"] = B.metok_prefill_prune(s["Q"], s["K"], s["hidden"], 0, s["n_vis"], s["groups"], s["budgets"],
-                                                self.scale, out=o.get(f"pf{i}"))
-            if i == 0 and "kv" in self.parts:
-                self.side.wait_stream(main)
-                with torch.cuda.stream(self.side):
-                    self._kv_call()
-                forked = True
-        if "kv" in self.parts and not forked:
-            self._kv_call()
-        if forked:
-            main.wait_stream(self.side)
+
+    def _prefill_level(self, i):
+        B, o, s = self.B, self.out, self.stages[i]
+        B.metok_profile_scope(f"prefill{i + 1}")
+        o[f"pf{i}"] = B.metok_prefill_prune(s["Q"], s["K"], s["hidden"], 0, s["n_vis"], s["groups"], s["budgets"],
+                                            self.scale, out=o.get(f"pf{i}"))
 
     def _kv_call(self):
         B, cfg, o = self.B, self.cfg, self.out
@@ -235,28 +244,61 @@ class Workload:
         return h2d, d2h
 
     def e2e_step(self):
+        """Host buffers in, host buffers out.  The uploads run on a copy stream in the order the calls need
+        them (frames and text, the pruning levels' inputs, the K/V cache last), each call starts when its
+        inputs have landed, and every result goes back on a second copy stream as soon as its call is done:
+        the downloads of everything but the compacted cache overlap the upload of the cache."""
         h, o = self.h, self.out
-        self.V.copy_(h["V"], non_blocking=True)
-        self.t.copy_(h["t"], non_blocking=True)
-        for i, s in enumerate(self.stages, start=1):
-            s["Q"].copy_(h[f"Q{i}"], non_blocking=True)
-            s["K"].copy_(h[f"K{i}"], non_blocking=True)
-            s["hidden"].copy_(h[f"hidden{i}"], non_blocking=True)
-            s["groups"].copy_(h[f"groups{i}"], non_blocking=True)
-        for d, s in zip(self.ks, h["ks"]):
-            d.copy_(s, non_blocking=True)
-        for d, s in zip(self.vs, h["vs"]):
-            d.copy_(s, non_blocking=True)
-        self.step()
-        self.d2h["out_feats"].copy_(o["cv"]["out_feats"][: self.n_out], non_blocking=True)
-        self.d2h["out_src"].copy_(o["cv"]["out_src"][: self.n_out], non_blocking=True)
-        self.d2h["offsets"].copy_(o["seg"]["event_offsets"], non_blocking=True)
+        cur = torch.cuda.current_stream()
+        if self.up is None:
+            self.up, self.down = torch.cuda.Stream(), torch.cuda.Stream()
+        up, down = self.up, self.down
+        # the step before has consumed its inputs; its last downloads (the compacted cache) may still run
+        # beside this step's first uploads
+        if self.consumed is None:
+            up.wait_stream(cur)
+        else:
+            up.wait_event(self.consumed)
+        ev = {}
+        with torch.cuda.stream(up):
+            self.V.copy_(h["V"], non_blocking=True)
+            self.t.copy_(h["t"], non_blocking=True)
+            ev["vision"] = up.record_event()
+            for i, s in enumerate(self.stages, start=1):
+                s["Q"].copy_(h[f"Q{i}"], non_blocking=True)
+                s["K"].copy_(h[f"K{i}"], non_blocking=True)
+                s["hidden"].copy_(h[f"hidden{i}"], non_blocking=True)
+                s["groups"].copy_(h[f"groups{i}"], non_blocking=True)
+                ev[i] = up.record_event()
+            up.wait_stream(down)              # the cache buffers hold the last step's result until it is on the host
+            for d, s in zip(self.ks, h["ks"]):
+                d.copy_(s, non_blocking=True)
+            for d, s in zip(self.vs, h["vs"]):
+                d.copy_(s, non_blocking=True)
+            ev["kv"] = up.record_event()
+        cur.wait_event(ev["vision"])
+        self._segment_compress()
+        down.wait_stream(cur)
+        with torch.cuda.stream(down):
+            self.d2h["out_feats"].copy_(o["cv"]["out_feats"][: self.n_out], non_blocking=True)
+            self.d2h["out_src"].copy_(o["cv"]["out_src"][: self.n_out], non_blocking=True)
+            self.d2h["offsets"].copy_(o["seg"]["event_offsets"], non_blocking=True)
         for i, s in enumerate(self.stages):
-            self.d2h[f"keep{i}"].copy_(o[f"pf{i}"]["keep_idx"][: s["S_out"]], non_blocking=True)
-            self.d2h[f"hidden{i}"].copy_(o[f"pf{i}"]["hidden_out"][: s["S_out"]], non_blocking=True)
-        for l in range(self.kv_layers):
-            self.d2h["kv_k"][l].copy_(self.ks[l][:, : self.kv_new], non_blocking=True)
-            self.d2h["kv_v"][l].copy_(self.vs[l][:, : self.kv_new], non_blocking=True)
+            cur.wait_event(ev[i + 1])
+            self._prefill_level(i)
+            down.wait_stream(cur)
+            with torch.cuda.stream(down):
+                self.d2h[f"keep{i}"].copy_(o[f"pf{i}"]["keep_idx"][: s["S_out"]], non_blocking=True)
+                self.d2h[f"hidden{i}"].copy_(o[f"pf{i}"]["hidden_out"][: s["S_out"]], non_blocking=True)
+        cur.wait_event(ev["kv"])
+        self._kv_call()
+        down.wait_stream(cur)
+        with torch.cuda.stream(down):
+            for l in range(self.kv_layers):
+                self.d2h["kv_k"][l].copy_(self.ks[l][:, : self.kv_new], non_blocking=True)
+                self.d2h["kv_v"][l].copy_(self.vs[l][:, : self.kv_new], non_blocking=True)
+        self.consumed = cur.record_event()
+        cur.wait_stream(down)                 # the step ends when the last result is on the host
 
     def stage_work(self):
         """Algorithmic work of one video per step of the path: what the method has to move or compute

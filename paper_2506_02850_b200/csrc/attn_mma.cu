@@ -152,13 +152,12 @@ attn_stats_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 for (int kb = 0; kb < KB; ++kb)
                     tma_load_2d(k_addr(s) + kb * kKBlk, &tmK, kb * 64, g * dm.S + (t_lo + it) * kStBN, fb);
             }
-            if (!ok) {
-                // let the copies already issued land before the CTA's shared memory goes away
-                mbar_wait(smem_u32(&q_bar), 0u, abort_flag);
-                for (int back = 1; back <= kStStages && back <= it; ++back) {
-                    const int j = it - back;
-                    mbar_wait(smem_u32(&full_bar[j % kStStages]), (uint32_t)(j / kStStages) & 1u, abort_flag);
-                }
+            // every copy issued has landed before the CTA's shared memory goes away, whichever way the
+            // other warps leave (in a normal run these waits are over already)
+            mbar_wait(smem_u32(&q_bar), 0u, abort_flag);
+            for (int back = 1; back <= kStStages && back <= it; ++back) {
+                const int j = it - back;
+                mbar_wait(smem_u32(&full_bar[j % kStStages]), (uint32_t)(j / kStStages) & 1u, abort_flag);
             }
         }
     } else if (warp == 1) {
@@ -349,12 +348,10 @@ attn_colsum_mma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 for (int kb = 0; kb < KB; ++kb)
                     tma_load_2d(k_addr(s) + kb * kKBlk, &tmK, kb * 64, g * dm.S + (t_lo + it) * kCsBM, fb);
             }
-            if (!ok) {
-                mbar_wait(smem_u32(&q_bar), 0u, abort_flag);
-                for (int back = 1; back <= kCsStages && back <= it; ++back) {
-                    const int j = it - back;
-                    mbar_wait(smem_u32(&full_bar[j % kCsStages]), (uint32_t)(j / kCsStages) & 1u, abort_flag);
-                }
+            mbar_wait(smem_u32(&q_bar), 0u, abort_flag);         // as in the stats kernel
+            for (int back = 1; back <= kCsStages && back <= it; ++back) {
+                const int j = it - back;
+                mbar_wait(smem_u32(&full_bar[j % kCsStages]), (uint32_t)(j / kCsStages) & 1u, abort_flag);
             }
         }
     } else if (warp == 1) {

@@ -21,10 +21,14 @@ Conventions
 Pins: every function below is pinned in tests/test_oracle_*.py against planted
 structure, closed forms, brute force on tiny inputs, independent float64
 restatements with library routines, constants printed in the paper, and
-invariants.  One value is not fixed by anything external: which of two key
-tokens wins a merge assignment when their cosines differ by less than 1e-3
-relative -- "parity unpinned" inside that band (the lower-index rule makes the
-oracle's own answer unique).
+invariants; none is left unpinned.  The oracle's answers are unique (exact
+float64 arithmetic on the inputs, lower index on exact ties).  What the GPU
+comparison tolerates is a separate matter: where the deciding gap of an index
+decision is below 1e-3 relative (a score against its top-k threshold, the best
+against the second-best cosine of a merge assignment) the kernel's bf16 / fp32
+rounding may decide the other way; ``near_threshold`` and the ``margin`` of
+``merge_assign`` report those cases (both pinned by construction), and the
+parity tests count them against ceilings.
 """
 
 from __future__ import annotations

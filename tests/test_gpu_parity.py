@@ -860,3 +860,49 @@ def test_benchmark_launch_configuration_equals_eager_calls_at_full_size():
             assert same(w.ks[layer][:, :m], ref.ks[layer][:, :m]) and same(w.vs[layer][:, :m], ref.vs[layer][:, :m])
     del graph, lanes_w, ref
     torch.cuda.empty_cache()
+
+
+# ------------------------------------------------- random shapes, all calls ---- #
+
+@pytest.mark.parametrize("seed", list(range(32)))
+def test_random_shapes_through_all_calls(seed):
+    """Seeded random small shapes, ratios, modes and types through segmentation, both compressors and
+    the pruning call: shapes nobody picked by hand (odd head counts, row lengths on and off the
+    tensor-core paths, classes without members, budgets of zero and above the population)."""
+    rng = np.random.default_rng(9000 + seed)
+    dtype = "bf16" if rng.random() < 0.6 else "f32"
+    T = int(rng.integers(1, 33))
+    Gs = int(rng.integers(1, 9))
+    N = Gs * Gs
+    d = int(rng.integers(1, 40)) * 8
+    k = int(rng.integers(1, T + 1))
+    cuts = np.sort(rng.choice(np.arange(1, T), size=k - 1, replace=False)) if k > 1 else np.zeros(0, np.int64)
+    offs = np.concatenate([[0], cuts, [T]]).astype(np.int32)
+    base = rng.standard_normal((k, N, d))
+    V = np.concatenate([base[e][None] + 0.4 * rng.standard_normal((offs[e + 1] - offs[e], N, d)) for e in range(k)])
+    V = W.quantize(V.astype(np.float32), dtype)
+    t = W.quantize(rng.standard_normal(d).astype(np.float32), dtype)
+    for mode in (O.SIM_FLATTEN, O.SIM_MEANPOOL):
+        R.segment_case(V, dtype, k, mode)
+    alpha = float(rng.choice([0.25, 0.5, 0.75, 1.0]))
+    kk, kn = float(rng.choice([0.02, 0.1, 0.3, 0.6, 1.0])), float(rng.choice([0.01, 0.05, 0.2, 0.5]))
+    agg = int(rng.integers(0, 2))
+    R.compress_case(V, t, offs, dtype, alpha, kk, kn, agg)
+    strides = tuple(int(x) for x in rng.integers(1, Gs + 2, size=4))
+    R.pool_case(V, t, offs, dtype, alpha, float(rng.choice([0.2, 0.5, 1.0])), strides, agg)
+
+    Hkv = int(rng.integers(1, 4))
+    Hq = Hkv * int(rng.integers(1, 5))
+    Lt = int(rng.integers(1, 40))
+    dh = int(rng.choice([64, 128])) if dtype == "bf16" else int(rng.choice([20, 32, 64, 128]))   # bf16 heads: 64 or 128 only
+    n_vis = int(rng.integers(1, 3000))
+    vis_start = int(rng.integers(0, 20))
+    G = int(rng.integers(1, 6))
+    S = vis_start + n_vis + int(rng.integers(0, 4)) + Lt
+    Q = W.quantize(rng.standard_normal((Hq, Lt, dh)).astype(np.float32), dtype)
+    K = W.quantize(rng.standard_normal((Hkv, S, dh)).astype(np.float32), dtype)
+    groups = rng.integers(0, G + 1, size=n_vis).astype(np.int32)
+    groups[groups == G] = int(rng.integers(0, G))               # some class may end up without members
+    budgets = [int(rng.integers(0, n_vis // G + 3)) for _ in range(G)]
+    hidden = W.payload_torch(7 + seed, S, 8 * int(rng.integers(1, 20)), dtype, "cuda")
+    R.prefill_case(Q, K, dtype, vis_start, n_vis, groups, budgets, float(dh) ** -0.5, hidden)

@@ -906,3 +906,18 @@ def test_random_shapes_through_all_calls(seed):
     budgets = [int(rng.integers(0, n_vis // G + 3)) for _ in range(G)]
     hidden = W.payload_torch(7 + seed, S, 8 * int(rng.integers(1, 20)), dtype, "cuda")
     R.prefill_case(Q, K, dtype, vis_start, n_vis, groups, budgets, float(dh) ** -0.5, hidden)
+
+
+@pytest.mark.parametrize("seed", list(range(16)))
+def test_random_kv_caches(seed):
+    """Seeded random cache shapes, ratios and policies through the K/V selection and in-place gather."""
+    import dataclasses
+    rng = np.random.default_rng(7000 + seed)
+    cfg = dataclasses.replace(
+        W.CONFIGS["tiny"], name=f"rand{seed}", index=100 + seed, T=int(rng.integers(1, 40)), N=int(rng.integers(1, 60)),
+        dtype="bf16" if rng.random() < 0.6 else "f32", Hkv=int(rng.integers(1, 5)),
+        dh=int(rng.choice([8, 32, 64, 128])), L=int(rng.integers(1, 7)),
+        keep_kv=float(rng.choice([0.0, 0.01, 0.065, 0.3, 0.8, 1.0])), kv_text=int(rng.integers(0, 30)))
+    policy = [O.KV_TOPK, O.KV_PAPER, O.KV_GIVEN][seed % 3]
+    R.kv_case(cfg, policy, per_layer_scores=bool(seed & 4), l1=int(rng.integers(0, cfg.L + 1)), sample_slabs=4,
+              given_from=seed)

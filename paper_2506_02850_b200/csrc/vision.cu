@@ -1,5 +1,6 @@
 // metok_compress_vision: text relevance and key events (Eq. 5), per-event key-token
 // top-k, merge-assign of the remaining tokens and averaging.
+#include <algorithm>
 #include <cstdlib>
 
 #include "common.cuh"
@@ -864,7 +865,8 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
                     int32_t* __restrict__ long_index, int32_t* __restrict__ long_slot,
                     int32_t* __restrict__ long_counter, int long_threshold, int long_cap,
                     int32_t* __restrict__ few_members, int few_cap, int32_t* __restrict__ heavy_index,
-                    int32_t* __restrict__ heavy_slot, int32_t* __restrict__ heavy_counter, int heavy_cap,
+                    int32_t* __restrict__ heavy_slot, int32_t* __restrict__ heavy_counter, int heavy_threshold,
+                    int heavy_cap,
                     const int32_t* __restrict__ n_out) {
     grid_dep_wait();
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
@@ -886,7 +888,7 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
     // scratch an output gets depends on arrival order, what is computed in it does not)
     const int pos = atomicAdd(&slot_cnt[slot], 1);
     if (pos < few_cap) few_members[(size_t)slot * few_cap + pos] = row;   // the first few_cap arrivals are listed
-    if (pos == few_cap) {                                     // more than that: an output to be started early
+    if (pos == heavy_threshold) {                             // many members: an output to be started early
         const int hh = atomicAdd(heavy_counter, 1);
         heavy_index[slot] = hh;
         if (hh < heavy_cap) heavy_slot[hh] = slot;
@@ -911,24 +913,32 @@ merge_decode_kernel(const unsigned long long* __restrict__ best64, const uint8_t
 constexpr int kAvgThreads = 128;
 constexpr int kAvgChunks = 4;      // 16-byte chunks per thread per pass over d
 constexpr int kAvgQuads = 5;       // 16-byte groups of `assign` per thread and pass
-constexpr int kAvgStages = 3;      // member rows in flight
+constexpr int kAvgStages = 3;      // member rows in flight when a pass over a row fills a stage (more than 4 KiB); the same
+                                   // bytes hold 6 or 12 shorter rows (template parameter NST of the kernel)
 constexpr int kAvgList = 512;      // members listed at a time
 constexpr int kAvgStageBytes = kAvgThreads * kAvgChunks * 16;
 constexpr size_t kAvgSmemBytes = (size_t)kAvgStages * kAvgStageBytes + 128;
-constexpr int kAvgFew = 16;        // outputs with at most this many members get them listed by merge_decode
-constexpr int kAvgLong = 32;       // outputs with more members than this are split ...
+constexpr int kAvgFew = 32;        // outputs with at most this many members get them listed by merge_decode (a warp ranks them)
+constexpr int kAvgHeavy = 16;      // outputs with more members than this are listed to be started first
+constexpr int kAvgLong = 32;       // outputs with more members than this (= kAvgFew: the others need no search) are split ...
 constexpr int kAvgParts = 8;       // ... over up to this many CTAs (fp32 partial sums, added in part order)
-constexpr int kAvgLongCap = 256;   // long outputs that get scratch for their partial sums
-constexpr int kAvgHeavyCap = 2048;  // outputs with more than kAvgFew members that are listed to be started first
+constexpr int kAvgLongCapMax = 1024;   // most long outputs that get scratch for their partial sums ...
+constexpr size_t kAvgLongBytes = (size_t)32 << 20;   // ... within this much scratch
+constexpr int kAvgHeavyCap = 2048;  // outputs with more than kAvgHeavy members that are listed to be started first
 constexpr int kAvgFrontCtas = 8 * kNumSMs;   // CTAs at the front of the grid that take the listed outputs and parts
-// parts of an output with `count` > kAvgLong members: about eight members each
+// long outputs that get scratch: as many as kAvgLongBytes hold (kAvgParts rows of d floats each)
+__host__ __device__ inline int avg_long_cap(int d) {
+    const long long c = (long long)(kAvgLongBytes / ((size_t)kAvgParts * (size_t)d * sizeof(float)));
+    return (int)(c < 64 ? 64 : c > kAvgLongCapMax ? kAvgLongCapMax : c);
+}
+// parts of an output with `count` > kAvgLong members: about eight members each if they lie evenly
 __host__ __device__ inline int avg_parts(int count) {
     const int p = (count + 7) / 8;
     return p < kAvgParts ? p : kAvgParts;
 }
 
-// One (output, part): the members of output c with ranks in this part's range, added in token order.
-template <typename T>
+// One (output, part): the members of output c in this part's share of the search, added in token order.
+template <typename T, int NST>
 __device__ __forceinline__ void
 merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_bar, int* s_list, int* s_wtot,
                int* s_blocks, int* s_abort_p, int* s_last_p,
@@ -949,21 +959,25 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
     const int count = slot_cnt[c];
     const bool few = count <= kAvgFew;
     int li = long_index[c];
-    if (li >= kAvgLongCap) li = -1;                            // no scratch left: one CTA does it all
+    if (li >= avg_long_cap(d)) li = -1;                        // no scratch left: one CTA does it all
     const int nparts = li >= 0 ? avg_parts(count) : 1;
-    const int per = (count + nparts - 1) / nparts;
-    const int r_lo = part * per, r_hi = min(count, r_lo + per);
     const int e = out_event[c];
     const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
     const int nchunk = d / VN;
     const int4* assign4 = reinterpret_cast<const int4*>(assign);
     const uint32_t stage0 = (smem_u32(avg_dyn) + 127u) & ~127u;
+    constexpr int nst = NST;
+    constexpr uint32_t stage_stride = (uint32_t)(kAvgStages * kAvgStageBytes) / NST;   // a pass over a row moves no more
     // the blocks to search, in order; a block is searched as bt/4 + 1 groups of four tokens (its
     // first token need not start a group)
     const unsigned long long blocks = slot_blocks[c];
     const int nblk = __popcll(blocks);
     const int bt = avg_block_tokens(hi - lo), qpb = bt / 4 + 1;
     const int total_q = nblk * qpb;
+    // a part takes an equal share of the groups to search (not of the members): what it finds there
+    // it adds up, so an output's search is done once however many parts it has
+    const int q_per = (total_q + nparts - 1) / nparts;
+    const int q_begin = min(total_q, part * q_per), q_end = min(total_q, q_begin + q_per);
     if (few) {
         if (warp == 0) {                                       // into token order: rank = members before it
             const int mine = lane < count ? few_tok : 0x7FFFFFFF;
@@ -982,26 +996,26 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
         float acc[kAvgChunks][VN];
 #pragma unroll
         for (int u = 0; u < kAvgChunks; ++u) Vec16<T>::zero(acc[u]);
-        // the listed members' rows, kAvgStages in flight, added in list order
+        // the listed members' rows, nst in flight, added in list order
         auto consume = [&](int nlist) {
-        // a ring: row m goes to stage m % kAvgStages; the stage is refilled with row m + kAvgStages as
-        // soon as every thread has added row m, so kAvgStages rows stay in flight until the list ends
+        // a ring: row m goes to stage m % nst; the stage is refilled with row m + nst as
+        // soon as every thread has added row m, so nst rows stay in flight until the list ends
         auto issue = [&](int m) {
-            const int j = m % kAvgStages;
+            const int j = m % nst;                             // nst is a constant: no division
             const uint32_t bar = smem_u32(&s_bar[j]);
             mbar_arrive_expect_tx(bar, seg_bytes);
             const long long src_row = dbg_bound(s_list[m], Nv, status);
             if (!(dbg_withhold(status, kDbgMergeAvg) && blockIdx.x == (unsigned)kAvgFrontCtas && m == 0 && cb == 0))   // debug builds: one copy never sent
-                bulk_load(stage0 + (uint32_t)j * kAvgStageBytes, feats + (size_t)src_row * d + (size_t)cb * VN, seg_bytes, bar);
+                bulk_load(stage0 + (uint32_t)j * stage_stride, feats + (size_t)src_row * d + (size_t)cb * VN, seg_bytes, bar);
         };
         if (tid == 0)
-            for (int m = 0; m < nlist && m < kAvgStages; ++m) issue(m);
+            for (int m = 0; m < nlist && m < nst; ++m) issue(m);
         for (int m = 0; m < nlist; ++m) {
-            const int j = m % kAvgStages;
+            const int j = m % nst;
             const bool ok = mbar_wait(smem_u32(&s_bar[j]), (phase >> j) & 1u, abort_flag);
             phase ^= 1u << j;
             if (ok) {
-                const uint8_t* row = avg_dyn + (stage0 - smem_u32(avg_dyn)) + (size_t)j * kAvgStageBytes;
+                const uint8_t* row = avg_dyn + (stage0 - smem_u32(avg_dyn)) + (size_t)j * stage_stride;
 #pragma unroll
                 for (int u = 0; u < kAvgChunks; ++u) {
                     const int ch = cb + u * kAvgThreads + tid;
@@ -1025,17 +1039,15 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
                 }
             }
             __syncthreads();                                   // every thread is done with stage j
-            if (tid == 0 && m + kAvgStages < nlist && !*abort_flag) issue(m + kAvgStages);
+            if (tid == 0 && m + nst < nlist && !*abort_flag) issue(m + nst);
         }
         };
         if (few) {
             consume(count);                                    // s_list holds them already
         } else {
-        int seen = 0;                                          // members met in earlier passes
-        // a thread's run is qpt consecutive groups: as few as cover the search in one pass (most
-        // outputs have a handful of groups: one each for the first threads, nothing for the rest)
-        const int qpt = min(kAvgQuads, (total_q + kAvgThreads - 1) / kAvgThreads);
-        for (int qs = 0; qs < total_q && seen < r_hi; qs += kAvgThreads * qpt) {
+        // a thread's run is qpt consecutive groups: as few as cover the search in one pass
+        const int qpt = max(1, min(kAvgQuads, (q_end - q_begin + kAvgThreads - 1) / kAvgThreads));
+        for (int qs = q_begin; qs < q_end; qs += kAvgThreads * qpt) {
             int4 a[kAvgQuads];
             int qidx[kAvgQuads], j_lo[kAvgQuads], j_hi[kAvgQuads];   // group index; the block's token range
 #pragma unroll
@@ -1043,7 +1055,7 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
                 const int qf = qs + tid * qpt + u;
                 a[u] = make_int4(-1, -1, -1, -1);
                 qidx[u] = 0; j_lo[u] = 0; j_hi[u] = 0;
-                if (u < qpt && qf < total_q) {
+                if (u < qpt && qf < q_end) {
                     const int bi = qf / qpb, wq = qf - bi * qpb;
                     const int st = lo + s_blocks[bi] * bt;
                     const int q = (st >> 2) + wq;
@@ -1076,17 +1088,16 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
             }
             if (lane == 31) s_wtot[warp] = incl;
             __syncthreads();
-            int before = seen + incl - mine, total = 0;        // rank of this thread's first member
+            int before = incl - mine, total = 0;               // rank of this thread's first member in the pass
 #pragma unroll
             for (int w = 0; w < kAvgThreads / 32; ++w) {
                 const int v = s_wtot[w];
                 if (w < warp) before += v;
                 total += v;
             }
-            // this part's ranks among the members of the pass, listed kAvgList at a time
-            const int b_lo = max(r_lo, seen), b_hi = min(r_hi, seen + total);
-            for (int b0 = b_lo; b0 < b_hi; b0 += kAvgList) {
-                const int nlist = min(kAvgList, b_hi - b0);
+            // the members of the pass, listed kAvgList at a time
+            for (int b0 = 0; b0 < total; b0 += kAvgList) {
+                const int nlist = min(kAvgList, total - b0);
                 {
                     unsigned mm = match;
                     int r = before;
@@ -1100,7 +1111,6 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
                 __syncthreads();
                 consume(nlist);
             }
-            seen += total;
             __syncthreads();                                   // s_wtot and s_list are reused by the next pass
         }
         }
@@ -1162,7 +1172,7 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
     }
 }
 
-template <typename T>
+template <typename T, int NST>
 __global__ void __launch_bounds__(kAvgThreads, 8)
 merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
                  const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
@@ -1176,40 +1186,42 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
     grid_dep_wait();
     using namespace sm100;
     extern __shared__ uint8_t avg_dyn[];
-    __shared__ __align__(8) uint64_t s_bar[kAvgStages];
+    __shared__ __align__(8) uint64_t s_bar[NST];
     __shared__ int s_list[kAvgList];
     __shared__ int s_wtot[kAvgThreads / 32];
     __shared__ int s_blocks[64];
     __shared__ int s_abort, s_last;
     // A CTA adds the rows of its output about three at a time, one memory latency per three rows:
     // an output with many members lasts many times longer than the usual one, and would set the
-    // kernel's time if it started late.  So merge_decode lists every output with more than kAvgFew
+    // kernel's time if it started late.  So merge_decode lists every output with more than kAvgHeavy
     // members, and the first front_ctas CTAs of the grid take the listed work round-robin, before the
     // other outputs' CTAs start: the outputs with more than kAvgLong members part by part (up to
-    // kAvgParts parts of about eight members, partial sums combined in part order by the last part
-    // to finish), the others whole.  A listed output's own CTA leaves at once.  The other CTAs start
+    // kAvgParts parts, each an equal share of the blocks to search, partial sums combined in part
+    // order by the last part to finish), the others whole (their members are listed: no search).
+    // A listed output's own CTA leaves at once.  The other CTAs start
     // in index order and take the outputs from the last one down, so that this pass begins with the
     // rows of V that the preceding (ascending) pass left in L2.
     const int tid = threadIdx.x;
+    const int long_cap = avg_long_cap(d);
     if (tid == 32) {                                           // not thread 0: it is busy with the block list below
-        for (int j = 0; j < kAvgStages; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
+        for (int j = 0; j < NST; ++j) mbar_init(smem_u32(&s_bar[j]), 1);
         s_abort = 0;
         mbar_fence_init();
     }
     uint32_t phase = 0;                                        // bit j: parity of the next completion of barrier j
 #define METOK_AVG_ITEM(C, PART)                                                                                     \
-    merge_avg_item<T>(C, PART, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,  \
+    merge_avg_item<T, NST>(C, PART, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,  \
                       ev_lo, out_event, assign, slot_blocks, slot_cnt, long_index, few_members, long_sums, long_done,  \
                       out_feats, out_members, status)
     if ((int)blockIdx.x >= front_ctas) {
         const int c = *n_out - 1 - ((int)blockIdx.x - front_ctas);
         if (c < 0) return;
         const int hh = heavy_index[c], ll = long_index[c];
-        if ((hh >= 0 && hh < kAvgHeavyCap) || (ll >= 0 && ll < kAvgLongCap)) return;   // listed: the front CTAs have it
+        if ((hh >= 0 && hh < kAvgHeavyCap) || (ll >= 0 && ll < long_cap)) return;   // listed: the front CTAs have it
         METOK_AVG_ITEM(c, 0);
         return;
     }
-    const int n_long = min(*long_counter, kAvgLongCap), n_heavy = min(*heavy_counter, kAvgHeavyCap);
+    const int n_long = min(*long_counter, long_cap), n_heavy = min(*heavy_counter, kAvgHeavyCap);
     const int n_items = n_long * kAvgParts + n_heavy;
     for (int it = (int)blockIdx.x; it < n_items; it += front_ctas) {
         int c, part;
@@ -1221,7 +1233,7 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
             c = heavy_slot[it - n_long * kAvgParts];
             part = 0;
             const int li = long_index[c];
-            if (li >= 0 && li < kAvgLongCap) continue;         // split into parts: taken above
+            if (li >= 0 && li < long_cap) continue;            // split into parts: taken above
         }
         METOK_AVG_ITEM(c, part);
         __syncthreads();                                       // the shared lists are reused by the next item
@@ -1245,7 +1257,7 @@ struct VisionWs {
     int32_t* long_done;                // ... parts of each that have finished
     int32_t* long_index;               // output -> index among the long ones, -1 otherwise
     int32_t* long_slot;                // and back
-    int32_t* heavy_counter;            // outputs with more than kAvgFew members ...
+    int32_t* heavy_counter;            // outputs with more than kAvgHeavy members ...
     int32_t* heavy_index;              // ... output -> index among them, -1 otherwise (directly after long_index)
     int32_t* heavy_slot;               // ... and back
     int32_t* few_members;              // per output token: its first kAvgFew members, in arrival order
@@ -1269,19 +1281,19 @@ static VisionWs carve_vision(Carver& cv, int Tn, int N, int k, int d, int cap, b
     w.best64 = mma ? cv.take<unsigned long long>((size_t)Tn * N) : nullptr;
     {
         const size_t n = (size_t)cap + 64;
-        w.zero_bytes = n * 8 + n * 4 + (size_t)(64 + kAvgLongCap + 64) * 4;
+        w.zero_bytes = n * 8 + n * 4 + (size_t)(64 + kAvgLongCapMax + 64) * 4;
         unsigned char* z = cv.take<unsigned char>(w.zero_bytes);
         w.slot_blocks = reinterpret_cast<unsigned long long*>(z);
         w.slot_cnt = reinterpret_cast<int32_t*>(z + n * 8);
         w.long_counter = w.slot_cnt + n;
         w.long_done = w.long_counter + 64;
-        w.heavy_counter = w.long_done + kAvgLongCap;
+        w.heavy_counter = w.long_done + kAvgLongCapMax;
         w.long_index = cv.take<int32_t>(2 * n);         // long_index, then heavy_index: filled with -1 together
         w.heavy_index = w.long_index + n;
         w.heavy_slot = cv.take<int32_t>(kAvgHeavyCap);
-        w.long_slot = cv.take<int32_t>(kAvgLongCap);
+        w.long_slot = cv.take<int32_t>(kAvgLongCapMax);
         w.few_members = cv.take<int32_t>(n * kAvgFew);
-        w.long_sums = cv.take<float>((size_t)kAvgLongCap * kAvgParts * d);
+        w.long_sums = cv.take<float>((size_t)avg_long_cap(d) * kAvgParts * d);
     }
     return w;
 }
@@ -1424,23 +1436,29 @@ static int launch_vision(const void* feats_, int Tn, int N, int d, const int32_t
         METOK_TIMED("merge_decode_kernel", st);
         launch_chained(merge_decode_kernel, dim3(ceil_div(Nv, 256)), dim3(256), 0, st, mma ? w.best64 : nullptr, w.is_key, Nv, N, w.ev_lo, k,
                                                                assign, w.slot_blocks, w.slot_cnt, w.long_index,
-                                                               w.long_slot, w.long_counter, kAvgLong, kAvgLongCap,
+                                                               w.long_slot, w.long_counter, kAvgLong, avg_long_cap(d),
                                                                w.few_members, kAvgFew, w.heavy_index, w.heavy_slot,
-                                                               w.heavy_counter, kAvgHeavyCap, n_out);
+                                                               w.heavy_counter, kAvgHeavy, kAvgHeavyCap, n_out);
     }
     METOK_LAUNCH_CHECK();
-    METOK_CUDA_TRY(cudaFuncSetAttribute(merge_avg_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)kAvgSmemBytes));
-    {
-        METOK_TIMED("merge_avg_kernel", st);
-        launch_chained(merge_avg_kernel<T>, dim3(kAvgFrontCtas + cap), dim3(kAvgThreads), kAvgSmemBytes, st, 
-            feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
-            w.long_counter, w.few_members, w.heavy_index, w.heavy_slot, w.heavy_counter, w.long_sums, w.long_done,
-            kAvgFrontCtas, n_out, out_feats, out_members,
-            w.status);
-    }
-    METOK_LAUNCH_CHECK();
-    return METOK_OK;
+    // rows in flight per CTA: a pass over a row moves at most seg0 bytes, the ring holds 24 KiB
+    const uint32_t seg0 = (uint32_t)std::min<long long>(kAvgThreads * kAvgChunks, (long long)d * sizeof(T) / 16) * 16u;
+    auto launch = [&](auto kernel) -> int {
+        METOK_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAvgSmemBytes));
+        {
+            METOK_TIMED("merge_avg_kernel", st);
+            launch_chained(kernel, dim3(kAvgFrontCtas + cap), dim3(kAvgThreads), kAvgSmemBytes, st,
+                feats, d, N, Nv, w.ev_lo, out_event, assign, w.slot_blocks, w.slot_cnt, w.long_index, w.long_slot,
+                w.long_counter, w.few_members, w.heavy_index, w.heavy_slot, w.heavy_counter, w.long_sums, w.long_done,
+                kAvgFrontCtas, n_out, out_feats, out_members,
+                w.status);
+        }
+        METOK_LAUNCH_CHECK();
+        return METOK_OK;
+    };
+    if (seg0 > (uint32_t)kAvgStageBytes / 2) return launch(merge_avg_kernel<T, kAvgStages>);
+    if (seg0 > (uint32_t)kAvgStageBytes / 4) return launch(merge_avg_kernel<T, 2 * kAvgStages>);
+    return launch(merge_avg_kernel<T, 4 * kAvgStages>);
 }
 
 }  // namespace metok

@@ -126,12 +126,16 @@ def _normal_prefill(args):
     return _with_normal_library(lambda: B.metok_prefill_prune(*args))
 
 
-@pytest.mark.parametrize("case", ["tiny", "frames32", "ragged"])
+@pytest.mark.parametrize("case", ["tiny", "frames32", "ragged", "long_lists"])
 def test_no_index_leaves_its_range(debug_lib, case):
     """Word 2 of the status area counts out-of-range row / slot indices met by the range-checked build."""
     if case == "ragged":
         Vd, offs, td, p = _vision_case(seed=9, T=7, N=37, d=72)
         offs = torch.tensor([0, 1, 2, 10], dtype=torch.int32).cuda()             # ten frames: events of 1, 1 and 8
+    elif case == "long_lists":
+        # 640 tokens and a handful of key tokens: member lists of a hundred and more, split into parts
+        Vd, offs, td, _ = _vision_case(seed=12, T=10, N=64, d=136)
+        p = B.vision_params(0.5, 0.006, 0.006)
     else:
         cfg = W.CONFIGS[case]
         vis = W.vision_inputs(cfg)
@@ -145,7 +149,7 @@ def test_no_index_leaves_its_range(debug_lib, case):
     words = B.workspace(1, Vd.device)[:16].view(torch.int32)
     assert int(words[0].item()) == 0 and int(words[2].item()) == 0
     _vision_equal(got, _normal_vision(Vd, offs, td, p))
-    args = _prefill_case(seed=11, n_vis=777 if case == "ragged" else 1500)
+    args = _prefill_case(seed=11, n_vis=777 if case in ("ragged", "long_lists") else 1500)
     pf = B.metok_prefill_prune(*args)
     torch.cuda.synchronize()
     words = B.workspace(1, Vd.device)[:16].view(torch.int32)

@@ -938,9 +938,30 @@ __host__ __device__ inline int avg_parts(int count) {
 }
 
 // One (output, part): the members of output c in this part's share of the search, added in token order.
+// What a CTA needs to know about its output before it can fetch a row; the loads are independent of
+// one another, so a caller issues them together with whatever else it has to look up about the output.
+struct AvgMeta {
+    int count, few_tok, li, e;
+    unsigned long long blocks;
+};
+__device__ __forceinline__ AvgMeta avg_meta(int c, const int32_t* __restrict__ slot_cnt,
+                                            const int32_t* __restrict__ few_members,
+                                            const int32_t* __restrict__ long_index,
+                                            const int32_t* __restrict__ out_event,
+                                            const unsigned long long* __restrict__ slot_blocks) {
+    AvgMeta m;
+    const int lane = threadIdx.x & 31;
+    m.few_tok = lane < kAvgFew ? few_members[(size_t)c * kAvgFew + lane] : 0;
+    m.count = slot_cnt[c];
+    m.li = long_index[c];
+    m.e = out_event[c];
+    m.blocks = slot_blocks[c];
+    return m;
+}
+
 template <typename T, int NST>
 __device__ __forceinline__ void
-merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_bar, int* s_list, int* s_wtot,
+merge_avg_item(int c, int part, const AvgMeta& meta, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_bar, int* s_list, int* s_wtot,
                int* s_blocks, int* s_abort_p, int* s_last_p,
                const T* __restrict__ feats, int d, int N, int Nv, const int32_t* __restrict__ ev_lo,
                const int32_t* __restrict__ out_event, const int32_t* __restrict__ assign,
@@ -955,13 +976,13 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
     int& s_last = *s_last_p;
     // an output with at most kAvgFew members has them listed by merge_decode (in arrival order):
     // fetched together with the output's other data, no search of `assign`
-    const int few_tok = lane < kAvgFew ? few_members[(size_t)c * kAvgFew + lane] : 0;
-    const int count = slot_cnt[c];
+    const int few_tok = meta.few_tok;
+    const int count = meta.count;
     const bool few = count <= kAvgFew;
-    int li = long_index[c];
+    int li = meta.li;
     if (li >= avg_long_cap(d)) li = -1;                        // no scratch left: one CTA does it all
     const int nparts = li >= 0 ? avg_parts(count) : 1;
-    const int e = out_event[c];
+    const int e = meta.e;
     const int lo = ev_lo[e] * N, hi = ev_lo[e + 1] * N;
     const int nchunk = d / VN;
     const int4* assign4 = reinterpret_cast<const int4*>(assign);
@@ -970,7 +991,7 @@ merge_avg_item(int c, int part, uint32_t& phase, uint8_t* avg_dyn, uint64_t* s_b
     constexpr uint32_t stage_stride = (uint32_t)(kAvgStages * kAvgStageBytes) / NST;   // a pass over a row moves no more
     // the blocks to search, in order; a block is searched as bt/4 + 1 groups of four tokens (its
     // first token need not start a group)
-    const unsigned long long blocks = slot_blocks[c];
+    const unsigned long long blocks = meta.blocks;
     const int nblk = __popcll(blocks);
     const int bt = avg_block_tokens(hi - lo), qpb = bt / 4 + 1;
     const int total_q = nblk * qpb;
@@ -1209,16 +1230,18 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
         mbar_fence_init();
     }
     uint32_t phase = 0;                                        // bit j: parity of the next completion of barrier j
-#define METOK_AVG_ITEM(C, PART)                                                                                     \
-    merge_avg_item<T, NST>(C, PART, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,  \
+#define METOK_AVG_ITEM(C, PART, META)                                                                                     \
+    merge_avg_item<T, NST>(C, PART, META, phase, avg_dyn, s_bar, s_list, s_wtot, s_blocks, &s_abort, &s_last, feats, d, N, Nv,  \
                       ev_lo, out_event, assign, slot_blocks, slot_cnt, long_index, few_members, long_sums, long_done,  \
                       out_feats, out_members, status)
     if ((int)blockIdx.x >= front_ctas) {
         const int c = *n_out - 1 - ((int)blockIdx.x - front_ctas);
         if (c < 0) return;
-        const int hh = heavy_index[c], ll = long_index[c];
-        if ((hh >= 0 && hh < kAvgHeavyCap) || (ll >= 0 && ll < long_cap)) return;   // listed: the front CTAs have it
-        METOK_AVG_ITEM(c, 0);
+        // everything about output c in one round trip: whether it is listed, and what its own CTA needs if not
+        const int hh = heavy_index[c];
+        const AvgMeta meta = avg_meta(c, slot_cnt, few_members, long_index, out_event, slot_blocks);
+        if ((hh >= 0 && hh < kAvgHeavyCap) || (meta.li >= 0 && meta.li < long_cap)) return;   // listed: the front CTAs have it
+        METOK_AVG_ITEM(c, 0, meta);
         return;
     }
     const int n_long = min(*long_counter, long_cap), n_heavy = min(*heavy_counter, kAvgHeavyCap);
@@ -1235,7 +1258,8 @@ merge_avg_kernel(const T* __restrict__ feats, int d, int N, int Nv, const int32_
             const int li = long_index[c];
             if (li >= 0 && li < long_cap) continue;            // split into parts: taken above
         }
-        METOK_AVG_ITEM(c, part);
+        const AvgMeta meta = avg_meta(c, slot_cnt, few_members, long_index, out_event, slot_blocks);
+        METOK_AVG_ITEM(c, part, meta);
         __syncthreads();                                       // the shared lists are reused by the next item
     }
 #undef METOK_AVG_ITEM

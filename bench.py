@@ -44,31 +44,31 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # captures (profiles/), keyed by (scope/kernel, workload); a kernel changed since its capture is left out
 # (its stage then reports traffic null).
 NCU_TRAFFIC_BYTES = {
-    ("segment/seg_score_kernel", "frames128"): 137890048,
-    ("segment/seg_finish_kernel", "frames128"): 58880,
-    ("compress/event_plan_kernel", "frames128"): 131328,
+    ("segment/seg_score_kernel", "frames128"): 136371200,
+    ("segment/seg_finish_kernel", "frames128"): 58624,
+    ("compress/event_plan_kernel", "frames128"): 131584,
     ("compress/event_topk_kernel", "frames128"): 132352,
-    ("compress/merge_assign_mma_kernel", "frames128"): 136162816,
-    ("compress/merge_decode_kernel", "frames128"): 282112,
-    ("compress/merge_avg_kernel", "frames128"): 146935296,
-    ("prefill1/attn_stats_mma_kernel", "frames128"): 19439104,
+    ("compress/merge_assign_mma_kernel", "frames128"): 137563392,
+    ("compress/merge_decode_kernel", "frames128"): 279808,
+    ("compress/merge_avg_kernel", "frames128"): 147466752,
+    ("prefill1/attn_stats_mma_kernel", "frames128"): 19438592,
     ("prefill1/attn_colsum_mma_kernel", "frames128"): 19495680,
     ("prefill1/attn_score_reduce_kernel", "frames128"): 1189120,
     ("prefill1/class_topk_kernel", "frames128"): 217856,
-    ("prefill1/gather_rows_kernel", "frames128"): 53465344,
-    ("prefill2/attn_stats_mma_kernel", "frames128"): 7494912,
-    ("prefill2/attn_colsum_mma_kernel", "frames128"): 7567872,
+    ("prefill1/gather_rows_kernel", "frames128"): 53984512,
+    ("prefill2/attn_stats_mma_kernel", "frames128"): 7494656,
+    ("prefill2/attn_colsum_mma_kernel", "frames128"): 7568128,
     ("prefill2/attn_score_reduce_kernel", "frames128"): 442880,
     ("prefill2/class_topk_kernel", "frames128"): 124928,
     ("prefill2/gather_rows_kernel", "frames128"): 15964672,
-    ("prefill3/attn_stats_mma_kernel", "frames128"): 2776064,
+    ("prefill3/attn_stats_mma_kernel", "frames128"): 2776576,
     ("prefill3/attn_colsum_mma_kernel", "frames128"): 2791936,
-    ("prefill3/attn_score_reduce_kernel", "frames128"): 147968,
-    ("prefill3/class_topk_kernel", "frames128"): 88064,
-    ("prefill3/gather_rows_kernel", "frames128"): 472832,
-    ("kv/class_topk_kernel", "frames128"): 140032,
-    ("kv/kv_stage_kernel", "frames128"): 4829184,
-    ("kv/kv_copy_kernel", "frames128"): 100760320,
+    ("prefill3/attn_score_reduce_kernel", "frames128"): 147456,
+    ("prefill3/class_topk_kernel", "frames128"): 87808,
+    ("prefill3/gather_rows_kernel", "frames128"): 473344,
+    ("kv/class_topk_kernel", "frames128"): 139776,
+    ("kv/kv_stage_kernel", "frames128"): 4828160,
+    ("kv/kv_copy_kernel", "frames128"): 100829184,
 }
 
 

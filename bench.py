@@ -3,7 +3,7 @@
 
 A "step" is one pass of the whole hot path over a batch of independent synthetic
 videos of the 128-frame workload (128 x 144 visual tokens, 28-layer 7B-shaped LLM;
-4 videos in flight by default, each on a stream of its own): event
+8 videos in flight by default, each on a stream of its own): event
 segmentation, stage-1 compression, the three prefill pruning levels at the
 sizes the Eq. 6/7 schedule implies, and the KV-cache compaction -- all through
 the C ABI.  `value` = visual tokens entering the path per second, inputs resident
@@ -622,7 +622,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the chained run and the run without planted relevance")
     ap.add_argument("--no-sustain", action="store_true",
                     help="time exactly --steps steps (for profiler captures, where a one-second region is thousands of launches)")
-    ap.add_argument("--videos", type=int, default=4,
+    ap.add_argument("--videos", type=int, default=8,
                     help="independent videos in flight per step, each on a stream of its own (a step = this batch)")
     ap.add_argument("--parts", default=",".join(PARTS),
                     help="comma-separated subset of the four calls (for profiler captures that should hold little "
